@@ -1,0 +1,294 @@
+"""Pins for the CPU oracle: everything here checks oracle/ against something that
+is not the oracle's own arithmetic (a library routine, a closed form, a brute-force
+sum written out separately, the paper's printed value, the event-by-event checker)."""
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as F
+
+from paper_1804_10727_b200.workloads import Layer, conv, POOL
+
+rng = np.random.default_rng(1234)
+
+
+def _rand_net(mode, layers, H, W, C0, S=2, bias=True, seed=0):
+    r = np.random.default_rng(seed)
+    if mode == "i8":
+        x = r.integers(-127, 128, size=(S, H, W, C0)).astype(np.int32)
+        x[r.random(x.shape) < 0.5] = 0
+    else:
+        x = r.standard_normal((S, H, W, C0))
+        if mode == "bf16":
+            x = torch.tensor(x, dtype=torch.float32).bfloat16().double().numpy()
+    ws, bs = [], []
+    for l in layers:
+        if l.kind != "conv":
+            ws.append(None); bs.append(None); continue
+        if mode == "i8":
+            ws.append(r.integers(-127, 128, size=(l.cout, l.kh, l.kw, l.cin)).astype(np.int32))
+            bs.append(r.integers(-500, 500, size=(l.cout,)).astype(np.int32) if bias else None)
+        else:
+            w = r.standard_normal((l.cout, l.kh, l.kw, l.cin)) * (2.0 / (l.cin * l.kh * l.kw)) ** 0.5
+            if mode == "bf16":
+                w = torch.tensor(w, dtype=torch.float32).bfloat16().double().numpy()
+            ws.append(w)
+            bs.append(r.standard_normal((l.cout,)) * 0.1 if bias else None)
+    return x, ws, bs
+
+
+def _torch_forward(mode, layers, x, ws, bs):
+    """Conventional inference with torch.nn.functional in float64 (exact for the integer nets)."""
+    a = torch.tensor(np.asarray(x, dtype=np.float64)).permute(0, 3, 1, 2)   # NCHW
+    convs = [i for i, l in enumerate(layers) if l.kind == "conv"]
+    for i, l in enumerate(layers):
+        if l.kind == "conv":
+            w = torch.tensor(np.asarray(ws[i], dtype=np.float64)).permute(0, 3, 1, 2)  # [Cout][Cin][Kh][Kw]
+            b = None if bs[i] is None else torch.tensor(np.asarray(bs[i], dtype=np.float64))
+            a = F.conv2d(a, w, b, stride=l.stride, padding=l.pad)
+            if l.relu:
+                a = F.relu(a)
+            if mode == "bf16" and i != convs[-1]:
+                a = a.float().bfloat16().double()       # float64 -> float32 is exact enough here? see test below
+            if mode == "i8":
+                ai = a.to(torch.int64)
+                if l.shift > 0:
+                    ai = torch.div(ai + (1 << (l.shift - 1)), 1 << l.shift, rounding_mode="floor")
+                a = ai.clamp(0 if l.relu else -127, 127).double()
+        else:
+            if a.shape[3] == 1:
+                a = F.max_pool2d(a, kernel_size=(2, 1), stride=(2, 1))
+            else:
+                a = F.max_pool2d(a, kernel_size=2, stride=2)
+    return a.permute(0, 2, 3, 1).numpy()
+
+
+NETS = {
+    "valid3": (conv(2, 4, 3), conv(4, 3, 3)),
+    "same_pool": (conv(3, 4, 3, pad=1), POOL, conv(4, 5, 3, pad=1), POOL),
+    "stride2": (conv(2, 4, 3, stride=2), conv(4, 4, 3, stride=1), POOL),
+    "stride2_pad": (conv(2, 3, 3, stride=2, pad=1), conv(3, 4, 3, stride=2, pad=1)),
+    "oned_k9": (conv(1, 4, 9, stride=2, one_d=True), conv(4, 5, 9, one_d=True)),
+    "oned_k3": (conv(1, 8, 3, one_d=True), conv(8, 8, 3, one_d=True), conv(8, 4, 3, one_d=True)),
+    "k5": (conv(2, 3, 5, stride=2, pad=2), conv(3, 2, 3)),
+    "norelu": (conv(2, 3, 3, relu=0), conv(3, 2, 3, relu=0)),
+}
+
+
+def _with_shifts(layers, s=7):
+    return tuple(Layer(**{**l.__dict__, "shift": s}) if l.kind == "conv" else l for l in layers)
+
+
+def _dims(name):
+    if name.startswith("oned"):
+        return 60, 1
+    return 17, 14
+
+
+# ---- P1: the library routine -------------------------------------------------------------------
+@pytest.mark.parametrize("name", list(NETS))
+@pytest.mark.parametrize("mode", ["f32", "bf16", "i8"])
+def test_matches_torch_functional(orc, name, mode):
+    layers = NETS[name]
+    if mode == "i8":
+        layers = _with_shifts(layers, 8)
+    H, W = _dims(name)
+    x, ws, bs = _rand_net(mode, layers, H, W, layers[0].cin, S=2, seed=hash(name) % 1000)
+    got = orc.forward(mode, layers, x, ws, bs)
+    want = _torch_forward(mode, layers, x, ws, bs)
+    assert got.shape == want.shape
+    if mode == "i8":
+        assert np.array_equal(got, want.astype(np.int32))
+    elif mode == "f32":
+        np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-12)
+    else:
+        # float32 conv results passed through bf16 on the torch side may hit a double-rounding
+        # tie that the oracle's direct rounding does not: allow a handful of 1-ulp deviations
+        close = np.isclose(got, want, rtol=1e-10, atol=1e-12)
+        assert close.mean() > 0.999
+        np.testing.assert_allclose(got, want, rtol=2.0 ** -6, atol=1e-6)
+
+
+# ---- P2: single-unit brute force ---------------------------------------------------------------
+def test_single_unit_brute_force(orc):
+    l = conv(3, 5, 3, stride=2, pad=1, relu=0)
+    x, ws, bs = _rand_net("f32", (l,), 11, 9, 3, S=1, seed=5)
+    got = orc.forward("f32", (l,), x, ws, bs)[0]
+    r = np.random.default_rng(0)
+    for _ in range(50):
+        oy, ox, co = r.integers(got.shape[0]), r.integers(got.shape[1]), r.integers(5)
+        acc = Fraction(float(bs[0][co]))
+        for ky in range(3):
+            for kx in range(3):
+                iy, ix = oy * 2 - 1 + ky, ox * 2 - 1 + kx
+                if 0 <= iy < 11 and 0 <= ix < 9:
+                    for ci in range(3):
+                        acc += Fraction(float(ws[0][co, ky, kx, ci])) * Fraction(float(x[0, iy, ix, ci]))
+        assert abs(float(acc) - got[oy, ox, co]) < 1e-12
+
+
+# ---- P4: closed forms --------------------------------------------------------------------------
+@pytest.mark.parametrize("stride,pad", [(1, 0), (1, 1), (2, 0), (2, 1)])
+def test_impulse_response_is_the_kernel(orc, stride, pad):
+    l = conv(2, 3, 3, stride=stride, pad=pad, relu=0)
+    H, W = 9, 8
+    _, ws, _ = _rand_net("f32", (l,), H, W, 2, S=1, bias=False, seed=3)
+    y0, x0, ci = 4, 3, 1
+    x = np.zeros((1, H, W, 2)); x[0, y0, x0, ci] = 1.0
+    got = orc.forward("f32", (l,), x, ws, None)[0]
+    for oy in range(got.shape[0]):
+        for ox in range(got.shape[1]):
+            ky, kx = y0 + pad - oy * stride, x0 + pad - ox * stride
+            for co in range(3):
+                want = ws[0][co, ky, kx, ci] if (0 <= ky < 3 and 0 <= kx < 3) else 0.0
+                assert got[oy, ox, co] == want
+
+
+def test_all_ones_counts_fan_in(orc):
+    layers = (conv(2, 3, 3, relu=0), conv(3, 2, 3, relu=0))
+    ws = [np.ones((3, 3, 3, 2)), np.ones((2, 3, 3, 3))]
+    x = np.ones((1, 8, 8, 2))
+    got = orc.forward("f32", layers, x, ws, None)
+    assert np.all(got == 18 * 27)
+    # with same padding, a corner unit sees only 2x2 taps
+    l = conv(2, 1, 3, pad=1, relu=0)
+    got = orc.forward("f32", (l,), x, [np.ones((1, 3, 3, 2))], None)[0]
+    assert got[0, 0, 0] == 8 and got[0, 3, 0] == 12 and got[3, 3, 0] == 18
+
+
+def test_linearity_and_positive_homogeneity(orc):
+    lin = NETS["norelu"]
+    x, ws, _ = _rand_net("f32", lin, 9, 9, 2, S=2, bias=False, seed=9)
+    y = np.random.default_rng(1).standard_normal(x.shape)
+    f = lambda v: orc.forward("f32", lin, v, ws, None)
+    np.testing.assert_allclose(f(2.5 * x - 0.5 * y), 2.5 * f(x) - 0.5 * f(y), rtol=1e-11, atol=1e-12)
+    rel = NETS["same_pool"]
+    x, ws, _ = _rand_net("f32", rel, 12, 12, 3, S=1, bias=False, seed=10)
+    g = lambda v: orc.forward("f32", rel, v, ws, None)
+    assert np.array_equal(g(4.0 * x), 4.0 * g(x))      # power of two: exact
+
+
+# ---- bf16 rounding and requantisation ----------------------------------------------------------
+def test_bf16_rounding_matches_torch_and_ties(orc):
+    v = torch.randn(20000, dtype=torch.float32) * torch.logspace(-20, 20, 20000, base=2.0)
+    want = v.bfloat16().double().numpy()
+    got = orc.round_bf16(v.double().numpy())
+    assert np.array_equal(got, want)
+    # ties go to the even neighbour; just above a tie goes up (a case float32 double rounding gets wrong)
+    assert orc.round_bf16(np.array([1 + 2.0 ** -8]))[0] == 1.0
+    assert orc.round_bf16(np.array([1 + 3 * 2.0 ** -8]))[0] == 1 + 2.0 ** -6
+    assert orc.round_bf16(np.array([1 + 2.0 ** -8 + 2.0 ** -40]))[0] == 1 + 2.0 ** -7
+    assert orc.round_bf16(np.array([-(1 + 2.0 ** -8 + 2.0 ** -40)]))[0] == -(1 + 2.0 ** -7)
+    assert orc.round_bf16(np.array([0.0]))[0] == 0.0
+
+
+def test_requant_matches_exact_rationals(orc):
+    r = np.random.default_rng(2)
+    c = r.integers(-200000, 200000, size=4000).astype(np.int32)
+    for shift in (0, 1, 4, 9):
+        for relu in (0, 1):
+            got = orc.requant(c, shift, relu)
+            for ci, gi in zip(c[:500], got[:500]):
+                q = Fraction(int(ci), 1 << shift)
+                v = int((q + Fraction(1, 2)).__floor__()) if shift > 0 else int(ci)  # round half up
+                v = max(0 if relu else -127, min(127, v))
+                assert v == gi
+
+
+# ---- P3/P5/P6: the event-by-event implementation and the paper's invariants --------------------
+@pytest.mark.parametrize("name", list(NETS))
+@pytest.mark.parametrize("mode", ["f32", "bf16", "i8"])
+@pytest.mark.parametrize("eager", [True, False])
+def test_event_by_event_equals_layer_by_layer(orc, name, mode, eager):
+    layers = NETS[name]
+    if mode == "i8":
+        layers = _with_shifts(layers, 8)
+    H, W = (40, 1) if name.startswith("oned") else (11, 10)
+    x, ws, bs = _rand_net(mode, layers, H, W, layers[0].cin, S=1, seed=7)
+    want = orc.forward(mode, layers, x, ws, bs)[0]
+    ev = orc.event_run(mode, layers, x[0], ws, bs, eager=eager)
+    if mode == "i8":
+        assert np.array_equal(ev["out"], want.astype(np.float64))
+        assert ev["telescoping_err"] == 0.0
+    elif mode == "f32":
+        np.testing.assert_allclose(ev["out"], want, rtol=1e-9, atol=1e-9)
+        assert ev["telescoping_err"] < 1e-9
+    else:
+        # event order changes the low bits of c, which can flip a bf16 rounding: rare, one ulp
+        close = np.isclose(ev["out"], want, rtol=1e-9, atol=1e-9)
+        assert close.mean() > 0.98
+        np.testing.assert_allclose(ev["out"], want, rtol=0.05, atol=0.02)
+    np.testing.assert_allclose(ev["sum_dh"], ev["out"], atol=1e-9)     # events telescope to the activation
+
+
+@pytest.mark.parametrize("eager", [True, False])
+def test_zero_input_emits_no_events(orc, eager):
+    layers = NETS["same_pool"]
+    _, ws, _ = _rand_net("f32", layers, 10, 10, 3, S=1, bias=False, seed=1)
+    ev = orc.event_run("f32", layers, np.zeros((10, 10, 3)), ws, None, eager=eager)
+    assert ev["events"].sum() == 0 and ev["updates"].sum() == 0
+    assert np.all(ev["out"] == 0)
+    assert np.all(orc.forward("f32", layers, np.zeros((1, 10, 10, 3)), ws, None) == 0)
+
+
+def test_sparse_input_costs_proportionally_fewer_updates(orc):
+    l = (conv(1, 4, 3),)
+    _, ws, _ = _rand_net("f32", l, 12, 12, 1, S=1, bias=False, seed=1)
+    x = np.zeros((12, 12, 1)); x[5, 5, 0] = 1.0; x[2, 9, 0] = -2.0
+    ev = orc.event_run("f32", l, x, ws, None, eager=True)
+    assert ev["events"][0] == 2 and ev["updates"][1] == 2 * 9 * 4
+
+
+def _golden_int(name):
+    path = os.path.join(os.path.dirname(__file__), "golden", name)
+    vals = [ln.strip() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    return int(vals[0])
+
+
+@pytest.mark.parametrize("length", [16, 64, 200])
+def test_fig1_toy_net_stores_seven_activations(orc, length):
+    """Fig. 1: two hidden layers with 3x1 kernels and one averaging output neuron need 7 stored
+    activations whatever the input length."""
+    seven = _golden_int("fig1_state_count.txt")
+    layers = (conv(1, 1, 3, one_d=True, relu=0), conv(1, 1, 3, one_d=True, relu=0), Layer("avg"))
+    r = np.random.default_rng(length)
+    ws = [r.standard_normal((1, 3, 1, 1)) + 2.0, r.standard_normal((1, 3, 1, 1)) + 2.0, None]
+    x = r.standard_normal((length, 1, 1)) + 3.0
+    ev = orc.event_run("f32", layers, x, ws, None, eager=True)
+    assert int(ev["live_between"][1:].sum()) == seven            # 2 + 4 + 1 between input steps
+    ev = orc.event_run("f32", layers, x, ws, None, eager=False)
+    assert int(ev["live_peak"][1:].sum()) == seven               # 3 + 3 + 1 with K-row rings
+    want = orc.forward("f32", layers, x[None], ws, None)[0]
+    np.testing.assert_allclose(ev["out"], want, rtol=1e-10)
+
+
+def test_deferred_state_is_ring_of_k_rows_independent_of_height(orc):
+    layers = (conv(2, 3, 3, pad=1), conv(3, 4, 3, stride=2), POOL)
+    peaks = []
+    for H in (12, 24):
+        x, ws, bs = _rand_net("f32", layers, H, 10, 2, S=1, seed=H)
+        x = np.abs(x) + 0.1
+        ws = [None if w is None else np.abs(w) for w in ws]
+        ev = orc.event_run("f32", layers, x[0], ws, None, eager=False)
+        peaks.append(ev["live_peak"][1:].tolist())
+    assert peaks[0] == peaks[1]
+    # ceil(Kh/stride) rows of Wout*Cout for convs, one row for the pool
+    assert peaks[0] == [3 * 10 * 3, 2 * 4 * 4, 1 * 2 * 4]
+    # doubling the width doubles the state (2D memory is proportional to the row width)
+    x, ws2, _ = _rand_net("f32", layers, 12, 20, 2, S=1, seed=1)
+    ev = orc.event_run("f32", layers, np.abs(x[0]) + 0.1, [None if w is None else np.abs(w) for w in ws2], None, eager=False)
+    assert ev["live_peak"][1] == 2 * peaks[0][0]
+
+
+def test_causality_rows_do_not_depend_on_later_input(orc):
+    layers = NETS["same_pool"]
+    x, ws, bs = _rand_net("f32", layers, 16, 12, 3, S=1, seed=4)
+    full = orc.forward("f32", layers, x, ws, bs)[0]
+    x2 = x.copy(); x2[0, 10:] = 7.0
+    alt = orc.forward("f32", layers, x2, ws, bs)[0]
+    # receptive field of output row o ends at input row 4*o + 6: rows 0..0 are safe for r = 9
+    safe = [o for o in range(full.shape[0]) if 4 * o + 6 <= 9]
+    assert safe and np.array_equal(full[safe], alt[safe])
+    assert not np.array_equal(full, alt)
