@@ -1,0 +1,296 @@
+#!/usr/bin/env python
+"""Benchmark of the incremental depth-first CNN path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload vgg2d] [--impl ours|reference]
+
+One step = one whole batch of streams pushed through the full net (all rows, then the end-of-input
+flush).  Prints ONE JSON line on rank 0.  Under torchrun every rank runs its own batch of streams
+(weak scaling, no collective on the data path); the time is the maximum over ranks.
+
+`--impl reference` times the CPU oracle (oracle/) on the host cores on a bounded sample of the
+same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_1804_10727_b200 import workloads  # noqa: E402
+
+METRIC = "input pixels/s through full net (batched streams)"
+UNIT = "pixels/s"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops_sustained"], "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback"}
+
+
+def conv_macs(w: workloads.Workload):
+    """Algorithmic multiply-accumulates per stream, per layer (the conventional count: under
+    deferred emission every unit receives each of its taps exactly once)."""
+    H, W, C = w.H, w.W, w.C
+    out = []
+    for l in w.layers:
+        if l.kind == "conv":
+            Ho = (H + 2 * l.pad - l.kh) // l.stride + 1
+            Wo = 1 if (W == 1 and l.kw == 1) else (W + 2 * l.pad - l.kw) // l.stride + 1
+            out.append(Ho * Wo * l.cout * l.cin * l.kh * l.kw)
+            H, W, C = Ho, Wo, l.cout
+        else:
+            out.append(0)
+            H, W = H // 2, (1 if W == 1 else W // 2)
+    return out
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln)
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [v.strip() for v in ln.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_rate(w: workloads.Workload, budget_s: float, steps: int = 1):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload.
+    Returns (pixels/s, threads used, description of the sample, seconds per step list)."""
+    from oracle import oracle
+    oracle.build()
+    cores = oracle.num_threads()
+    n_s = max(1, min(w.n_streams, cores))
+    ws, bs = workloads.make_params(w)
+    # calibrate on a thin slice, then pick the number of rows that fits the budget
+    probe_rows = min(w.H, 24 if w.W > 1 else 1500)
+    wp = workloads.get(w.name, n_streams=n_s, H=probe_rows)
+    xp = workloads.make_input(wp)
+    t0 = time.perf_counter()
+    oracle.forward(wp.dtype, wp.layers, xp, ws, bs)
+    tp = time.perf_counter() - t0
+    rows = w.H
+    while rows > probe_rows and tp * rows / probe_rows * steps > budget_s:
+        rows //= 2
+    rows = max(rows, probe_rows)
+    wsamp = workloads.get(w.name, n_streams=n_s, H=rows)
+    x = workloads.make_input(wsamp)
+    times = []
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        oracle.forward(wsamp.dtype, wsamp.layers, x, ws, bs)
+        times.append(time.perf_counter() - t0)
+    px = n_s * rows * w.W
+    sample = f"{n_s} of {w.n_streams} streams, first {rows} of {w.H} rows each, {len(times)} pass(es)"
+    return px / float(np.mean(times)), min(cores, n_s), sample, times
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    total = args.steps + args.warmup
+    rate, cores, sample, times = oracle_rate(w, budget_s=150.0, steps=total)
+    timed = times[args.warmup:] if len(times) > args.warmup else times
+    from oracle import oracle
+    # recompute the rate on the timed passes only
+    px_per_pass = rate * float(np.mean(times))
+    v = px_per_pass / float(np.mean(timed))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(timed)), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": {"f32": "f64", "bf16": "f64", "i8": "int32"}[w.dtype],
+        "data": "synthetic", "config": {"workload": w.name, "n_streams": w.n_streams, "H": w.H, "W": w.W, "sample": sample},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, w):
+    import torch.distributed as dist
+    from paper_1804_10727_b200 import idf
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # every rank owns its own batch of streams (weak scaling); data differs per rank via the stream offset
+    ws, bs = workloads.make_params(w)
+    x = workloads.make_input(w, first=0, count=w.n_streams)
+    if world > 1:
+        x = np.roll(x, rank, axis=0)
+    net = idf.net_from_workload(w, ws, bs, row_block=args.row_block)
+    h_seg = idf.segments_from_maps(x, w.dtype).pin_memory()
+    d_seg = h_seg.to(dev)
+    d_out = net.alloc_out(w.H, dev)
+    h_out = torch.empty(d_out.shape, dtype=d_out.dtype).pin_memory()
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
+    stream = torch.cuda.current_stream()
+
+    def step():
+        net.open(dev)
+        net.push(d_seg, d_out)
+        net.finish(d_out)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    # ---- timed region: device-resident inputs, CUDA events on the launching stream -------------
+    evs = []
+    barrier()
+    l0 = net.launches
+    n_launch = 0
+    for _ in range(args.steps):
+        flush_buf.fill_(1)                                  # evict L2 between iterations (untimed)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        step()
+        b.record(stream)
+        evs.append((a, b))
+        n_launch += net.launches                            # launch counter restarts at every open
+    barrier()
+    ms = sum(a.elapsed_time(b) for a, b in evs)
+    # ---- end to end through idf_run_host: pinned host in, host out, copies inside --------------
+    for _ in range(2):
+        net.open(dev); net.run_host(h_seg, d_seg, h_out, d_out)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        net.open(dev)
+        net.run_host(h_seg, d_seg, h_out, d_out)
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    clocks = sampler.stop() if rank == 0 else None
+    # ---- per-layer device time of the same step (instrumented pass, CUDA events per launch) ----
+    net.set_timing(True)
+    flush_buf.fill_(1)
+    step()
+    lms, ln = net.layer_times()
+    net.set_timing(False)
+
+    t = torch.tensor([ms, e2e_s * 1e3], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, e2e_ms = float(t[0]), float(t[1])
+    if rank == 0:
+        peaks = measured_peaks()
+        px_step = world * w.n_streams * w.H * w.W
+        macs = conv_macs(w)
+        dense = [i for i, l in enumerate(w.layers) if l.kind == "conv" and macs[i] > 0]
+        dom_ms = sum(lms[i] for i in dense)
+        dom_launches = sum(ln[i] for i in dense)
+        flops = 2.0 * sum(macs[i] for i in dense) * w.n_streams
+        achieved = flops / (dom_ms * 1e-3) / 1e12 if dom_ms > 0 else 0.0
+        ratio = {"bf16": 1.0, "i8": 2.0, "f32": 0.5}[w.dtype]      # nominal ratio to the bf16 dense peak
+        peak = peaks["bf16_tflops"] * ratio
+        line = {
+            "metric": METRIC, "value": px_step * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": {"f32": "f32", "bf16": "bf16", "i8": "int8"}[w.dtype], "data": "synthetic",
+            "config": {"workload": w.name, "n_streams_per_gpu": w.n_streams, "H": w.H, "W": w.W, "C": w.C,
+                       "row_block": args.row_block or "default", "l2": "flushed between iterations (256 MiB write)",
+                       "state_bytes_per_stream": net.state_bytes},
+            "clocks": clocks,
+            "e2e": {"value": px_step * args.steps / (e2e_ms * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": h_seg.numel() * h_seg.element_size(),
+                    "d2h_bytes_per_step": h_out.numel() * h_out.element_size()},
+            "gpu_launches": n_launch,
+            "roofline": {"bound": "tensor", "kernel": "dense conv update (all conv layers)", "achieved": achieved,
+                         "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak if peak else None,
+                         "peak_source": f"{peaks['source']} bf16 sustained x{ratio}", "traffic": None,
+                         "launches_per_step": dom_launches, "ms_per_step": dom_ms,
+                         "layer_ms": [round(v, 4) for v in lms]},
+        }
+        if world == 1 and not args.no_cpu:
+            rate, cores, sample, _ = oracle_rate(w, budget_s=25.0)
+            line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="vgg2d", choices=list(workloads.NAMES))
+    ap.add_argument("--streams", type=int, default=None, help="streams per GPU (default: the workload's)")
+    ap.add_argument("--row-block", type=int, default=0)
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    args = ap.parse_args()
+    w = workloads.get(args.workload, n_streams=args.streams)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

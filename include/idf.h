@@ -1,0 +1,165 @@
+/*
+ * idf - incremental depth-first CNN inference (Binas & Bengio, arXiv 1804.10727)
+ * C ABI of the CUDA (sm_100a) library.
+ *
+ * The paper's "streaming core" takes input segments as they arrive and updates
+ * its output incrementally (Introduction, last paragraph; Discussion, second
+ * paragraph).  A segment is one sample of a 1D signal or one row of a 2D image
+ * (Section "Asynchronous incremental updates", the 1D/2D paragraphs and Fig. 2).
+ * Every unit keeps a state variable c (Eq. 2); an arriving event dh is added as
+ * c += w * dh (Eq. 4); a unit whose activation f(c) has changed passes the
+ * change on to the next layer (Eq. 3, Eq. 5).  This library uses the
+ * segment-synchronous form of that rule: a unit emits once, when no present or
+ * future segment can reach it any more, so every conv layer keeps only
+ * ceil(Kh/stride) rows of state ("activation subset buffers", Discussion) and the
+ * result equals conventional layer-by-layer inference (Eq. 1).
+ *
+ * Many independent streams advance in lockstep: every call handles the same
+ * number of segments for each of n_streams streams.
+ *
+ * Conventions
+ *   - All functions return IDF_OK (0) or a negative idf_status; no exceptions, no abort,
+ *     no device traps.  idf_last_error() gives a message for the calling thread's last failure.
+ *   - "host" / "device" in a parameter comment says where the pointer must live.
+ *   - The library allocates no device memory: the caller passes the workspace, the segment
+ *     buffer and the output buffer (device memory it owns) and the CUDA stream all work is
+ *     enqueued on.  A handle is not thread-safe; distinct handles are independent.
+ *   - There is no CPU fallback and no other backend.
+ *   - Layouts have channels innermost.  Weights: [Cout][Kh][Kw][Cin], cross-correlation
+ *     (no kernel flip), zero padding `pad` on all four sides, one stride for both axes,
+ *     output extent floor((n + 2 pad - k) / stride) + 1.  A 1D net has in_w == 1 and kw == 1.
+ */
+#ifndef IDF_H
+#define IDF_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct idf_net idf_net;   /* opaque; owns packed host copies of the parameters and the layout */
+
+/* activation/weight type _ state type */
+typedef enum {
+    IDF_F32 = 0,       /* fp32 activations and weights, fp32 state                                   */
+    IDF_BF16_F32 = 1,  /* bf16 activations and weights, fp32 state; a conv layer that feeds a later  */
+                       /* conv layer rounds f(c) to bf16 (nearest even); the last conv layer and     */
+                       /* whatever follows it stay fp32; the net's output is fp32                    */
+    IDF_I8_I32 = 2     /* int8 activations and weights, int32 state; per conv layer                  */
+                       /* q = clamp((c + 2^(shift-1)) >> shift, relu ? 0 : -127, 127); output int8   */
+} idf_dtype;
+
+typedef enum { IDF_CONV = 0, IDF_MAXPOOL2 = 1 } idf_kind;   /* 2x2 max pool, stride 2, floor; rows only when width is 1 */
+typedef enum { IDF_PATH_AUTO = 0, IDF_PATH_DENSE = 1, IDF_PATH_SPARSE = 2 } idf_path;
+
+typedef enum {
+    IDF_OK = 0,
+    IDF_ERR_ARG = -1,          /* null pointer, negative count, ...                                   */
+    IDF_ERR_SPEC = -2,         /* inconsistent layer spec (channel mismatch, empty map, ...)          */
+    IDF_ERR_STATE = -3,        /* push before open or after finish                                    */
+    IDF_ERR_CAPACITY = -4,     /* workspace or output buffer too small                                */
+    IDF_ERR_UNSUPPORTED = -5,  /* valid request this build cannot serve                               */
+    IDF_ERR_CUDA = -6,         /* a CUDA call failed                                                  */
+    IDF_ERR_TIMEOUT = -7       /* a bounded device-side wait ran out                                  */
+} idf_status;
+
+typedef struct {
+    int kind;      /* idf_kind                                                        */
+    int cin, cout; /* conv only                                                       */
+    int kh, kw;    /* conv only; kw == 1 for 1D nets                                  */
+    int stride;    /* conv only; 1 <= stride <= kh                                    */
+    int pad;       /* conv only; 0 <= pad < kh                                        */
+    int relu;      /* conv only; f = ReLU if non-zero, identity otherwise             */
+    int shift;     /* conv only, IDF_I8_I32: requantisation shift, 0..30              */
+    int path;      /* conv only; idf_path: how the layer's events are applied         */
+} idf_layer;
+
+typedef struct {
+    int n_layers;
+    const idf_layer* layers;   /* host */
+    int dtype;                 /* idf_dtype */
+    int in_w, in_c;            /* segment width (1 for 1D) and channels */
+    int n_streams;             /* streams advanced together by every call */
+    int row_block;             /* most segments pushed through all layers at once (bounds the   */
+                               /* transient workspace); 0 = library default                     */
+} idf_spec;
+
+/* Build a net from a layer list and the parameters of a conventionally trained CNN
+ * (Section "Experimental verification": learned parameters are copied into the incremental
+ * model).  weights[i] / biases[i] belong to layers[i]; entries of non-conv layers are ignored.
+ *   weights: host, per conv layer [Cout][Kh][Kw][Cin] in the activation type (fp32 / bf16 bits / int8)
+ *   biases : host, per conv layer [Cout] in the state type (fp32 / int32); the array or an entry may
+ *            be NULL = zero bias.  The paper takes b = 0 without loss of generality; here the bias
+ *            joins at emission, h = f(c + b).
+ * Everything is copied; the caller may free its buffers on return.  *out receives the handle. */
+int idf_net_create(const idf_spec* spec, const void* const* weights, const void* const* biases, idf_net** out);
+
+/* Release the handle (host memory only; device buffers belong to the caller). */
+int idf_net_destroy(idf_net* net);
+
+/* Rolling state PER STREAM in bytes: sum over conv layers of ceil(Kh/stride) rows of Wout*Cout
+ * state words, plus one row per pooling layer.  Constant in the number of segments (1D: constant;
+ * 2D: proportional to the row width), as the paper's abstract claims.  0 if net is NULL. */
+size_t idf_net_state_bytes(const idf_net* net);
+
+/* Device bytes the caller must provide to idf_stream_open: all streams' rolling state, the packed
+ * parameters, and the transient row_block-sized buffers between layers. */
+size_t idf_net_workspace_bytes(const idf_net* net);
+
+/* Shape of the output map after in_rows segments (out_rows may be 0). Any out pointer may be NULL. */
+int idf_out_shape(const idf_net* net, long long in_rows, long long* out_rows, int* out_w, int* out_c);
+
+/* Bind a workspace (device, 256-byte aligned, >= idf_net_workspace_bytes) and a CUDA stream
+ * (a cudaStream_t passed as void*, NULL = default stream); upload the parameters, zero all state,
+ * reset the segment counters.  May be called again after idf_stream_finish to start new streams. */
+int idf_stream_open(idf_net* net, void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Push n_seg consecutive segments of every stream through all layers, depth first.
+ *   d_segments: device, [n_seg][n_streams][in_w][in_c] in the activation type
+ *   d_out     : device, [n_streams][out_capacity_rows][out_w][out_c], fp32 (float nets) or int8;
+ *               output rows that become complete are written at their absolute row index
+ *   rows_emitted: host, may be NULL; receives the number of output rows completed by this call.
+ *               The count is known on the host, so no synchronisation is implied; the work is
+ *               enqueued on the stream given to idf_stream_open.
+ * The result does not depend on how segments are grouped into calls (bit-exact for int nets).
+ * Errors: IDF_ERR_STATE before open / after finish; IDF_ERR_CAPACITY if a completed row would not
+ * fit out_capacity_rows (nothing is enqueued in that case). */
+int idf_stream_push(idf_net* net, const void* d_segments, int n_seg,
+                    void* d_out, long long out_capacity_rows, int* rows_emitted);
+
+/* End of input: complete the rows that wait only for bottom zero padding, in depth order, and
+ * drop rows that can never complete.  total_rows (host, may be NULL) receives the number of output
+ * rows per stream since open.  After this call only idf_stream_open or idf_net_destroy are valid. */
+int idf_stream_finish(idf_net* net, void* d_out, long long out_capacity_rows, long long* total_rows);
+
+/* Whole streams from host memory: copy h_segments ([n_seg][n_streams][in_w][in_c], host, ideally
+ * pinned) to d_segments, push, finish, copy the output map back to h_out
+ * ([n_streams][out_capacity_rows][out_w][out_c], host) and wait for the stream.  d_segments and
+ * d_out are device staging buffers of the same sizes, owned by the caller.  The handle must be
+ * freshly opened. */
+int idf_run_host(idf_net* net, const void* h_segments, int n_seg, void* d_segments,
+                 void* h_out, void* d_out, long long out_capacity_rows, long long* total_rows);
+
+/* Counters of the sparse-event path since open, read back from the device (synchronises the
+ * stream): events[i] = number of non-zero input events layer i has applied; entries of layers on
+ * the dense path are 0.  events: host, n_layers entries. */
+int idf_event_counts(idf_net* net, long long* events);
+
+/* Kernel launches enqueued by this handle since open. */
+long long idf_launch_count(const idf_net* net);
+
+/* Per-layer device time.  With timing on, every kernel launch of the handle is bracketed by CUDA
+ * events on its stream.  idf_layer_times synchronises the stream, adds up the elapsed time of the
+ * launches recorded since the last query into ms[i] (milliseconds, host, n_layers entries) and
+ * their number into launches[i], and clears the record. */
+int idf_set_timing(idf_net* net, int on);
+int idf_layer_times(idf_net* net, double* ms, long long* launches);
+
+/* Message for the most recent failure on the calling thread ("" if none). */
+const char* idf_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IDF_H */

@@ -129,10 +129,12 @@ static void deliver(evc_net* N, int n, int y, int x, int ch, double d)
             if (ty < 0 || ty % l->stride) continue;
             int oy = ty / l->stride;
             if (oy >= N->H[n]) continue;
+            const int one_d = (N->W[n - 1] == 1 && l->kw == 1);   /* degenerate x axis: no pad, no stride */
+            const int pad_x = one_d ? 0 : l->pad, stride_x = one_d ? 1 : l->stride;
             for (int kx = 0; kx < l->kw; ++kx) {
-                int tx = x + l->pad - kx;
-                if (tx < 0 || tx % l->stride) continue;
-                int ox = tx / l->stride;
+                int tx = x + pad_x - kx;
+                if (tx < 0 || tx % stride_x) continue;
+                int ox = tx / stride_x;
                 if (ox >= N->W[n]) continue;
                 for (int co = 0; co < l->cout; ++co) {
                     size_t i = ((size_t)oy * N->W[n] + ox) * N->C[n] + co;
@@ -239,7 +241,7 @@ int evc_run(int mode, int eager, int n_layers, const evc_layer* layers,
         const evc_layer* l = &layers[n - 1];
         if (l->kind == EVC_CONV) {
             N.H[n] = (N.H[n - 1] + 2 * l->pad - l->kh) / l->stride + 1;
-            N.W[n] = (N.W[n - 1] + 2 * l->pad - l->kw) / l->stride + 1;
+            N.W[n] = (N.W[n - 1] == 1 && l->kw == 1) ? 1 : (N.W[n - 1] + 2 * l->pad - l->kw) / l->stride + 1;
             N.C[n] = l->cout;
         } else if (l->kind == EVC_MAXPOOL2) {
             N.H[n] = N.H[n - 1] / 2; N.W[n] = (N.W[n - 1] == 1) ? 1 : N.W[n - 1] / 2; N.C[n] = N.C[n - 1];

@@ -18,7 +18,8 @@
  *   maps     [n_streams][H][W][C]
  *   weights  [Cout][Kh][Kw][Cin]      (cross-correlation, no kernel flip)
  * Zero padding of `pad` on all four sides, the same stride on both axes,
- * output size floor((H + 2 pad - Kh) / stride) + 1.  A 1D net is W = Kw = 1.
+ * output size floor((H + 2 pad - Kh) / stride) + 1.  A 1D net is W = Kw = 1:
+ * its x axis is degenerate and takes neither padding nor stride.
  *
  * Pins (tests that do not depend on this file's own arithmetic):
  *   - torch.nn.functional conv/relu/max_pool2d in float64 on CPU,
@@ -39,9 +40,11 @@ void orc_conv_f64(const double* in, long long n_streams, int H, int W, int Cin,
                   const double* w, const double* b, int Cout, int Kh, int Kw,
                   int stride, int pad, int relu, double* out)
 {
+    const int one_d = (W == 1 && Kw == 1);
+    const int pad_x = one_d ? 0 : pad, stride_x = one_d ? 1 : stride;
     const int Ho = (H + 2 * pad - Kh) / stride + 1;
-    const int Wo = (W + 2 * pad - Kw) / stride + 1;
-    if (H + 2 * pad < Kh || W + 2 * pad < Kw) return;
+    const int Wo = (W + 2 * pad_x - Kw) / stride_x + 1;
+    if (H + 2 * pad < Kh || W + 2 * pad_x < Kw) return;
 #pragma omp parallel for schedule(dynamic, 1)
     for (long long s = 0; s < n_streams; ++s) {
         const double* ins = in + (size_t)s * H * W * Cin;
@@ -54,7 +57,7 @@ void orc_conv_f64(const double* in, long long n_streams, int H, int W, int Cin,
                         const int iy = oy * stride - pad + ky;
                         if (iy < 0 || iy >= H) continue;
                         for (int kx = 0; kx < Kw; ++kx) {
-                            const int ix = ox * stride - pad + kx;
+                            const int ix = ox * stride_x - pad_x + kx;
                             if (ix < 0 || ix >= W) continue;
                             const double* a = ins + ((size_t)iy * W + ix) * Cin;
                             const double* ww = w + (((size_t)co * Kh + ky) * Kw + kx) * Cin;
@@ -75,9 +78,11 @@ void orc_conv_i32(const int32_t* in, long long n_streams, int H, int W, int Cin,
                   const int32_t* w, const int32_t* b, int Cout, int Kh, int Kw,
                   int stride, int pad, int relu, int32_t* out)
 {
+    const int one_d = (W == 1 && Kw == 1);
+    const int pad_x = one_d ? 0 : pad, stride_x = one_d ? 1 : stride;
     const int Ho = (H + 2 * pad - Kh) / stride + 1;
-    const int Wo = (W + 2 * pad - Kw) / stride + 1;
-    if (H + 2 * pad < Kh || W + 2 * pad < Kw) return;
+    const int Wo = (W + 2 * pad_x - Kw) / stride_x + 1;
+    if (H + 2 * pad < Kh || W + 2 * pad_x < Kw) return;
 #pragma omp parallel for schedule(dynamic, 1)
     for (long long s = 0; s < n_streams; ++s) {
         const int32_t* ins = in + (size_t)s * H * W * Cin;
@@ -90,7 +95,7 @@ void orc_conv_i32(const int32_t* in, long long n_streams, int H, int W, int Cin,
                         const int iy = oy * stride - pad + ky;
                         if (iy < 0 || iy >= H) continue;
                         for (int kx = 0; kx < Kw; ++kx) {
-                            const int ix = ox * stride - pad + kx;
+                            const int ix = ox * stride_x - pad_x + kx;
                             if (ix < 0 || ix >= W) continue;
                             const int32_t* a = ins + ((size_t)iy * W + ix) * Cin;
                             const int32_t* ww = w + (((size_t)co * Kh + ky) * Kw + kx) * Cin;

@@ -81,7 +81,10 @@ def out_shape(layers, H: int, W: int, C: int):
     for l in layers:
         kind = _kind(l)
         if kind == "conv":
-            H, W, C = conv_out(H, _g(l, "kh"), _g(l, "stride"), _g(l, "pad")), conv_out(W, _g(l, "kw"), _g(l, "stride"), _g(l, "pad")), _g(l, "cout")
+            one_d = (W == 1 and _g(l, "kw") == 1)
+            H = conv_out(H, _g(l, "kh"), _g(l, "stride"), _g(l, "pad"))
+            W = 1 if one_d else conv_out(W, _g(l, "kw"), _g(l, "stride"), _g(l, "pad"))
+            C = _g(l, "cout")
         elif kind == "pool":
             H, W = H // 2, (1 if W == 1 else W // 2)
         else:
@@ -108,7 +111,8 @@ def conv_layer(mode: str, layer, x: np.ndarray, w: np.ndarray, b) -> np.ndarray:
     Cout, Kh, Kw = _g(layer, "cout"), _g(layer, "kh"), _g(layer, "kw")
     st, pd, relu = _g(layer, "stride"), _g(layer, "pad"), _g(layer, "relu")
     assert Cin == _g(layer, "cin") and w.shape == (Cout, Kh, Kw, Cin), (x.shape, w.shape)
-    Ho, Wo = conv_out(H, Kh, st, pd), conv_out(W, Kw, st, pd)
+    Ho = conv_out(H, Kh, st, pd)
+    Wo = 1 if (W == 1 and Kw == 1) else conv_out(W, Kw, st, pd)     # 1D: degenerate x axis
     assert Ho >= 1 and Wo >= 1
     L = lib()
     if mode == "i8":

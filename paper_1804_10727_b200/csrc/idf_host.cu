@@ -1,0 +1,497 @@
+// Host side of the C ABI: spec validation, shape inference, workspace layout, parameter packing
+// and the depth-first schedule that walks every block of pushed segments through all layers.
+#include "../../include/idf.h"
+#include "idf_internal.h"
+
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+using namespace idf;
+
+namespace {
+
+thread_local std::string g_err;
+
+int fail(int code, const char* fmt, ...)
+{
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_err = buf;
+    return code;
+}
+
+size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+struct LayerPlan {
+    idf_layer l;
+    int in_w, out_w, in_c, out_c;
+    int ring_rows;           // conv: ceil(kh/stride); pool: 1
+    int in_elem, out_elem;   // Elem of the rows this layer receives / emits
+    int use_sparse;
+    // host copies of the packed parameters
+    std::vector<unsigned char> w_packed;   // [Kh][Kw][Cin][Cout] float (float nets) or int8
+    std::vector<unsigned char> b_packed;   // [Cout] float / int32 (empty = zero bias)
+    // workspace offsets
+    size_t w_off = 0, b_off = 0, state_off = 0, out_off = 0;
+    size_t state_bytes_all = 0;            // all streams
+    size_t state_bytes_stream = 0;
+    int out_cap_rows = 0;                  // capacity of the buffer this layer emits into
+    // progress (identical for all streams)
+    long long rows_in = 0, rows_done = 0;
+};
+
+enum Phase { CREATED = 0, OPEN = 1, FINISHED = 2 };
+
+}  // namespace
+
+struct idf_net {
+    int dtype = 0, in_w = 0, in_c = 0, n_streams = 0, row_block = 0;
+    std::vector<LayerPlan> L;
+    size_t workspace_bytes = 0, state_region_off = 0, state_region_bytes = 0, counters_off = 0;
+    size_t state_bytes_stream = 0;
+    unsigned char* ws = nullptr;
+    cudaStream_t stream = nullptr;
+    int phase = CREATED;
+    long long launches = 0;
+    long long out_rows_total = 0;
+    // optional per-launch timing (CUDA events on the handle's stream)
+    bool timing = false;
+    struct Timed { int layer; cudaEvent_t a, b; };
+    std::vector<Timed> timed;
+    std::vector<cudaEvent_t> event_pool;
+};
+
+namespace {
+
+float bf16_bits_to_float(uint16_t b)
+{
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+long long conv_done_after(const idf_layer& l, long long rows_in)
+{
+    // number of output rows whose last tap (row o*stride - pad + Kh - 1) lies below rows_in
+    const long long q = rows_in + l.pad - l.kh;
+    return q < 0 ? 0 : q / l.stride + 1;
+}
+
+long long conv_rows_at_flush(const idf_layer& l, long long rows_in)
+{
+    // floor((H + 2 pad - Kh) / stride) + 1 rows exist once the input is known to have H rows
+    if (rows_in <= 0) return 0;
+    const long long q = rows_in + 2LL * l.pad - l.kh;
+    return q < 0 ? 0 : q / l.stride + 1;
+}
+
+// One layer takes n_in new input rows (and, when flushing, learns that the input has ended).
+// Returns the number of rows it emits; enqueues nothing when `dry` is set.
+int advance_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, bool flush, bool dry,
+                  void* final_out, long long out_cap, long long* n_out_p, long long* rows_in_sim,
+                  long long* rows_done_sim)
+{
+    LayerPlan& P = net->L[i];
+    const bool last = (i + 1 == net->L.size());
+    const long long r0 = rows_in_sim[i], r1 = r0 + n_in;
+    long long done_end, o_end;
+    if (P.l.kind == IDF_CONV) {
+        done_end = flush ? conv_rows_at_flush(P.l, r1) : conv_done_after(P.l, r1);
+        const long long started = r1 > 0 ? (r1 - 1 + P.l.pad) / P.l.stride + 1 : 0;   // rows reached so far
+        o_end = std::max(started, done_end);
+    } else {
+        done_end = r1 / 2;
+        o_end = (r1 + 1) / 2;
+    }
+    const long long o_begin = rows_done_sim[i];
+    if (done_end < o_begin) done_end = o_begin;
+    const long long n_out = done_end - o_begin;
+    *n_out_p = n_out;
+    rows_in_sim[i] = r1;
+    rows_done_sim[i] = done_end;
+    if (last && done_end > out_cap)
+        return fail(IDF_ERR_CAPACITY, "output row %lld does not fit out_capacity_rows=%lld", done_end - 1, out_cap);
+    if (!last && n_out > P.out_cap_rows)
+        return fail(IDF_ERR_CAPACITY, "internal: layer %zu emits %lld rows into a %d-row buffer", i, n_out, P.out_cap_rows);
+    if (dry || (n_in == 0 && n_out == 0)) return IDF_OK;
+
+    const long long S = net->n_streams;
+    void* out_ptr;
+    long long row_stride, stream_stride, row_base;
+    if (last) {
+        out_ptr = final_out;
+        row_stride = (long long)P.out_w * P.out_c;
+        stream_stride = out_cap * row_stride;
+        row_base = 0;
+    } else {
+        out_ptr = net->ws + P.out_off;
+        stream_stride = (long long)P.out_w * P.out_c;
+        row_stride = S * stream_stride;
+        row_base = o_begin;
+    }
+    cudaError_t ce;
+    cudaEvent_t ev_a = nullptr, ev_b = nullptr;
+    if (net->timing) {
+        for (cudaEvent_t* e : {&ev_a, &ev_b}) {
+            if (!net->event_pool.empty()) { *e = net->event_pool.back(); net->event_pool.pop_back(); }
+            else if (cudaEventCreate(e) != cudaSuccess) return fail(IDF_ERR_CUDA, "cudaEventCreate failed");
+        }
+        cudaEventRecord(ev_a, net->stream);
+    }
+    if (P.l.kind == IDF_CONV) {
+        ConvArgs a{};
+        a.in = in_ptr;
+        a.w = net->ws + P.w_off;
+        a.bias = P.b_packed.empty() ? nullptr : net->ws + P.b_off;
+        a.ring = net->ws + P.state_off;
+        a.out = out_ptr;
+        a.out_row_stride = row_stride; a.out_stream_stride = stream_stride; a.out_row_base = row_base;
+        a.event_counter = (unsigned long long*)(net->ws + net->counters_off) + i;
+        a.S = (int)S; a.Win = P.in_w; a.Wout = P.out_w; a.Cin = P.in_c; a.Cout = P.out_c;
+        a.Kh = P.l.kh; a.Kw = P.l.kw; a.stride = P.l.stride; a.pad = P.l.pad; a.relu = P.l.relu; a.shift = P.l.shift;
+        a.stride_x = P.in_w == 1 ? 1 : P.l.stride; a.pad_x = P.in_w == 1 ? 0 : P.l.pad;
+        a.ring_rows = P.ring_rows; a.in_elem = P.in_elem; a.out_elem = P.out_elem;
+        a.r0 = r0; a.r1 = r1; a.o_begin = o_begin; a.o_end = o_end; a.done_end = done_end;
+        ce = P.use_sparse ? launch_conv_sparse(a, net->dtype, net->stream) : launch_conv_simple(a, net->dtype, net->stream);
+    } else {
+        PoolArgs a{};
+        a.in = in_ptr;
+        a.state = net->ws + P.state_off;
+        a.out = out_ptr;
+        a.out_row_stride = row_stride; a.out_stream_stride = stream_stride; a.out_row_base = row_base;
+        a.S = (int)S; a.Win = P.in_w; a.Wout = P.out_w; a.C = P.in_c; a.elem = P.in_elem;
+        a.r0 = r0; a.r1 = r1; a.o_begin = o_begin; a.o_end = o_end; a.done_end = done_end;
+        ce = launch_pool(a, net->stream);
+    }
+    if (net->timing) {
+        cudaEventRecord(ev_b, net->stream);
+        net->timed.push_back({(int)i, ev_a, ev_b});
+    }
+    if (ce != cudaSuccess) return fail(IDF_ERR_CUDA, "kernel launch failed at layer %zu: %s", i, cudaGetErrorString(ce));
+    net->launches += 1;
+    return IDF_OK;
+}
+
+// Depth-first pass of one block of segments (or of the end-of-input flush) through all layers.
+int run_block(idf_net* net, const void* d_seg, long long n_seg, bool flush, bool dry, void* d_out,
+              long long out_cap, long long* rows_in_sim, long long* rows_done_sim, long long* emitted)
+{
+    const void* in_ptr = d_seg;
+    long long n_in = n_seg;
+    for (size_t i = 0; i < net->L.size(); ++i) {
+        long long n_out = 0;
+        int rc = advance_layer(net, i, in_ptr, n_in, flush, dry, d_out, out_cap, &n_out, rows_in_sim, rows_done_sim);
+        if (rc != IDF_OK) return rc;
+        if (i + 1 == net->L.size()) *emitted += n_out;
+        if (n_out == 0 && !flush) break;    // nothing travels further up in this block
+        in_ptr = net->ws + net->L[i].out_off;
+        n_in = n_out;
+    }
+    return IDF_OK;
+}
+
+int run_segments(idf_net* net, const void* d_segments, long long n_seg, bool flush, void* d_out,
+                 long long out_cap, long long* emitted)
+{
+    const size_t nl = net->L.size();
+    std::vector<long long> rin(nl), rdone(nl);
+    const size_t seg_bytes = (size_t)net->n_streams * net->in_w * net->in_c * elem_size(net->L[0].in_elem);
+    for (int pass = 0; pass < 2; ++pass) {       // pass 0: dry run (capacity check), pass 1: enqueue
+        const bool dry = (pass == 0);
+        for (size_t i = 0; i < nl; ++i) { rin[i] = net->L[i].rows_in; rdone[i] = net->L[i].rows_done; }
+        long long em = 0;
+        for (long long s0 = 0; s0 < n_seg; s0 += net->row_block) {
+            const long long n = std::min<long long>(net->row_block, n_seg - s0);
+            int rc = run_block(net, (const unsigned char*)d_segments + (size_t)s0 * seg_bytes, n, false, dry, d_out,
+                               out_cap, rin.data(), rdone.data(), &em);
+            if (rc != IDF_OK) return rc;
+        }
+        if (flush) {
+            int rc = run_block(net, nullptr, 0, true, dry, d_out, out_cap, rin.data(), rdone.data(), &em);
+            if (rc != IDF_OK) return rc;
+        }
+        if (!dry) {
+            for (size_t i = 0; i < nl; ++i) { net->L[i].rows_in = rin[i]; net->L[i].rows_done = rdone[i]; }
+            *emitted = em;
+        }
+    }
+    return IDF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* idf_last_error(void) { return g_err.c_str(); }
+
+int idf_net_create(const idf_spec* spec, const void* const* weights, const void* const* biases, idf_net** out)
+{
+    if (!spec || !out) return fail(IDF_ERR_ARG, "spec and out must not be NULL");
+    *out = nullptr;
+    if (!spec->layers || spec->n_layers < 1 || spec->n_layers > 256) return fail(IDF_ERR_ARG, "n_layers must be 1..256");
+    if (!weights) return fail(IDF_ERR_ARG, "weights must not be NULL");
+    if (spec->dtype < IDF_F32 || spec->dtype > IDF_I8_I32) return fail(IDF_ERR_SPEC, "unknown dtype %d", spec->dtype);
+    if (spec->in_w < 1 || spec->in_c < 1) return fail(IDF_ERR_SPEC, "in_w and in_c must be positive");
+    if (spec->n_streams < 1) return fail(IDF_ERR_SPEC, "n_streams must be positive");
+    if (spec->row_block < 0 || spec->row_block > 4096) return fail(IDF_ERR_SPEC, "row_block must be 0..4096");
+
+    idf_net* net = new (std::nothrow) idf_net();
+    if (!net) return fail(IDF_ERR_ARG, "out of host memory");
+    net->dtype = spec->dtype; net->in_w = spec->in_w; net->in_c = spec->in_c; net->n_streams = spec->n_streams;
+    net->row_block = spec->row_block > 0 ? spec->row_block : 8;
+    const int act_elem = spec->dtype == IDF_F32 ? E_F32 : (spec->dtype == IDF_BF16_F32 ? E_BF16 : E_I8);
+    const size_t state_word = 4;
+
+    int last_conv = -1;
+    for (int i = 0; i < spec->n_layers; ++i)
+        if (spec->layers[i].kind == IDF_CONV) last_conv = i;
+    if (last_conv < 0) { delete net; return fail(IDF_ERR_SPEC, "a net needs at least one conv layer"); }
+
+    int w = spec->in_w, c = spec->in_c, elem = act_elem;
+    int cap = net->row_block;
+    net->L.resize(spec->n_layers);
+    for (int i = 0; i < spec->n_layers; ++i) {
+        LayerPlan& P = net->L[i];
+        P.l = spec->layers[i];
+        P.in_w = w; P.in_c = c; P.in_elem = elem;
+        const idf_layer& l = P.l;
+        if (l.kind == IDF_CONV) {
+            if (l.cin != c) { delete net; return fail(IDF_ERR_SPEC, "layer %d: cin=%d but the incoming map has %d channels", i, l.cin, c); }
+            if (l.cout < 1 || l.kh < 1 || l.kw < 1) { delete net; return fail(IDF_ERR_SPEC, "layer %d: cout, kh, kw must be positive", i); }
+            if (l.stride < 1 || l.stride > l.kh) { delete net; return fail(IDF_ERR_SPEC, "layer %d: stride must be 1..kh", i); }
+            if (l.pad < 0 || l.pad >= l.kh) { delete net; return fail(IDF_ERR_SPEC, "layer %d: pad must be 0..kh-1", i); }
+            if (w == 1 && l.kw != 1) { delete net; return fail(IDF_ERR_SPEC, "layer %d: a width-1 map needs kw == 1", i); }
+            if (l.shift < 0 || l.shift > 30) { delete net; return fail(IDF_ERR_SPEC, "layer %d: shift must be 0..30", i); }
+            if (l.path < IDF_PATH_AUTO || l.path > IDF_PATH_SPARSE) { delete net; return fail(IDF_ERR_SPEC, "layer %d: unknown path", i); }
+            if (!weights[i]) { delete net; return fail(IDF_ERR_ARG, "layer %d: weights missing", i); }
+            const int padw = (w == 1) ? 0 : l.pad;     // 1D nets pad the streaming axis only
+            if (w + 2 * padw < l.kw) { delete net; return fail(IDF_ERR_SPEC, "layer %d: kernel wider than the padded row", i); }
+            P.out_w = (w + 2 * padw - l.kw) / l.stride + 1;
+            if (w == 1) P.out_w = 1;
+            P.out_c = l.cout;
+            P.ring_rows = (l.kh + l.stride - 1) / l.stride;
+            P.out_elem = spec->dtype == IDF_F32 ? E_F32
+                       : spec->dtype == IDF_I8_I32 ? E_I8
+                       : (i == last_conv ? E_F32 : E_BF16);
+            // sparse path by default only for the thin first layer of an integer net (raw, sparse input)
+            P.use_sparse = l.path == IDF_PATH_SPARSE ||
+                           (l.path == IDF_PATH_AUTO && i == 0 && spec->dtype == IDF_I8_I32 && l.cin <= 4);
+            P.state_bytes_stream = (size_t)P.ring_rows * P.out_w * P.out_c * state_word;
+            cap = (cap + l.stride - 1) / l.stride + 1 + P.ring_rows;
+            // parameters -> [Kh][Kw][Cin][Cout]
+            const size_t nw = (size_t)l.cout * l.kh * l.kw * l.cin;
+            if (spec->dtype == IDF_I8_I32) {
+                P.w_packed.resize(nw);
+                const int8_t* src = (const int8_t*)weights[i];
+                for (int co = 0; co < l.cout; ++co)
+                    for (int k = 0; k < l.kh * l.kw; ++k)
+                        for (int ci = 0; ci < l.cin; ++ci)
+                            ((int8_t*)P.w_packed.data())[((size_t)k * l.cin + ci) * l.cout + co] =
+                                src[((size_t)co * l.kh * l.kw + k) * l.cin + ci];
+            } else {
+                P.w_packed.resize(nw * 4);
+                float* dst = (float*)P.w_packed.data();
+                for (int co = 0; co < l.cout; ++co)
+                    for (int k = 0; k < l.kh * l.kw; ++k)
+                        for (int ci = 0; ci < l.cin; ++ci) {
+                            const size_t si = ((size_t)co * l.kh * l.kw + k) * l.cin + ci;
+                            const float v = spec->dtype == IDF_F32 ? ((const float*)weights[i])[si]
+                                                                  : bf16_bits_to_float(((const uint16_t*)weights[i])[si]);
+                            dst[((size_t)k * l.cin + ci) * l.cout + co] = v;
+                        }
+            }
+            if (biases && biases[i]) {
+                P.b_packed.resize((size_t)l.cout * 4);
+                memcpy(P.b_packed.data(), biases[i], (size_t)l.cout * 4);
+            }
+        } else if (l.kind == IDF_MAXPOOL2) {
+            P.out_w = (w == 1) ? 1 : w / 2;
+            if (P.out_w < 1) { delete net; return fail(IDF_ERR_SPEC, "layer %d: pooling an empty row", i); }
+            P.out_c = c;
+            P.ring_rows = 1;
+            P.out_elem = elem;
+            P.use_sparse = 0;
+            P.state_bytes_stream = (size_t)P.out_w * P.out_c * elem_size(elem);
+            cap = cap / 2 + 1;
+        } else {
+            delete net;
+            return fail(IDF_ERR_SPEC, "layer %d: unknown kind %d", i, l.kind);
+        }
+        P.out_cap_rows = cap;
+        P.state_bytes_all = P.state_bytes_stream * (size_t)net->n_streams;
+        net->state_bytes_stream += P.state_bytes_stream;
+        w = P.out_w; c = P.out_c; elem = P.out_elem;
+    }
+    // workspace: [parameters][state of all streams][rows travelling between layers][counters]
+    size_t off = 0;
+    for (auto& P : net->L) {
+        P.w_off = off; off = align_up(off + P.w_packed.size());
+        P.b_off = off; off = align_up(off + P.b_packed.size());
+    }
+    net->state_region_off = off;
+    for (auto& P : net->L) { P.state_off = off; off = align_up(off + P.state_bytes_all); }
+    net->state_region_bytes = off - net->state_region_off;
+    for (size_t i = 0; i + 1 < net->L.size(); ++i) {
+        LayerPlan& P = net->L[i];
+        P.out_off = off;
+        off = align_up(off + (size_t)P.out_cap_rows * net->n_streams * P.out_w * P.out_c * elem_size(P.out_elem));
+    }
+    net->counters_off = off;
+    off = align_up(off + net->L.size() * sizeof(unsigned long long));
+    net->workspace_bytes = off;
+    *out = net;
+    return IDF_OK;
+}
+
+int idf_net_destroy(idf_net* net)
+{
+    if (net) {
+        for (auto& t : net->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
+        for (auto e : net->event_pool) cudaEventDestroy(e);
+    }
+    delete net;
+    return IDF_OK;
+}
+
+size_t idf_net_state_bytes(const idf_net* net) { return net ? net->state_bytes_stream : 0; }
+
+size_t idf_net_workspace_bytes(const idf_net* net) { return net ? net->workspace_bytes : 0; }
+
+int idf_out_shape(const idf_net* net, long long in_rows, long long* out_rows, int* out_w, int* out_c)
+{
+    if (!net) return fail(IDF_ERR_ARG, "net must not be NULL");
+    if (in_rows < 0) return fail(IDF_ERR_ARG, "in_rows must not be negative");
+    long long h = in_rows;
+    for (const auto& P : net->L) h = P.l.kind == IDF_CONV ? conv_rows_at_flush(P.l, h) : h / 2;
+    if (out_rows) *out_rows = h;
+    if (out_w) *out_w = net->L.back().out_w;
+    if (out_c) *out_c = net->L.back().out_c;
+    return IDF_OK;
+}
+
+int idf_stream_open(idf_net* net, void* d_workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (!net || !d_workspace) return fail(IDF_ERR_ARG, "net and d_workspace must not be NULL");
+    if (workspace_bytes < net->workspace_bytes)
+        return fail(IDF_ERR_CAPACITY, "workspace has %zu bytes, %zu needed", workspace_bytes, net->workspace_bytes);
+    if (((uintptr_t)d_workspace & 255) != 0) return fail(IDF_ERR_ARG, "d_workspace must be 256-byte aligned");
+    net->ws = (unsigned char*)d_workspace;
+    net->stream = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaSuccess;
+    for (auto& P : net->L) {
+        if (!P.w_packed.empty() && e == cudaSuccess)
+            e = cudaMemcpyAsync(net->ws + P.w_off, P.w_packed.data(), P.w_packed.size(), cudaMemcpyHostToDevice, net->stream);
+        if (!P.b_packed.empty() && e == cudaSuccess)
+            e = cudaMemcpyAsync(net->ws + P.b_off, P.b_packed.data(), P.b_packed.size(), cudaMemcpyHostToDevice, net->stream);
+        P.rows_in = 0; P.rows_done = 0;
+    }
+    if (e == cudaSuccess) e = cudaMemsetAsync(net->ws + net->state_region_off, 0, net->state_region_bytes, net->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(net->ws + net->counters_off, 0, net->L.size() * sizeof(unsigned long long), net->stream);
+    if (e != cudaSuccess) { net->phase = CREATED; return fail(IDF_ERR_CUDA, "stream_open: %s", cudaGetErrorString(e)); }
+    net->phase = OPEN;
+    net->launches = 0;
+    net->out_rows_total = 0;
+    return IDF_OK;
+}
+
+int idf_stream_push(idf_net* net, const void* d_segments, int n_seg, void* d_out, long long out_capacity_rows,
+                    int* rows_emitted)
+{
+    if (!net) return fail(IDF_ERR_ARG, "net must not be NULL");
+    if (net->phase != OPEN) return fail(IDF_ERR_STATE, net->phase == CREATED ? "push before stream_open" : "push after stream_finish");
+    if (n_seg < 0 || out_capacity_rows < 0) return fail(IDF_ERR_ARG, "negative count");
+    if (rows_emitted) *rows_emitted = 0;
+    if (n_seg == 0) return IDF_OK;
+    if (!d_segments || !d_out) return fail(IDF_ERR_ARG, "d_segments and d_out must not be NULL");
+    long long em = 0;
+    int rc = run_segments(net, d_segments, n_seg, false, d_out, out_capacity_rows, &em);
+    if (rc != IDF_OK) return rc;
+    net->out_rows_total += em;
+    if (rows_emitted) *rows_emitted = (int)em;
+    return IDF_OK;
+}
+
+int idf_stream_finish(idf_net* net, void* d_out, long long out_capacity_rows, long long* total_rows)
+{
+    if (!net) return fail(IDF_ERR_ARG, "net must not be NULL");
+    if (net->phase != OPEN) return fail(IDF_ERR_STATE, net->phase == CREATED ? "finish before stream_open" : "finish called twice");
+    if (!d_out || out_capacity_rows < 0) return fail(IDF_ERR_ARG, "d_out must not be NULL");
+    long long em = 0;
+    int rc = run_segments(net, nullptr, 0, true, d_out, out_capacity_rows, &em);
+    if (rc != IDF_OK) return rc;
+    net->out_rows_total += em;
+    net->phase = FINISHED;
+    if (total_rows) *total_rows = net->out_rows_total;
+    return IDF_OK;
+}
+
+int idf_run_host(idf_net* net, const void* h_segments, int n_seg, void* d_segments, void* h_out, void* d_out,
+                 long long out_capacity_rows, long long* total_rows)
+{
+    if (!net || !h_segments || !d_segments || !h_out || !d_out) return fail(IDF_ERR_ARG, "NULL argument");
+    if (net->phase != OPEN || net->L[0].rows_in != 0) return fail(IDF_ERR_STATE, "run_host needs a freshly opened handle");
+    if (n_seg < 0) return fail(IDF_ERR_ARG, "negative count");
+    const size_t in_bytes = (size_t)n_seg * net->n_streams * net->in_w * net->in_c * elem_size(net->L[0].in_elem);
+    cudaError_t e = cudaMemcpyAsync(d_segments, h_segments, in_bytes, cudaMemcpyHostToDevice, net->stream);
+    if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "run_host h2d: %s", cudaGetErrorString(e));
+    int rc = idf_stream_push(net, d_segments, n_seg, d_out, out_capacity_rows, nullptr);
+    if (rc != IDF_OK) return rc;
+    long long tot = 0;
+    rc = idf_stream_finish(net, d_out, out_capacity_rows, &tot);
+    if (rc != IDF_OK) return rc;
+    const LayerPlan& P = net->L.back();
+    const size_t out_bytes = (size_t)net->n_streams * out_capacity_rows * P.out_w * P.out_c * elem_size(P.out_elem);
+    e = cudaMemcpyAsync(h_out, d_out, out_bytes, cudaMemcpyDeviceToHost, net->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(net->stream);
+    if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "run_host d2h: %s", cudaGetErrorString(e));
+    if (total_rows) *total_rows = tot;
+    return IDF_OK;
+}
+
+int idf_event_counts(idf_net* net, long long* events)
+{
+    if (!net || !events) return fail(IDF_ERR_ARG, "NULL argument");
+    if (net->phase == CREATED) return fail(IDF_ERR_STATE, "no open stream");
+    cudaError_t e = cudaMemcpyAsync(events, net->ws + net->counters_off, net->L.size() * sizeof(long long),
+                                    cudaMemcpyDeviceToHost, net->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(net->stream);
+    if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "event_counts: %s", cudaGetErrorString(e));
+    return IDF_OK;
+}
+
+long long idf_launch_count(const idf_net* net) { return net ? net->launches : 0; }
+
+int idf_set_timing(idf_net* net, int on)
+{
+    if (!net) return fail(IDF_ERR_ARG, "net must not be NULL");
+    net->timing = on != 0;
+    return IDF_OK;
+}
+
+int idf_layer_times(idf_net* net, double* ms, long long* launches)
+{
+    if (!net || !ms || !launches) return fail(IDF_ERR_ARG, "NULL argument");
+    for (size_t i = 0; i < net->L.size(); ++i) { ms[i] = 0.0; launches[i] = 0; }
+    if (net->timed.empty()) return IDF_OK;
+    cudaError_t e = cudaStreamSynchronize(net->stream);
+    if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "layer_times: %s", cudaGetErrorString(e));
+    for (auto& t : net->timed) {
+        float f = 0.f;
+        if (cudaEventElapsedTime(&f, t.a, t.b) == cudaSuccess) { ms[t.layer] += f; launches[t.layer] += 1; }
+        net->event_pool.push_back(t.a);
+        net->event_pool.push_back(t.b);
+    }
+    net->timed.clear();
+    return IDF_OK;
+}
+
+}  // extern "C"

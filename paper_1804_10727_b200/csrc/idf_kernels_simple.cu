@@ -1,0 +1,350 @@
+// CUDA-core kernels: the general path for every type and shape.
+//
+//  conv_rows_kernel    dense Δ-row update + row finalisation (Eq. 4 applied tap by tap, then Eq. 2-3
+//                      once per unit), one thread per ring-slot element
+//  conv_sparse_kernel  compaction of the non-zero Δ-events of a row (warp ballot + prefix sum) and
+//                      scatter of w*Δh into the ring (Eq. 4 event by event), one CTA per stream
+//  pool_rows_kernel    2x2 max-pool fold with a one-row running maximum
+#include "idf_internal.h"
+
+namespace idf {
+
+__device__ __forceinline__ float to_acc(float v) { return v; }
+__device__ __forceinline__ float to_acc(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ int to_acc(int8_t v) { return (int)v; }
+
+template <typename TO, typename TS>
+struct Emit;
+template <>
+struct Emit<float, float> {
+    static __device__ __forceinline__ float run(float c, float b, int relu, int) {
+        float v = c + b;
+        return (relu && v < 0.f) ? 0.f : v;
+    }
+};
+template <>
+struct Emit<__nv_bfloat16, float> {
+    static __device__ __forceinline__ __nv_bfloat16 run(float c, float b, int relu, int) {
+        float v = c + b;
+        if (relu && v < 0.f) v = 0.f;
+        return __float2bfloat16_rn(v);
+    }
+};
+template <>
+struct Emit<int8_t, int> {
+    static __device__ __forceinline__ int8_t run(int c, int b, int relu, int shift) {
+        int v = c + b;
+        if (relu && v < 0) v = 0;
+        if (shift > 0) v = (v + (1 << (shift - 1))) >> shift;   // arithmetic shift = floor division
+        const int lo = relu ? 0 : -127;
+        v = v < lo ? lo : (v > 127 ? 127 : v);
+        return (int8_t)v;
+    }
+};
+
+// ------------------------------------------------------------------------------------------------
+// Dense update + finalisation.  One thread owns one element (slot, stream, x, co) of the ring and
+// walks, in order, every output row of this block that lives in that slot, so a slot is never read
+// and written by different threads.  Weights: [Kh][Kw][Cin][Cout] (threads of a warp differ in co).
+// ------------------------------------------------------------------------------------------------
+template <typename TI, typename TW, typename TS, typename TO>
+__global__ void __launch_bounds__(256) conv_rows_kernel(ConvArgs a)
+{
+    const TI* __restrict__ in = (const TI*)a.in;
+    const TW* __restrict__ w = (const TW*)a.w;
+    const TS* __restrict__ bias = (const TS*)a.bias;
+    TS* ring = (TS*)a.ring;
+    TO* out = (TO*)a.out;
+    const long long row_elems = (long long)a.Wout * a.Cout;
+    const long long total = (long long)a.ring_rows * a.S * row_elems;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int co = (int)(idx % a.Cout);
+        long long t = idx / a.Cout;
+        const int x = (int)(t % a.Wout);
+        t /= a.Wout;
+        const int s = (int)(t % a.S);
+        const int slot = (int)(t / a.S);
+        const TS b = bias ? bias[co] : (TS)0;
+        // first visited row that lives in this slot
+        long long o = a.o_begin + ((slot - a.o_begin % a.ring_rows) + a.ring_rows) % a.ring_rows;
+        bool dirty = false;
+        TS leave = 0;
+        TS* rp = ring + ((long long)slot * a.S + s) * row_elems + (long long)x * a.Cout + co;
+        for (; o < a.o_end; o += a.ring_rows) {
+            TS acc = 0;
+            for (int ky = 0; ky < a.Kh; ++ky) {
+                const long long r = o * a.stride - a.pad + ky;
+                if (r < a.r0 || r >= a.r1) continue;
+                const TI* row = in + ((r - a.r0) * a.S + s) * (long long)a.Win * a.Cin;
+                for (int kx = 0; kx < a.Kw; ++kx) {
+                    const int ix = x * a.stride_x - a.pad_x + kx;
+                    if (ix < 0 || ix >= a.Win) continue;
+                    const TI* ap = row + (long long)ix * a.Cin;
+                    const TW* wp = w + ((long long)(ky * a.Kw + kx) * a.Cin) * a.Cout + co;
+                    for (int ci = 0; ci < a.Cin; ++ci) acc += to_acc(ap[ci]) * to_acc(wp[(long long)ci * a.Cout]);
+                }
+            }
+            const bool carried_in = (a.r0 > 0) && (o * a.stride - a.pad < a.r0);
+            const TS c = acc + (carried_in ? *rp : (TS)0);
+            if (o < a.done_end) {
+                out[(o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride +
+                    (long long)x * a.Cout + co] = Emit<TO, TS>::run(c, b, a.relu, a.shift);
+                if (carried_in) { dirty = true; leave = 0; }
+            } else {
+                dirty = true;
+                leave = c;
+            }
+        }
+        if (dirty) *rp = leave;
+    }
+}
+
+template <typename TI, typename TW, typename TS, typename TO>
+static cudaError_t launch_rows(const ConvArgs& a, cudaStream_t st)
+{
+    const long long total = (long long)a.ring_rows * a.S * a.Wout * a.Cout;
+    if (total == 0 || a.o_end <= a.o_begin) return cudaSuccess;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148LL * 64) blocks = 148LL * 64;
+    conv_rows_kernel<TI, TW, TS, TO><<<(unsigned)blocks, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_conv_simple(const ConvArgs& a, int dtype, cudaStream_t st)
+{
+    if (dtype == 0) return launch_rows<float, float, float, float>(a, st);
+    if (dtype == 1) {
+        if (a.in_elem != E_BF16) return cudaErrorInvalidValue;
+        if (a.out_elem == E_BF16) return launch_rows<__nv_bfloat16, float, float, __nv_bfloat16>(a, st);
+        return launch_rows<__nv_bfloat16, float, float, float>(a, st);
+    }
+    return launch_rows<int8_t, int8_t, int, int8_t>(a, st);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Sparse-event path.  One CTA owns one stream and takes the block's input rows in order:
+//   1. compaction: each warp looks at 32 input components at a time, ballots "non-zero", and
+//      appends the survivors (position, channel, value) to a list in shared memory at the offset
+//      given by the prefix popcount of the ballot (Eq. 3: only non-zero events are sent);
+//   2. scatter: every (event, kernel tap, output channel) triple adds w*Δh to the ring row it
+//      reaches (Eq. 4) with shared-memory atomics (or global atomics when the ring is too large
+//      for shared memory; the ring of a stream is private to its CTA either way);
+//   3. finalisation of the ring rows that this input row completed: emit f(c + b), zero the slot.
+// Rows still open at the end of the block go back to the ring in global memory.
+// ------------------------------------------------------------------------------------------------
+constexpr int SPARSE_THREADS = 256;
+constexpr int SPARSE_MAX_EVENTS = 2048;   // list capacity per pass; longer rows take several passes
+
+template <typename TS> __device__ __forceinline__ void atomic_add(TS* p, TS v) { atomicAdd(p, v); }
+
+template <typename TI, typename TW, typename TS, typename TO, bool RING_IN_SMEM>
+__global__ void __launch_bounds__(SPARSE_THREADS) conv_sparse_kernel(ConvArgs a)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ int ev_pos[SPARSE_MAX_EVENTS];      // x * Cin + ci
+    __shared__ TS ev_val[SPARSE_MAX_EVENTS];
+    __shared__ int ev_count;
+    __shared__ unsigned long long ev_total;
+
+    const int s = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const TI* __restrict__ in = (const TI*)a.in;
+    const TW* __restrict__ w = (const TW*)a.w;
+    const TS* __restrict__ bias = (const TS*)a.bias;
+    TO* out = (TO*)a.out;
+    const int row_elems = a.Wout * a.Cout;
+    TS* gring = (TS*)a.ring;     // element (slot, s, x, co) at ((slot*S + s)*row_elems + x*Cout + co)
+    TS* ring = RING_IN_SMEM ? (TS*)smem_raw : gring;
+    const long long slot_stride = RING_IN_SMEM ? row_elems : (long long)a.S * row_elems;
+    const long long ring_base = RING_IN_SMEM ? 0 : (long long)s * row_elems;
+
+    if (tid == 0) ev_total = 0;
+    if (RING_IN_SMEM) {
+        for (int i = tid; i < a.ring_rows * row_elems; i += SPARSE_THREADS) {
+            const int slot = i / row_elems, e = i - slot * row_elems;
+            ring[i] = gring[((long long)slot * a.S + s) * row_elems + e];
+        }
+    }
+    __syncthreads();
+
+    const int n_comp = a.Win * a.Cin;
+    const int taps = a.Kh * a.Kw;
+    long long done = a.o_begin;                      // rows below `done` have been emitted
+    for (long long r = a.r0; r <= a.r1; ++r) {
+        // r == r1 is the flush pass: no input, only rows up to done_end are finalised
+        if (r < a.r1) {
+            const TI* row = in + ((r - a.r0) * a.S + s) * (long long)n_comp;
+            for (int base = 0; base < n_comp; base += SPARSE_MAX_EVENTS) {
+                if (tid == 0) ev_count = 0;
+                __syncthreads();
+                const int lim = min(n_comp, base + SPARSE_MAX_EVENTS);
+                for (int i0 = base + (tid - lane); i0 < lim; i0 += SPARSE_THREADS) {
+                    const int i = i0 + lane;
+                    const TS v = (i < lim) ? (TS)to_acc(row[i]) : (TS)0;
+                    const unsigned m = __ballot_sync(0xffffffffu, v != (TS)0);
+                    if (m) {
+                        int off = 0;
+                        if (lane == 0) off = atomicAdd(&ev_count, __popc(m));
+                        off = __shfl_sync(0xffffffffu, off, 0);
+                        if (v != (TS)0) {
+                            const int k = off + __popc(m & ((1u << lane) - 1u));
+                            ev_pos[k] = i;
+                            ev_val[k] = v;
+                        }
+                    }
+                }
+                __syncthreads();
+                const int n_ev = ev_count;
+                if (tid == 0) ev_total += (unsigned long long)n_ev;
+                // scatter: item = (event, tap, co); consecutive threads differ in co
+                const long long items = (long long)n_ev * taps * a.Cout;
+                for (long long it = tid; it < items; it += SPARSE_THREADS) {
+                    const int co = (int)(it % a.Cout);
+                    const int t2 = (int)(it / a.Cout);
+                    const int tap = t2 % taps, e = t2 / taps;
+                    const int ky = tap / a.Kw, kx = tap - ky * a.Kw;
+                    const int pos = ev_pos[e];
+                    const int x = pos / a.Cin, ci = pos - x * a.Cin;
+                    const long long ty = r + a.pad - ky;
+                    const int tx = x + a.pad_x - kx;
+                    if (ty < 0 || tx < 0 || ty % a.stride || tx % a.stride_x) continue;
+                    const long long o = ty / a.stride;
+                    const int ox = tx / a.stride_x;
+                    if (ox >= a.Wout || o < a.o_begin) continue;
+                    const TS wv = (TS)to_acc(w[((long long)(ky * a.Kw + kx) * a.Cin + ci) * a.Cout + co]);
+                    atomic_add(&ring[ring_base + (o % a.ring_rows) * slot_stride + (long long)ox * a.Cout + co],
+                               ev_val[e] * wv);
+                }
+                __syncthreads();
+            }
+        }
+        // rows completed by input row r (or, in the flush pass, everything below done_end)
+        long long upto;
+        if (r < a.r1) {
+            const long long q = r + a.pad - a.Kh + 1;    // row o completes at r = o*stride - pad + Kh - 1
+            upto = q < 0 ? 0 : q / a.stride + 1;
+            if (upto > a.done_end) upto = a.done_end;
+        } else {
+            upto = a.done_end;
+        }
+        for (; done < upto; ++done) {
+            const long long slot = done % a.ring_rows;
+            for (int i = tid; i < row_elems; i += SPARSE_THREADS) {
+                TS* p = &ring[ring_base + slot * slot_stride + i];
+                const TS c = *p;
+                *p = 0;
+                const int co = i % a.Cout;
+                out[(done - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride + i] =
+                    Emit<TO, TS>::run(c, bias ? bias[co] : (TS)0, a.relu, a.shift);
+            }
+        }
+        __syncthreads();
+    }
+    if (RING_IN_SMEM) {
+        for (int i = tid; i < a.ring_rows * row_elems; i += SPARSE_THREADS) {
+            const int slot = i / row_elems, e = i - slot * row_elems;
+            gring[((long long)slot * a.S + s) * row_elems + e] = ring[i];
+        }
+    }
+    if (tid == 0 && a.event_counter && ev_total) atomicAdd(a.event_counter, ev_total);
+}
+
+size_t conv_sparse_max_smem() { return 200 * 1024; }
+
+template <typename TI, typename TW, typename TS, typename TO>
+static cudaError_t launch_sparse_t(const ConvArgs& a, cudaStream_t st)
+{
+    if (a.S == 0) return cudaSuccess;
+    const size_t ring_bytes = (size_t)a.ring_rows * a.Wout * a.Cout * sizeof(TS);
+    if (ring_bytes <= conv_sparse_max_smem()) {
+        auto k = conv_sparse_kernel<TI, TW, TS, TO, true>;
+        cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring_bytes);
+        if (e != cudaSuccess) return e;
+        k<<<a.S, SPARSE_THREADS, ring_bytes, st>>>(a);
+    } else {
+        conv_sparse_kernel<TI, TW, TS, TO, false><<<a.S, SPARSE_THREADS, 0, st>>>(a);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_conv_sparse(const ConvArgs& a, int dtype, cudaStream_t st)
+{
+    if (dtype == 0) return launch_sparse_t<float, float, float, float>(a, st);
+    if (dtype == 1) {
+        if (a.in_elem != E_BF16) return cudaErrorInvalidValue;
+        if (a.out_elem == E_BF16) return launch_sparse_t<__nv_bfloat16, float, float, __nv_bfloat16>(a, st);
+        return launch_sparse_t<__nv_bfloat16, float, float, float>(a, st);
+    }
+    return launch_sparse_t<int8_t, int8_t, int, int8_t>(a, st);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Max-pool fold: the x-pair is reduced at once; the first row of a y-pair waits in a one-row
+// running maximum; the second row emits.  Width-1 maps pool over rows only.
+// ------------------------------------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ T max_of(T a, T b) { return a > b ? a : b; }
+template <> __device__ __forceinline__ __nv_bfloat16 max_of(__nv_bfloat16 a, __nv_bfloat16 b)
+{
+    return __bfloat162float(a) > __bfloat162float(b) ? a : b;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) pool_rows_kernel(PoolArgs a)
+{
+    const T* __restrict__ in = (const T*)a.in;
+    T* state = (T*)a.state;
+    T* out = (T*)a.out;
+    const int px = (a.Win == 1) ? 1 : 2;
+    const long long total = (long long)a.S * a.Wout * a.C;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(idx % a.C);
+        long long t = idx / a.C;
+        const int ox = (int)(t % a.Wout);
+        const int s = (int)(t / a.Wout);
+        for (long long o = a.o_begin; o < a.o_end; ++o) {
+            bool have = false;
+            T m = (T)0;
+            if (2 * o < a.r0) { m = state[idx]; have = true; }
+            for (int dy = 0; dy < 2; ++dy) {
+                const long long r = 2 * o + dy;
+                if (r < a.r0 || r >= a.r1) continue;
+                const T* row = in + ((r - a.r0) * a.S + s) * (long long)a.Win * a.C;
+                for (int dx = 0; dx < px; ++dx) {
+                    const T v = row[(long long)(px * ox + dx) * a.C + c];
+                    m = have ? max_of(m, v) : v;
+                    have = true;
+                }
+            }
+            if (o < a.done_end)
+                out[(o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride +
+                    (long long)ox * a.C + c] = m;
+            else
+                state[idx] = m;
+        }
+    }
+}
+
+template <typename T>
+static cudaError_t launch_pool_t(const PoolArgs& a, cudaStream_t st)
+{
+    const long long total = (long long)a.S * a.Wout * a.C;
+    if (total == 0 || a.o_end <= a.o_begin) return cudaSuccess;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148LL * 32) blocks = 148LL * 32;
+    pool_rows_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pool(const PoolArgs& a, cudaStream_t st)
+{
+    switch (a.elem) {
+        case E_F32: return launch_pool_t<float>(a, st);
+        case E_BF16: return launch_pool_t<__nv_bfloat16>(a, st);
+        case E_I8: return launch_pool_t<int8_t>(a, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace idf

@@ -1,0 +1,257 @@
+"""Thin ctypes binding over the C ABI in ``include/idf.h`` (argument marshalling only).
+
+PyTorch provides device memory and CUDA streams; every step of the path runs in
+the library's kernels.  There is no fallback: if ``libidf.so`` has not been
+built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = Path(__file__).resolve().parent
+LIB_PATH = _HERE / "libidf.so"
+_lib = None
+
+F32, BF16_F32, I8_I32 = 0, 1, 2
+CONV, MAXPOOL2 = 0, 1
+PATH_AUTO, PATH_DENSE, PATH_SPARSE = 0, 1, 2
+DTYPES = {"f32": F32, "bf16": BF16_F32, "i8": I8_I32}
+
+OK, ERR_ARG, ERR_SPEC, ERR_STATE, ERR_CAPACITY, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5, -6, -7
+
+EXPORTS = (
+    "idf_net_create", "idf_net_destroy", "idf_net_state_bytes", "idf_net_workspace_bytes", "idf_out_shape",
+    "idf_stream_open", "idf_stream_push", "idf_stream_finish", "idf_run_host", "idf_event_counts",
+    "idf_launch_count", "idf_set_timing", "idf_layer_times", "idf_last_error",
+)
+
+
+class IdfLayer(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in
+                ("kind", "cin", "cout", "kh", "kw", "stride", "pad", "relu", "shift", "path")]
+
+
+class IdfSpec(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int), ("layers", ctypes.POINTER(IdfLayer)), ("dtype", ctypes.c_int),
+                ("in_w", ctypes.c_int), ("in_c", ctypes.c_int), ("n_streams", ctypes.c_int),
+                ("row_block", ctypes.c_int)]
+
+
+class IdfError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"idf error {code}: {msg}")
+        self.code = code
+
+
+def lib():
+    """Load ``libidf.so`` (built by ``python -m paper_1804_10727_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_1804_10727_b200.build` "
+                               "(there is no CPU fallback)")
+        L = ctypes.CDLL(str(LIB_PATH))
+        vp, ll, sz = ctypes.c_void_p, ctypes.c_longlong, ctypes.c_size_t
+        L.idf_net_create.argtypes = [ctypes.POINTER(IdfSpec), ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
+        L.idf_net_destroy.argtypes = [vp]
+        L.idf_net_state_bytes.argtypes = [vp]; L.idf_net_state_bytes.restype = sz
+        L.idf_net_workspace_bytes.argtypes = [vp]; L.idf_net_workspace_bytes.restype = sz
+        L.idf_out_shape.argtypes = [vp, ll, ctypes.POINTER(ll), ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
+        L.idf_stream_open.argtypes = [vp, vp, sz, vp]
+        L.idf_stream_push.argtypes = [vp, vp, ctypes.c_int, vp, ll, ctypes.POINTER(ctypes.c_int)]
+        L.idf_stream_finish.argtypes = [vp, vp, ll, ctypes.POINTER(ll)]
+        L.idf_run_host.argtypes = [vp, vp, ctypes.c_int, vp, vp, vp, ll, ctypes.POINTER(ll)]
+        L.idf_event_counts.argtypes = [vp, ctypes.POINTER(ll)]
+        L.idf_launch_count.argtypes = [vp]; L.idf_launch_count.restype = ll
+        L.idf_set_timing.argtypes = [vp, ctypes.c_int]
+        L.idf_layer_times.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
+        L.idf_last_error.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise IdfError(rc, lib().idf_last_error().decode())
+
+
+def _layer_struct(l) -> IdfLayer:
+    kind = l.kind if isinstance(l.kind, int) else {"conv": CONV, "pool": MAXPOOL2}[l.kind]
+    return IdfLayer(kind, l.cin, l.cout, l.kh, l.kw, l.stride, l.pad, l.relu, l.shift, l.path)
+
+
+def _act_torch_dtype(dtype: int):
+    return {F32: torch.float32, BF16_F32: torch.bfloat16, I8_I32: torch.int8}[dtype]
+
+
+def to_act_bits(a: np.ndarray, dtype: int) -> np.ndarray:
+    """Host array in the activation type's memory format (bf16 -> uint16 bit patterns)."""
+    if dtype == F32:
+        return np.ascontiguousarray(a, dtype=np.float32)
+    if dtype == I8_I32:
+        return np.ascontiguousarray(a, dtype=np.int8)
+    t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(torch.bfloat16)
+    return t.view(torch.int16).numpy().view(np.uint16)
+
+
+class Net:
+    """A net handle: ``net_create`` on construction, ``net_destroy`` on close()."""
+
+    def __init__(self, dtype, layers: Sequence, in_w: int, in_c: int, n_streams: int,
+                 weights: Sequence[Optional[np.ndarray]], biases: Optional[Sequence[Optional[np.ndarray]]] = None,
+                 row_block: int = 0):
+        self.dtype = DTYPES[dtype] if isinstance(dtype, str) else int(dtype)
+        self.n_streams, self.in_w, self.in_c = int(n_streams), int(in_w), int(in_c)
+        n = len(layers)
+        self._layers = (IdfLayer * n)(*[_layer_struct(l) for l in layers])
+        spec = IdfSpec(n, self._layers, self.dtype, in_w, in_c, n_streams, row_block)
+        keep = []
+        wptr = (ctypes.c_void_p * n)()
+        bptr = (ctypes.c_void_p * n)()
+        for i in range(n):
+            if weights[i] is not None:
+                w = to_act_bits(weights[i], self.dtype)
+                keep.append(w)
+                wptr[i] = w.ctypes.data
+            if biases is not None and biases[i] is not None:
+                b = np.ascontiguousarray(biases[i], dtype=np.int32 if self.dtype == I8_I32 else np.float32)
+                keep.append(b)
+                bptr[i] = b.ctypes.data
+        h = ctypes.c_void_p()
+        _check(lib().idf_net_create(ctypes.byref(spec), wptr, bptr, ctypes.byref(h)))
+        self._h = h
+        self._ws = None
+        self.n_layers = n
+
+    # -- queries ---------------------------------------------------------------------------------
+    @property
+    def state_bytes(self) -> int:
+        return int(lib().idf_net_state_bytes(self._h))
+
+    @property
+    def workspace_bytes(self) -> int:
+        return int(lib().idf_net_workspace_bytes(self._h))
+
+    def out_shape(self, in_rows: int):
+        r, w, c = ctypes.c_longlong(), ctypes.c_int(), ctypes.c_int()
+        _check(lib().idf_out_shape(self._h, in_rows, ctypes.byref(r), ctypes.byref(w), ctypes.byref(c)))
+        return int(r.value), int(w.value), int(c.value)
+
+    @property
+    def out_torch_dtype(self):
+        return torch.int8 if self.dtype == I8_I32 else torch.float32
+
+    @property
+    def act_torch_dtype(self):
+        return _act_torch_dtype(self.dtype)
+
+    @property
+    def launches(self) -> int:
+        return int(lib().idf_launch_count(self._h))
+
+    def event_counts(self):
+        ev = (ctypes.c_longlong * self.n_layers)()
+        _check(lib().idf_event_counts(self._h, ev))
+        return list(ev)
+
+    def set_timing(self, on: bool):
+        _check(lib().idf_set_timing(self._h, int(on)))
+
+    def layer_times(self):
+        """(ms, launches) per layer since the last query; synchronises the stream."""
+        ms = (ctypes.c_double * self.n_layers)()
+        n = (ctypes.c_longlong * self.n_layers)()
+        _check(lib().idf_layer_times(self._h, ms, n))
+        return list(ms), list(n)
+
+    # -- streaming -------------------------------------------------------------------------------
+    def open(self, device="cuda:0", stream: Optional[torch.cuda.Stream] = None, workspace: Optional[torch.Tensor] = None):
+        if workspace is None:
+            if self._ws is None or self._ws.device != torch.device(device):
+                self._ws = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=device)
+            workspace = self._ws
+        self._ws = workspace
+        base = workspace.data_ptr()
+        aligned = (base + 255) // 256 * 256
+        nbytes = workspace.numel() - (aligned - base)
+        st = stream.cuda_stream if stream is not None else torch.cuda.current_stream(workspace.device).cuda_stream
+        _check(lib().idf_stream_open(self._h, aligned, nbytes, st))
+
+    def alloc_out(self, in_rows: int, device="cuda:0") -> torch.Tensor:
+        r, w, c = self.out_shape(in_rows)
+        return torch.zeros((self.n_streams, max(r, 1), w, c), dtype=self.out_torch_dtype, device=device)
+
+    def push(self, segments: torch.Tensor, out: torch.Tensor) -> int:
+        """segments: device tensor [n_seg][n_streams][in_w][in_c] in the activation type."""
+        assert segments.is_cuda and segments.is_contiguous() and out.is_cuda and out.is_contiguous()
+        assert segments.dtype == self.act_torch_dtype and out.dtype == self.out_torch_dtype
+        assert tuple(segments.shape[1:]) == (self.n_streams, self.in_w, self.in_c), segments.shape
+        em = ctypes.c_int()
+        _check(lib().idf_stream_push(self._h, segments.data_ptr(), segments.shape[0], out.data_ptr(), out.shape[1],
+                                     ctypes.byref(em)))
+        return int(em.value)
+
+    def finish(self, out: torch.Tensor) -> int:
+        tot = ctypes.c_longlong()
+        _check(lib().idf_stream_finish(self._h, out.data_ptr(), out.shape[1], ctypes.byref(tot)))
+        return int(tot.value)
+
+    def run_host(self, h_segments: torch.Tensor, d_segments: torch.Tensor, h_out: torch.Tensor, d_out: torch.Tensor) -> int:
+        """Whole streams from (pinned) host memory and back; see idf_run_host."""
+        assert not h_segments.is_cuda and not h_out.is_cuda and d_segments.is_cuda and d_out.is_cuda
+        assert h_segments.is_contiguous() and h_out.is_contiguous()
+        assert h_segments.dtype == self.act_torch_dtype and h_out.dtype == self.out_torch_dtype
+        assert h_out.shape == d_out.shape and h_segments.shape == d_segments.shape
+        tot = ctypes.c_longlong()
+        _check(lib().idf_run_host(self._h, h_segments.data_ptr(), h_segments.shape[0], d_segments.data_ptr(),
+                                  h_out.data_ptr(), d_out.data_ptr(), d_out.shape[1], ctypes.byref(tot)))
+        return int(tot.value)
+
+    def close(self):
+        if self._h:
+            lib().idf_net_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def segments_from_maps(x: np.ndarray, dtype) -> torch.Tensor:
+    """Host maps [n_streams][H][W][C] -> host tensor [H][n_streams][W][C] in the activation type."""
+    d = DTYPES[dtype] if isinstance(dtype, str) else dtype
+    t = torch.from_numpy(np.ascontiguousarray(x))
+    t = t.permute(1, 0, 2, 3).contiguous()
+    return t.to(_act_torch_dtype(d))
+
+
+def net_from_workload(w, weights, biases, n_streams: Optional[int] = None, row_block: int = 0) -> Net:
+    return Net(w.dtype, w.layers, w.W, w.C, n_streams or w.n_streams, weights, biases, row_block=row_block)
+
+
+def infer(net: Net, x: np.ndarray, chunks: Optional[Sequence[int]] = None, device="cuda:0") -> np.ndarray:
+    """Run whole maps x [n_streams][H][W][C] through the net; ``chunks`` gives the number of
+    segments per push (default: one push).  Returns the output map as a numpy array."""
+    seg = segments_from_maps(x, net.dtype).to(device)
+    H = seg.shape[0]
+    out = net.alloc_out(H, device)
+    net.open(device)
+    pos = 0
+    for n in (chunks or [H]):
+        n = min(n, H - pos)
+        if n > 0:
+            net.push(seg[pos:pos + n], out)
+        pos += n
+    if pos < H:
+        net.push(seg[pos:], out)
+    rows = net.finish(out)
+    torch.cuda.synchronize()
+    assert rows == net.out_shape(H)[0], (rows, net.out_shape(H))
+    return out[:, :rows].cpu().numpy()

@@ -47,7 +47,8 @@ def _torch_forward(mode, layers, x, ws, bs):
         if l.kind == "conv":
             w = torch.tensor(np.asarray(ws[i], dtype=np.float64)).permute(0, 3, 1, 2)  # [Cout][Cin][Kh][Kw]
             b = None if bs[i] is None else torch.tensor(np.asarray(bs[i], dtype=np.float64))
-            a = F.conv2d(a, w, b, stride=l.stride, padding=l.pad)
+            one_d = a.shape[3] == 1 and l.kw == 1
+            a = F.conv2d(a, w, b, stride=(l.stride, 1 if one_d else l.stride), padding=(l.pad, 0 if one_d else l.pad))
             if l.relu:
                 a = F.relu(a)
             if mode == "bf16" and i != convs[-1]:
@@ -72,6 +73,7 @@ NETS = {
     "stride2_pad": (conv(2, 3, 3, stride=2, pad=1), conv(3, 4, 3, stride=2, pad=1)),
     "oned_k9": (conv(1, 4, 9, stride=2, one_d=True), conv(4, 5, 9, one_d=True)),
     "oned_k3": (conv(1, 8, 3, one_d=True), conv(8, 8, 3, one_d=True), conv(8, 4, 3, one_d=True)),
+    "oned_pad": (conv(2, 3, 5, stride=2, pad=2, one_d=True), POOL, conv(3, 4, 3, pad=1, one_d=True)),
     "k5": (conv(2, 3, 5, stride=2, pad=2), conv(3, 2, 3)),
     "norelu": (conv(2, 3, 3, relu=0), conv(3, 2, 3, relu=0)),
 }
