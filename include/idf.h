@@ -156,6 +156,38 @@ long long idf_launch_count(const idf_net* net);
 int idf_set_timing(idf_net* net, int on);
 int idf_layer_times(idf_net* net, double* ms, long long* launches);
 
+/* One fp32 conv layer over whole streams, for callers that cannot allocate device memory.
+ * (The paper has no counterpart to this call; it exists for deployment reasons only.)
+ *
+ * Some callers hold nothing but their input and output buffers at the moment they need a result:
+ * a plugin handed two pointers by its host program, code inside a pre-partitioned memory pool, a
+ * latency-critical loop that must keep away from the allocator.  They cannot supply the workspace
+ * the regular calls need, and this call needs none: the rolling state (ceil(kh/stride) rows per
+ * stream) and the repacked weights live in a fixed array inside the library image, of
+ * IDF_NOALLOC_SCRATCH_BYTES bytes, which every GPU that loads the library holds until exit.
+ * The call allocates and frees nothing, on the device or through any library.
+ *
+ *   d_in      device, [n_rows][n_streams][in_w][cin] fp32 - all segments of every stream
+ *   d_weights device, [cout][kh][kw][cin] fp32;  d_bias device, [cout] fp32 or NULL
+ *   d_out     device, [n_streams][out_capacity_rows][out_w][cout] fp32; receives every output row
+ *             (the end-of-input flush is included), f = ReLU if relu != 0
+ *   out_rows  host, may be NULL: floor((n_rows + 2 pad - kh) / stride) + 1 (0 if negative)
+ *   cuda_stream  a cudaStream_t as void*, NULL = default stream; the work is enqueued, not awaited
+ *
+ * Limits and sharing: ring bytes (rounded up to 256) + weight bytes must fit the array, else
+ * IDF_ERR_CAPACITY and nothing is enqueued.  All calls on a device share the one array, which keeps
+ * the previous call's contents; the call clears the part that must start at zero itself.  Two calls
+ * whose GPU work overlaps in time (different streams, different threads) race on the array and give
+ * wrong results: serialise them.  The first call on each device resolves the array's device address
+ * (a one-time set-up step with that device current); make that first call before any CUDA stream
+ * capture begins.  Results equal those of a one-layer IDF_F32 net run through
+ * idf_stream_push + idf_stream_finish. */
+#define IDF_NOALLOC_SCRATCH_BYTES (8u << 20)
+int idf_conv_rows_noalloc(const float* d_in, int n_rows, int n_streams, int in_w, int cin,
+                          const float* d_weights, const float* d_bias, int cout, int kh, int kw,
+                          int stride, int pad, int relu, float* d_out, long long out_capacity_rows,
+                          long long* out_rows, void* cuda_stream);
+
 /* Message for the most recent failure on the calling thread ("" if none). */
 const char* idf_last_error(void);
 

@@ -229,6 +229,10 @@ int run_segments(idf_net* net, const void* d_segments, long long n_seg, bool flu
 
 }  // namespace
 
+namespace idf {
+int set_last_error(int code, const char* msg) { return fail(code, "%s", msg); }
+}  // namespace idf
+
 extern "C" {
 
 const char* idf_last_error(void) { return g_err.c_str(); }

@@ -27,7 +27,7 @@ OK, ERR_ARG, ERR_SPEC, ERR_STATE, ERR_CAPACITY, ERR_UNSUPPORTED, ERR_CUDA, ERR_T
 EXPORTS = (
     "idf_net_create", "idf_net_destroy", "idf_net_state_bytes", "idf_net_workspace_bytes", "idf_out_shape",
     "idf_stream_open", "idf_stream_push", "idf_stream_finish", "idf_run_host", "idf_event_counts",
-    "idf_launch_count", "idf_set_timing", "idf_layer_times", "idf_last_error",
+    "idf_launch_count", "idf_set_timing", "idf_layer_times", "idf_conv_rows_noalloc", "idf_last_error",
 )
 
 
@@ -70,6 +70,9 @@ def lib():
         L.idf_launch_count.argtypes = [vp]; L.idf_launch_count.restype = ll
         L.idf_set_timing.argtypes = [vp, ctypes.c_int]
         L.idf_layer_times.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
+        L.idf_conv_rows_noalloc.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp,
+                                            ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                            ctypes.c_int, vp, ll, ctypes.POINTER(ll), vp]
         L.idf_last_error.restype = ctypes.c_char_p
         _lib = L
     return _lib
@@ -255,3 +258,30 @@ def infer(net: Net, x: np.ndarray, chunks: Optional[Sequence[int]] = None, devic
     torch.cuda.synchronize()
     assert rows == net.out_shape(H)[0], (rows, net.out_shape(H))
     return out[:, :rows].cpu().numpy()
+
+
+NOALLOC_SCRATCH_BYTES = 8 << 20
+
+
+def conv_rows_noalloc(segments: torch.Tensor, weights: torch.Tensor, bias: Optional[torch.Tensor], stride: int, pad: int,
+                      relu: bool, out: torch.Tensor) -> int:
+    """One fp32 conv layer over whole streams without any device allocation (idf_conv_rows_noalloc).
+
+    For callers that own only their input and output buffers and may not allocate: the ring state
+    and the repacked weights live in a fixed array inside the library (8 MiB per GPU, shared by
+    all calls, so calls must not overlap on the GPU).  ``segments`` [n_rows][n_streams][in_w][cin],
+    ``weights`` [cout][kh][kw][cin], ``out`` [n_streams][capacity][out_w][cout], all fp32 device
+    tensors owned by the caller.  Enqueues on the current stream; returns the number of output rows.
+    """
+    assert segments.is_cuda and weights.is_cuda and out.is_cuda
+    assert segments.dtype == weights.dtype == out.dtype == torch.float32
+    assert segments.is_contiguous() and weights.is_contiguous() and out.is_contiguous()
+    n_rows, S, in_w, cin = segments.shape
+    cout, kh, kw, cin2 = weights.shape
+    assert cin == cin2 and out.shape[0] == S and out.shape[3] == cout
+    rows = ctypes.c_longlong()
+    st = torch.cuda.current_stream(segments.device).cuda_stream
+    _check(lib().idf_conv_rows_noalloc(segments.data_ptr(), n_rows, S, in_w, cin, weights.data_ptr(),
+                                       bias.data_ptr() if bias is not None else None, cout, kh, kw, stride, pad,
+                                       int(relu), out.data_ptr(), out.shape[1], ctypes.byref(rows), st))
+    return int(rows.value)
