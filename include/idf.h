@@ -149,6 +149,11 @@ int idf_event_counts(idf_net* net, long long* events);
 /* Kernel launches enqueued by this handle since open. */
 long long idf_launch_count(const idf_net* net);
 
+/* Wait for the stream and report whether any kernel of this handle gave up on a bounded device-side
+ * wait since idf_stream_open (IDF_ERR_TIMEOUT; results are then invalid).  tensor_core_launches
+ * (host, n_layers entries, may be NULL) receives per layer how many launches took the tcgen05 path. */
+int idf_stream_status(idf_net* net, long long* tensor_core_launches);
+
 /* Per-layer device time.  With timing on, every kernel launch of the handle is bracketed by CUDA
  * events on its stream.  idf_layer_times synchronises the stream, adds up the elapsed time of the
  * launches recorded since the last query into ms[i] (milliseconds, host, n_layers entries) and

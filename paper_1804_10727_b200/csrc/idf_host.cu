@@ -6,6 +6,7 @@
 #include <algorithm>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -36,6 +37,11 @@ struct LayerPlan {
     int ring_rows;           // conv: ceil(kh/stride); pool: 1
     int in_elem, out_elem;   // Elem of the rows this layer receives / emits
     int use_sparse;
+    TcPlan tc;                              // tensor-core path (tc.ok) for the dense update
+    std::vector<unsigned char> wtc_packed;  // [tap][Cout][Cin] in the activation type
+    size_t wtc_off = 0;
+    alignas(64) unsigned char w_map[128];   // TMA descriptor of wtc in the workspace (made at open)
+    long long tc_launches = 0;
     // host copies of the packed parameters
     std::vector<unsigned char> w_packed;   // [Kh][Kw][Cin][Cout] float (float nets) or int8
     std::vector<unsigned char> b_packed;   // [Cout] float / int32 (empty = zero bias)
@@ -55,7 +61,7 @@ enum Phase { CREATED = 0, OPEN = 1, FINISHED = 2 };
 struct idf_net {
     int dtype = 0, in_w = 0, in_c = 0, n_streams = 0, row_block = 0;
     std::vector<LayerPlan> L;
-    size_t workspace_bytes = 0, state_region_off = 0, state_region_bytes = 0, counters_off = 0;
+    size_t workspace_bytes = 0, state_region_off = 0, state_region_bytes = 0, counters_off = 0, status_off = 0;
     size_t state_bytes_stream = 0;
     unsigned char* ws = nullptr;
     cudaStream_t stream = nullptr;
@@ -161,7 +167,13 @@ int advance_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, bo
         a.stride_x = P.in_w == 1 ? 1 : P.l.stride; a.pad_x = P.in_w == 1 ? 0 : P.l.pad;
         a.ring_rows = P.ring_rows; a.in_elem = P.in_elem; a.out_elem = P.out_elem;
         a.r0 = r0; a.r1 = r1; a.o_begin = o_begin; a.o_end = o_end; a.done_end = done_end;
-        ce = P.use_sparse ? launch_conv_sparse(a, net->dtype, net->stream) : launch_conv_simple(a, net->dtype, net->stream);
+        ce = cudaErrorNotSupported;
+        if (P.tc.ok && !P.use_sparse && !flush && n_in > 0) {
+            ce = launch_conv_tc(a, P.tc, net->dtype, P.w_map, (int)n_in, (unsigned int*)(net->ws + net->status_off), net->stream);
+            if (ce == cudaSuccess) P.tc_launches += 1;
+        }
+        if (ce == cudaErrorNotSupported)
+            ce = P.use_sparse ? launch_conv_sparse(a, net->dtype, net->stream) : launch_conv_simple(a, net->dtype, net->stream);
     } else {
         PoolArgs a{};
         a.in = in_ptr;
@@ -313,6 +325,19 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
                             dst[((size_t)k * l.cin + ci) * l.cout + co] = v;
                         }
             }
+            // tensor-core layout [tap][Cout][Cin], activation type, when the layer qualifies
+            const char* no_tc = getenv("IDF_DISABLE_TC");
+            if (!P.use_sparse && !(no_tc && no_tc[0] == '1') &&
+                tc_make_plan(spec->dtype, net->n_streams, w, P.out_w, l.cin, l.cout, l.kh, l.kw, w == 1 ? 1 : l.stride,
+                             P.ring_rows, &P.tc)) {
+                const size_t es = spec->dtype == IDF_I8_I32 ? 1 : 2;
+                P.wtc_packed.resize(nw * es);
+                const int taps = l.kh * l.kw;
+                for (int co = 0; co < l.cout; ++co)
+                    for (int k = 0; k < taps; ++k)
+                        memcpy(P.wtc_packed.data() + (((size_t)k * l.cout + co) * l.cin) * es,
+                               (const unsigned char*)weights[i] + (((size_t)co * taps + k) * l.cin) * es, (size_t)l.cin * es);
+            }
             if (biases && biases[i]) {
                 P.b_packed.resize((size_t)l.cout * 4);
                 memcpy(P.b_packed.data(), biases[i], (size_t)l.cout * 4);
@@ -340,6 +365,7 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
     for (auto& P : net->L) {
         P.w_off = off; off = align_up(off + P.w_packed.size());
         P.b_off = off; off = align_up(off + P.b_packed.size());
+        P.wtc_off = off; off = align_up(off + P.wtc_packed.size(), 1024);
     }
     net->state_region_off = off;
     for (auto& P : net->L) { P.state_off = off; off = align_up(off + P.state_bytes_all); }
@@ -351,6 +377,8 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
     }
     net->counters_off = off;
     off = align_up(off + net->L.size() * sizeof(unsigned long long));
+    net->status_off = off;
+    off = align_up(off + sizeof(unsigned int));
     net->workspace_bytes = off;
     *out = net;
     return IDF_OK;
@@ -396,8 +424,14 @@ int idf_stream_open(idf_net* net, void* d_workspace, size_t workspace_bytes, voi
             e = cudaMemcpyAsync(net->ws + P.w_off, P.w_packed.data(), P.w_packed.size(), cudaMemcpyHostToDevice, net->stream);
         if (!P.b_packed.empty() && e == cudaSuccess)
             e = cudaMemcpyAsync(net->ws + P.b_off, P.b_packed.data(), P.b_packed.size(), cudaMemcpyHostToDevice, net->stream);
-        P.rows_in = 0; P.rows_done = 0;
+        if (!P.wtc_packed.empty() && e == cudaSuccess) {
+            e = cudaMemcpyAsync(net->ws + P.wtc_off, P.wtc_packed.data(), P.wtc_packed.size(), cudaMemcpyHostToDevice, net->stream);
+            if (tc_encode_weights(P.tc, net->dtype, net->ws + P.wtc_off, P.l.kh * P.l.kw, P.l.cin, P.l.cout, P.w_map) != 0)
+                P.tc.ok = 0;               // no TMA descriptor: this layer stays on the CUDA-core kernel
+        }
+        P.rows_in = 0; P.rows_done = 0; P.tc_launches = 0;
     }
+    if (e == cudaSuccess) e = cudaMemsetAsync(net->ws + net->status_off, 0, sizeof(unsigned int), net->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(net->ws + net->state_region_off, 0, net->state_region_bytes, net->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(net->ws + net->counters_off, 0, net->L.size() * sizeof(unsigned long long), net->stream);
     if (e != cudaSuccess) { net->phase = CREATED; return fail(IDF_ERR_CUDA, "stream_open: %s", cudaGetErrorString(e)); }
@@ -473,6 +507,20 @@ int idf_event_counts(idf_net* net, long long* events)
 }
 
 long long idf_launch_count(const idf_net* net) { return net ? net->launches : 0; }
+
+int idf_stream_status(idf_net* net, long long* tensor_core_launches)
+{
+    if (!net) return fail(IDF_ERR_ARG, "net must not be NULL");
+    if (net->phase == CREATED) return fail(IDF_ERR_STATE, "no open stream");
+    unsigned int st = 0;
+    cudaError_t e = cudaMemcpyAsync(&st, net->ws + net->status_off, sizeof st, cudaMemcpyDeviceToHost, net->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(net->stream);
+    if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "stream_status: %s", cudaGetErrorString(e));
+    if (tensor_core_launches)
+        for (size_t i = 0; i < net->L.size(); ++i) tensor_core_launches[i] = net->L[i].tc_launches;
+    if (st != 0) return fail(IDF_ERR_TIMEOUT, "a bounded device-side wait ran out (kernel gave up)");
+    return IDF_OK;
+}
 
 int idf_set_timing(idf_net* net, int on)
 {

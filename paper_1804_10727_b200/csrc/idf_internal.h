@@ -44,6 +44,26 @@ struct PoolArgs {
     long long r0, r1, o_begin, o_end, done_end;
 };
 
+// Static plan of the tensor-core path for one conv layer (tile shapes, shared-memory budget).
+struct TcPlan {
+    int ok = 0;
+    int BX = 0, BS = 0;      // a 128-row M tile = BS streams x BX consecutive x positions
+    int n_xt = 0, n_mt = 0;  // x tiles per row, M tiles in all
+    int Ntile = 0, n_nt = 0; // output channels per CTA, N tiles
+    int KB = 0, n_kb = 0;    // input channels per K block (one swizzled shared-memory row), K blocks
+    int swb = 0;             // bytes of one K-block row: 32, 64 or 128 = the swizzle span
+    int nslot = 0;           // ring rows resident in tensor memory at once (>= ring rows + 1)
+    int nstage = 0;          // Δ-row tiles in flight
+    int tmem_cols = 0;
+    size_t smem_bytes = 0;
+    size_t w_bytes = 0;      // device weights for this path: [tap][Cout][Cin] in the activation type
+};
+bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh, int Kw, int stride_x, int ring_rows,
+                  TcPlan* p);
+int tc_encode_weights(const TcPlan& p, int dtype, const void* d_w, int taps, int Cin, int Cout, void* map_out);
+cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const void* w_map, int n_in_rows,
+                           unsigned int* status, cudaStream_t st);
+
 // CUDA-core kernels (every type, every shape)
 cudaError_t launch_conv_simple(const ConvArgs& a, int dtype, cudaStream_t st);
 cudaError_t launch_conv_sparse(const ConvArgs& a, int dtype, cudaStream_t st);

@@ -27,7 +27,7 @@ OK, ERR_ARG, ERR_SPEC, ERR_STATE, ERR_CAPACITY, ERR_UNSUPPORTED, ERR_CUDA, ERR_T
 EXPORTS = (
     "idf_net_create", "idf_net_destroy", "idf_net_state_bytes", "idf_net_workspace_bytes", "idf_out_shape",
     "idf_stream_open", "idf_stream_push", "idf_stream_finish", "idf_run_host", "idf_event_counts",
-    "idf_launch_count", "idf_set_timing", "idf_layer_times", "idf_conv_rows_noalloc", "idf_last_error",
+    "idf_launch_count", "idf_stream_status", "idf_set_timing", "idf_layer_times", "idf_conv_rows_noalloc", "idf_last_error",
 )
 
 
@@ -68,6 +68,7 @@ def lib():
         L.idf_run_host.argtypes = [vp, vp, ctypes.c_int, vp, vp, vp, ll, ctypes.POINTER(ll)]
         L.idf_event_counts.argtypes = [vp, ctypes.POINTER(ll)]
         L.idf_launch_count.argtypes = [vp]; L.idf_launch_count.restype = ll
+        L.idf_stream_status.argtypes = [vp, ctypes.POINTER(ll)]
         L.idf_set_timing.argtypes = [vp, ctypes.c_int]
         L.idf_layer_times.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
         L.idf_conv_rows_noalloc.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp,
@@ -162,6 +163,12 @@ class Net:
         _check(lib().idf_event_counts(self._h, ev))
         return list(ev)
 
+    def status(self):
+        """Synchronise; raise if a kernel gave up on a bounded wait; return tensor-core launches per layer."""
+        n = (ctypes.c_longlong * self.n_layers)()
+        _check(lib().idf_stream_status(self._h, n))
+        return list(n)
+
     def set_timing(self, on: bool):
         _check(lib().idf_set_timing(self._h, int(on)))
 
@@ -255,6 +262,7 @@ def infer(net: Net, x: np.ndarray, chunks: Optional[Sequence[int]] = None, devic
     if pos < H:
         net.push(seg[pos:], out)
     rows = net.finish(out)
+    net.status()
     torch.cuda.synchronize()
     assert rows == net.out_shape(H)[0], (rows, net.out_shape(H))
     return out[:, :rows].cpu().numpy()

@@ -1,0 +1,87 @@
+"""GPU parity of the tensor-core (tcgen05) dense path: single layers and short nets whose shapes
+qualify for it, against the CPU oracle.  A single bf16 conv layer emits unrounded fp32, so the strict
+float tolerance applies; int8 layers must match bit for bit.  Every case also checks that the
+launches really took the tensor-core path and that no bounded device wait ran out."""
+import numpy as np
+import pytest
+
+from paper_1804_10727_b200 import idf
+from paper_1804_10727_b200.workloads import conv, POOL
+from helpers import assert_close, assert_equal, rand_net, with_shifts
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(mode, layers, x, ws, bs, chunks=None, row_block=0):
+    S, H, W, C = x.shape
+    net = idf.Net(mode, layers, W, C, S, ws, bs, row_block=row_block)
+    seg = idf.segments_from_maps(x, mode).cuda()
+    out = net.alloc_out(H)
+    net.open()
+    pos = 0
+    for n in (chunks or [H]):
+        n = min(n, H - pos)
+        if n > 0:
+            net.push(seg[pos:pos + n], out)
+        pos += n
+    if pos < H:
+        net.push(seg[pos:], out)
+    rows = net.finish(out)
+    tc = net.status()
+    return out[:, :rows].cpu().numpy(), tc
+
+
+# (name, mode, layers, H, W, S)
+CASES = [
+    ("bf16_64_w16", "bf16", (conv(64, 64, 3, pad=1),), 10, 16, 8),
+    ("bf16_64_w16_ragged_streams", "bf16", (conv(64, 64, 3, pad=1),), 11, 16, 5),
+    ("bf16_64_valid", "bf16", (conv(64, 32, 3),), 12, 20, 7),
+    ("bf16_128_w40", "bf16", (conv(128, 64, 3, pad=1),), 9, 40, 4),
+    ("bf16_64_wide", "bf16", (conv(64, 64, 3, pad=1),), 7, 224, 2),
+    ("bf16_64_w130", "bf16", (conv(64, 16, 3, pad=1),), 6, 130, 3),
+    ("bf16_256_n32", "bf16", (conv(256, 256, 3, pad=1),), 8, 28, 9),
+    ("bf16_stride2y_1d", "bf16", (conv(64, 128, 9, stride=2, one_d=True),), 80, 1, 200),
+    ("bf16_1d_k9", "bf16", (conv(128, 128, 9, one_d=True),), 40, 1, 130),
+    ("bf16_32ch", "bf16", (conv(32, 64, 9, stride=2, one_d=True),), 60, 1, 77),
+    ("bf16_16ch", "bf16", (conv(16, 32, 3, pad=1),), 12, 24, 6),
+    ("bf16_two_layers", "bf16", (conv(64, 64, 3, pad=1), POOL, conv(64, 128, 3, pad=1)), 16, 24, 5),
+    ("bf16_k5", "bf16", (conv(64, 32, 5, pad=2),), 14, 33, 4),
+    ("i8_64", "i8", (conv(64, 64, 3),), 12, 30, 6),
+    ("i8_32", "i8", (conv(32, 64, 3),), 12, 30, 6),
+    ("i8_128", "i8", (conv(128, 32, 3, pad=1),), 9, 20, 7),
+    ("i8_256", "i8", (conv(256, 64, 3, pad=1),), 9, 20, 7),
+    ("i8_net", "i8", (conv(32, 32, 3), POOL, conv(32, 64, 3, pad=1)), 20, 26, 9),
+]
+
+
+@pytest.mark.parametrize("name,mode,layers,H,W,S", CASES, ids=[c[0] for c in CASES])
+def test_tensor_core_layers_match_oracle(orc, name, mode, layers, H, W, S):
+    if mode == "i8":
+        layers = with_shifts(layers, 9)
+    C0 = layers[0].cin
+    x, ws, bs = rand_net(mode, layers, H, W, C0, S=S, seed=len(name))
+    want = orc.forward(mode, layers, x, ws, bs)
+    n_conv = sum(l.kind == "conv" for l in layers)
+    for chunks, rb in ((None, 0), ([1] * H, 0), ([3, 2, 5], 3), (None, 64)):
+        got, tc = _run(mode, layers, x, ws, bs, chunks=chunks, row_block=rb)
+        assert sum(t > 0 for t in tc) == n_conv, f"{name}: tensor-core path not taken: {tc}"
+        what = f"{name}/chunks={chunks and len(chunks)}/rb={rb}"
+        if mode == "i8":
+            assert_equal(got, want, what)
+        elif n_conv == 1:
+            assert_close(got, want, what)
+        else:
+            err = np.abs(got - want)
+            ok = err <= 1e-4 + 1e-3 * np.abs(want)
+            assert ok.mean() > 0.97 and err.max() < 0.05, (what, ok.mean(), err.max())
+
+
+def test_tensor_core_and_cuda_core_paths_agree_bitwise_on_int8(orc, monkeypatch):
+    layers = with_shifts((conv(64, 64, 3, pad=1), conv(64, 32, 3, stride=1)), 9)
+    x, ws, bs = rand_net("i8", layers, 18, 37, 64, S=5, seed=77)
+    got_tc, tc = _run("i8", layers, x, ws, bs)
+    assert all(t > 0 for t in tc)
+    monkeypatch.setenv("IDF_DISABLE_TC", "1")
+    got_cc, tc2 = _run("i8", layers, x, ws, bs)
+    assert not any(tc2)
+    assert np.array_equal(got_tc, got_cc)
