@@ -48,6 +48,9 @@ struct PoolArgs {
 struct TcPlan {
     int ok = 0;
     int BX = 0, BS = 0;      // a 128-row M tile = BS streams x BX consecutive x positions
+    int BXP = 0;             // positions per stream held in the shared-memory tile (BX + kx halo)
+    int shift_mode = 0;      // kx taps read one haloed tile at row offsets instead of one box per kx
+    int a_stage_bytes = 0;
     int n_xt = 0, n_mt = 0;  // x tiles per row, M tiles in all
     int Ntile = 0, n_nt = 0; // output channels per CTA, N tiles
     int KB = 0, n_kb = 0;    // input channels per K block (one swizzled shared-memory row), K blocks

@@ -133,9 +133,17 @@ struct TcArgs {
     void* out;
     unsigned int* status;
     long long out_row_stride, out_stream_stride, out_row_base;
-    long long r0, r1, o_begin, o_end, done_end;
-    int S, Wout, Cout, Kh, Kw, stride, pad, pad_x, relu, shift, ring_rows, out_elem;
-    int BX, BS, n_xt, Ntile, n_nt, KB, n_kb, swb, nslot, nstage, tmem_cols;
+    long long o_begin;           // absolute index of the first visited output row
+    int r0_positive;             // input rows arrived before this block (r0 > 0)
+    int n_rows;                  // input rows in this block
+    int n_orows;                 // visited output rows: o_begin + [0, n_orows)
+    int done_rel;                // rows with relative index < done_rel are emitted, the others go back to the ring
+    int base_ty;                 // r0 + pad - o_begin*stride: input row ri reaches relative output row
+                                 // (base_ty + ri - ky) / stride through tap ky when that is a whole number >= 0
+    int S, Wout, Cout, Kh, Kw, stride, pad_x, relu, shift, ring_rows, out_elem;
+    int BX, BXP, BS, n_xt, Ntile, n_nt, KB, n_kb, swb, nslot, nstage, tmem_cols;
+    int shift_mode;              // 1: one box per (row, K block) holds the kx halo, taps address it at row offsets
+    int a_stage_bytes;
 };
 
 template <int DT> struct Acc;
@@ -151,17 +159,19 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     __shared__ int s_issued;
+    __shared__ int s_tap_ky[32], s_tap_orel[32], s_tap_first[32];   // scratch of the MMA thread
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int taps = a.Kh * a.Kw;
     const uint32_t w_tile_bytes = (uint32_t)a.Ntile * a.swb;
-    const uint32_t a_tile_bytes = 128u * a.swb;
-    const uint32_t a_box_bytes = (uint32_t)a.BX * a.BS * a.swb;
+    const uint32_t a_stage_bytes = (uint32_t)a.a_stage_bytes;
+    const uint32_t a_box_bytes = (uint32_t)a.BXP * a.BS * a.swb;
+    const int n_xload = a.shift_mode ? 1 : a.Kw;
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sW = base;
     const uint32_t sA = (sW + (uint32_t)taps * a.n_kb * w_tile_bytes + 1023u) & ~1023u;
-    const uint32_t bars = sA + (uint32_t)a.nstage * a_tile_bytes;
+    const uint32_t bars = sA + (uint32_t)a.nstage * a_stage_bytes;
     const uint32_t bar_full = bars;
     const uint32_t bar_empty = bar_full + 8u * a.nstage;
     const uint32_t bar_w = bar_empty + 8u * a.nstage;
@@ -190,7 +200,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
     volatile int* abort_flag = &s_abort;
-    const int n_rows = (int)(a.r1 - a.r0);
+    const int n_rows = a.n_rows;
 
     if (warp == 0) {
         // ------------------------------ TMA producer -------------------------------------------
@@ -203,17 +213,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         tma_load_2d(sW + (uint32_t)(tap * a.n_kb + kb) * w_tile_bytes, &tmW, bar_w + 8u * tap,
                                     kb * a.KB, tap * a.Cout + n0);
                 }
-            int t = 0;
+            int stage = 0, t = 0;
+            uint32_t phase = 0;
             bool ok = true;
             for (int ri = 0; ri < n_rows && ok; ++ri)
-                for (int kx = 0; kx < a.Kw && ok; ++kx)
-                    for (int kb = 0; kb < a.n_kb; ++kb, ++t) {
-                        const int stage = t % a.nstage, use = t / a.nstage;
-                        if (!mbar_wait(bar_empty + 8u * stage, (uint32_t)((use & 1) ^ 1), abort_flag)) { ok = false; break; }
+                for (int xl = 0; xl < n_xload && ok; ++xl)
+                    for (int kb = 0; kb < a.n_kb; ++kb) {
+                        if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                         mbar_expect_tx(bar_full + 8u * stage, a_box_bytes);
-                        tma_load_4d(sA + (uint32_t)stage * a_tile_bytes, &tmA, bar_full + 8u * stage,
-                                    kb * a.KB, x0 - a.pad_x + kx, s0, ri);
-                        s_issued = t + 1;
+                        tma_load_4d(sA + (uint32_t)stage * a_stage_bytes, &tmA, bar_full + 8u * stage,
+                                    kb * a.KB, x0 - a.pad_x + xl, s0, ri);
+                        s_issued = ++t;
+                        if (++stage == a.nstage) { stage = 0; phase ^= 1u; }
                     }
         }
         __syncwarp();
@@ -223,52 +234,69 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t idesc = (DT == 1 ? ((1u << 4) | (1u << 7) | (1u << 10)) : ((2u << 4) | (1u << 7) | (1u << 10))) |
                                    ((uint32_t)(a.Ntile >> 3) << 17) | ((128u >> 4) << 24);
             const int ksteps = a.swb / 32;
+            const uint64_t desc_hi = make_smem_desc(0, a.swb);
+            const int n_kx = a.shift_mode ? a.Kw : 1;
             uint32_t w_seen = 0;
-            int t = 0;
+            int stage = 0;
+            uint32_t phase = 0;
             bool ok = true;
             for (int ri = 0; ri < n_rows && ok; ++ri) {
-                const long long r = a.r0 + ri;
-                for (int kx = 0; kx < a.Kw && ok; ++kx)
-                    for (int kb = 0; kb < a.n_kb && ok; ++kb, ++t) {
-                        const int stage = t % a.nstage, use = t / a.nstage;
-                        if (!mbar_wait(bar_full + 8u * stage, (uint32_t)(use & 1), abort_flag)) { ok = false; break; }
+                // output rows this input row reaches (a handful): slot, first touch, completion
+                int n_t = 0;
+                for (int ky = 0; ky < a.Kh && ok; ++ky) {
+                    const int ty = a.base_ty + ri - ky;
+                    if (ty < 0) break;
+                    const int orel = ty / a.stride;
+                    if (orel * a.stride != ty) continue;
+                    int fr = orel * a.stride - a.base_ty;
+                    if (fr < 0) fr = 0;
+                    const int first = (ri == fr);
+                    if (first && orel >= a.nslot) {      // the slot's previous row must have been read out
+                        const int u = orel / a.nslot;
+                        if (!mbar_wait(bar_free + 8u * (orel % a.nslot), (uint32_t)((u - 1) & 1), abort_flag)) { ok = false; break; }
                         tc_fence_after();
-                        const uint64_t adesc = make_smem_desc(sA + (uint32_t)stage * a_tile_bytes, a.swb);
-                        for (int ky = 0; ky < a.Kh; ++ky) {
-                            const long long ty = r + a.pad - ky;
-                            if (ty < 0 || ty % a.stride) continue;
-                            const long long o = ty / a.stride;
-                            const int rel = (int)(o - a.o_begin);
-                            const int slot = rel % a.nslot, u = rel / a.nslot;
-                            long long first_r = o * a.stride - a.pad;
-                            if (first_r < a.r0) first_r = a.r0;
-                            const bool first = (r == first_r) && kx == 0 && kb == 0;
-                            if (first && u >= 1) {
-                                if (!mbar_wait(bar_free + 8u * slot, (uint32_t)((u - 1) & 1), abort_flag)) { ok = false; break; }
-                                tc_fence_after();
+                    }
+                    s_tap_ky[n_t] = ky; s_tap_orel[n_t] = orel; s_tap_first[n_t] = first;
+                    ++n_t;
+                }
+                for (int xl = 0; xl < n_xload && ok; ++xl)
+                    for (int kb = 0; kb < a.n_kb && ok; ++kb) {
+                        if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t abase = sA + (uint32_t)stage * a_stage_bytes;
+                        for (int kxi = 0; kxi < n_kx && ok; ++kxi) {
+                            const int kx = a.shift_mode ? kxi : xl;
+                            // tap kx reads the same tile kxi rows further down: the swizzle is a function of
+                            // the absolute shared-memory address, so a start address moved by whole rows
+                            // still meets the pattern the TMA wrote (base-offset field stays 0)
+                            const uint32_t aaddr = abase + (uint32_t)kxi * a.swb;
+                            const uint64_t adesc = desc_hi | (uint64_t)((aaddr & 0x3FFFFu) >> 4);
+                            const bool first_tile = (xl == 0 && kxi == 0 && kb == 0);
+                            for (int i = 0; i < n_t; ++i) {
+                                const int tap = s_tap_ky[i] * a.Kw + kx;
+                                if (!((w_seen >> tap) & 1u)) {
+                                    if (!mbar_wait(bar_w + 8u * tap, 0, abort_flag)) { ok = false; break; }
+                                    tc_fence_after();
+                                    w_seen |= 1u << tap;
+                                }
+                                const uint32_t baddr = sW + (uint32_t)(tap * a.n_kb + kb) * w_tile_bytes;
+                                const uint64_t bdesc = desc_hi | (uint64_t)((baddr & 0x3FFFFu) >> 4);
+                                const uint32_t d = tmem_base + (uint32_t)((s_tap_orel[i] % a.nslot) * a.Ntile);
+                                const uint32_t acc0 = (first_tile && s_tap_first[i]) ? 0u : 1u;
+                                umma<DT>(d, adesc, bdesc, idesc, acc0);
+                                for (int k = 1; k < ksteps; ++k)
+                                    umma<DT>(d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, 1u);
                             }
-                            const int tap = ky * a.Kw + kx;
-                            if (!((w_seen >> tap) & 1u)) {
-                                if (!mbar_wait(bar_w + 8u * tap, 0, abort_flag)) { ok = false; break; }
-                                tc_fence_after();
-                                w_seen |= 1u << tap;
-                            }
-                            const uint64_t bdesc = make_smem_desc(sW + (uint32_t)(tap * a.n_kb + kb) * w_tile_bytes, a.swb);
-                            const uint32_t d = tmem_base + (uint32_t)(slot * a.Ntile);
-                            for (int k = 0; k < ksteps; ++k)
-                                umma<DT>(d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
-                                         (first && k == 0) ? 0u : 1u);
                         }
                         if (ok) umma_commit(bar_empty + 8u * stage);
+                        if (++stage == a.nstage) { stage = 0; phase ^= 1u; }
                     }
                 if (!ok) break;
-                // accumulators that input row r completed (or, on the block's last row, everything still open)
-                for (int ky = a.Kh - 1; ky >= 0; --ky) {
-                    const long long ty = r + a.pad - ky;
-                    if (ty < 0 || ty % a.stride) continue;
-                    const long long o = ty / a.stride;
-                    const long long fin = (o < a.done_end) ? o * a.stride - a.pad + a.Kh - 1 : a.r1 - 1;
-                    if (fin == r) umma_commit(bar_ready + 8u * (uint32_t)((o - a.o_begin) % a.nslot));
+                // accumulators that this input row completed (on the block's last row: everything still open)
+                for (int i = n_t - 1; i >= 0; --i) {
+                    const int orel = s_tap_orel[i];
+                    const int fin = (orel < a.done_rel) ? orel * a.stride - a.base_ty + a.Kh - 1 : n_rows - 1;
+                    if (fin == ri) umma_commit(bar_ready + 8u * (uint32_t)(orel % a.nslot));
                 }
             }
         }
@@ -277,23 +305,23 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ------------------------------ epilogue: row finalisation -----------------------------
         const int q = warp & 3;                          // TMEM lane quarter this warp may read
         const int m = q * 32 + lane;                     // row of the tile = TMEM lane
-        const int bs = m / a.BX, bx = m - bs * a.BX;
+        const int bs = m / a.BXP, bx = m - bs * a.BXP;
         const int s = s0 + bs, x = x0 + bx;
-        const bool valid = (m < a.BX * a.BS) && (s < a.S) && (x < a.Wout) && (bx < a.BX);
+        const bool valid = (bs < a.BS) && (bx < a.BX) && (s < a.S) && (x < a.Wout);
         const TS* bias = (const TS*)a.bias;
         TS* ring = (TS*)a.ring;
         const long long row_elems = (long long)a.Wout * a.Cout;
         bool ok = true;
-        for (long long o = a.o_begin; o < a.o_end && ok; ++o) {
-            const int rel = (int)(o - a.o_begin);
-            const int slot = rel % a.nslot, u = rel / a.nslot;
+        for (int orel = 0; orel < a.n_orows && ok; ++orel) {
+            const long long o = a.o_begin + orel;
+            const int slot = orel % a.nslot, u = orel / a.nslot;
             int got = 0;
             if (lane == 0) got = mbar_wait(bar_ready + 8u * slot, (uint32_t)(u & 1), abort_flag) ? 1 : 0;
             got = __shfl_sync(0xffffffffu, got, 0);
             if (!got) { ok = false; break; }
             tc_fence_after();
-            const bool carried_in = (a.r0 > 0) && (o * a.stride - a.pad < a.r0);
-            const bool emit = o < a.done_end;
+            const bool carried_in = a.r0_positive && (orel * a.stride - a.base_ty < 0);
+            const bool emit = orel < a.done_rel;
             TS* rp = ring + ((o % a.ring_rows) * a.S + s) * row_elems + (long long)x * a.Cout + n0;
             const long long obase = (o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride +
                                     (long long)x * a.Cout + n0;
@@ -441,6 +469,10 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     p->swb = row_bytes >= 128 ? 128 : row_bytes;
     p->KB = p->swb / esize;
     p->n_kb = Cin / p->KB;
+    // With 128-byte rows one box per (input row, K block) carries the Kw-1 halo positions of every
+    // stream in the tile and the kx taps read it at row offsets; narrower rows take one box per kx.
+    p->shift_mode = (p->swb == 128 && Kw > 1) ? 1 : 0;
+    const int halo = p->shift_mode ? Kw - 1 : 0;
     if (Wout >= 128) {
         p->n_xt = (Wout + 127) / 128;
         p->BX = (Wout + p->n_xt - 1) / p->n_xt;
@@ -448,9 +480,13 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     } else {
         p->n_xt = 1;
         p->BX = Wout;
-        p->BS = 128 / Wout;
+        p->BS = 1 + (128 - Wout) / (Wout + halo);     // (BS-1)*(BX+halo) + BX <= 128 output lanes
         if (p->BS > S) p->BS = S;
     }
+    p->BXP = p->BX + halo;
+    if (p->BXP > 256) return false;
+    const size_t a_stage = ((size_t)((128 + halo + 7) / 8 * 8) * p->swb + 1023) / 1024 * 1024;
+    p->a_stage_bytes = (int)a_stage;
     p->n_mt = p->n_xt * ((S + p->BS - 1) / p->BS);
     const int taps = Kh * Kw;
     int best = 0, best_units = -1;
@@ -458,7 +494,7 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
         if (Cout % nt) continue;
         if ((ring_rows + 1) * nt > 512) continue;
         const size_t wb = (size_t)taps * p->n_kb * nt * p->swb;
-        if (wb + 3 * 128 * (size_t)p->swb + 4096 > SMEM_LIMIT) continue;
+        if (wb + 3 * a_stage + 4096 > SMEM_LIMIT) continue;
         const int units = p->n_mt * (Cout / nt);
         if (units >= 120) { best = nt; break; }          // enough CTAs for the 148 SMs: take the widest such tile
         if (units > best_units) { best_units = units; best = nt; }
@@ -474,11 +510,11 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     p->tmem_cols = cols;
     const size_t wb = ((size_t)taps * p->n_kb * best * p->swb + 1023) / 1024 * 1024;
     const size_t room = SMEM_LIMIT - 2048 - wb - 1024;
-    int nstage = (int)(room / (128 * (size_t)p->swb));
+    int nstage = (int)(room / a_stage);
     if (nstage > 8) nstage = 8;
     if (nstage < 2) return false;
     p->nstage = nstage;
-    p->smem_bytes = 1024 + wb + (size_t)nstage * 128 * p->swb + 8 * (2 * nstage + taps + 2 * p->nslot) + 64;
+    p->smem_bytes = 1024 + wb + (size_t)nstage * a_stage + 8 * (2 * nstage + taps + 2 * p->nslot) + 64;
     p->w_bytes = (size_t)taps * Cout * Cin * esize;
     p->ok = 1;
     return true;
@@ -512,7 +548,7 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     cuuint64_t dims[4] = {(cuuint64_t)a.Cin, (cuuint64_t)a.Win, (cuuint64_t)a.S, (cuuint64_t)n_in_rows};
     cuuint64_t strides[3] = {(cuuint64_t)a.Cin * esize, (cuuint64_t)a.Win * a.Cin * esize,
                              (cuuint64_t)a.S * a.Win * a.Cin * esize};
-    cuuint32_t box[4] = {(cuuint32_t)p.KB, (cuuint32_t)p.BX, (cuuint32_t)p.BS, 1};
+    cuuint32_t box[4] = {(cuuint32_t)p.KB, (cuuint32_t)p.BXP, (cuuint32_t)p.BS, 1};
     cuuint32_t es[4] = {1, 1, 1, 1};
     CUresult r = enc(&tmA, dtype == 1 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 4,
                      const_cast<void*>(a.in), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(p.swb),
@@ -522,11 +558,13 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     TcArgs t{};
     t.bias = a.bias; t.ring = a.ring; t.out = a.out; t.status = status;
     t.out_row_stride = a.out_row_stride; t.out_stream_stride = a.out_stream_stride; t.out_row_base = a.out_row_base;
-    t.r0 = a.r0; t.r1 = a.r1; t.o_begin = a.o_begin; t.o_end = a.o_end; t.done_end = a.done_end;
-    t.S = a.S; t.Wout = a.Wout; t.Cout = a.Cout; t.Kh = a.Kh; t.Kw = a.Kw; t.stride = a.stride; t.pad = a.pad;
+    t.o_begin = a.o_begin; t.r0_positive = a.r0 > 0; t.n_rows = (int)(a.r1 - a.r0); t.n_orows = (int)(a.o_end - a.o_begin);
+    t.done_rel = (int)(a.done_end - a.o_begin); t.base_ty = (int)(a.r0 + a.pad - a.o_begin * a.stride);
+    t.S = a.S; t.Wout = a.Wout; t.Cout = a.Cout; t.Kh = a.Kh; t.Kw = a.Kw; t.stride = a.stride;
     t.pad_x = a.pad_x; t.relu = a.relu; t.shift = a.shift; t.ring_rows = a.ring_rows; t.out_elem = a.out_elem;
     t.BX = p.BX; t.BS = p.BS; t.n_xt = p.n_xt; t.Ntile = p.Ntile; t.n_nt = p.n_nt; t.KB = p.KB; t.n_kb = p.n_kb;
     t.swb = p.swb; t.nslot = p.nslot; t.nstage = p.nstage; t.tmem_cols = p.tmem_cols;
+    t.BXP = p.BXP; t.shift_mode = p.shift_mode; t.a_stage_bytes = p.a_stage_bytes;
     const unsigned grid = (unsigned)(p.n_mt * p.n_nt);
     static bool attr_set[2][64] = {};
     int dev = 0;
