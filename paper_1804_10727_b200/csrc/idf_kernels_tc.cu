@@ -99,6 +99,34 @@ __device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t b
             ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
     }
 }
+// All K steps of one shared-memory tile pair in one go (always accumulating): the descriptors move
+// 32 bytes (2 units of 16 B) per step inside the swizzled row.
+template <int DT, int KSTEPS>
+__device__ __forceinline__ void umma_tile(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc)
+{
+#define IDF_MMA_KIND(kind)                                                                              \
+    if (KSTEPS == 1)                                                                                    \
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.b32 p, 0, 0;\n\t"                                   \
+                     "tcgen05.mma.cta_group::1.kind::" kind " [%0], %1, %2, %3, p;\n\t}"                 \
+                     ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc));                     \
+    else if (KSTEPS == 2)                                                                               \
+        asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 a1, b1;\n\tsetp.eq.b32 p, 0, 0;\n\t"              \
+                     "add.s64 a1, %1, 2;\n\tadd.s64 b1, %2, 2;\n\t"                                     \
+                     "tcgen05.mma.cta_group::1.kind::" kind " [%0], %1, %2, %3, p;\n\t"                  \
+                     "tcgen05.mma.cta_group::1.kind::" kind " [%0], a1, b1, %3, p;\n\t}"                 \
+                     ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc));                     \
+    else                                                                                                \
+        asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 a1, b1, a2, b2, a3, b3;\n\tsetp.eq.b32 p, 0, 0;\n\t" \
+                     "add.s64 a1, %1, 2;\n\tadd.s64 b1, %2, 2;\n\tadd.s64 a2, %1, 4;\n\tadd.s64 b2, %2, 4;\n\t" \
+                     "add.s64 a3, %1, 6;\n\tadd.s64 b3, %2, 6;\n\t"                                     \
+                     "tcgen05.mma.cta_group::1.kind::" kind " [%0], %1, %2, %3, p;\n\t"                  \
+                     "tcgen05.mma.cta_group::1.kind::" kind " [%0], a1, b1, %3, p;\n\t"                  \
+                     "tcgen05.mma.cta_group::1.kind::" kind " [%0], a2, b2, %3, p;\n\t"                  \
+                     "tcgen05.mma.cta_group::1.kind::" kind " [%0], a3, b3, %3, p;\n\t}"                 \
+                     ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc));
+    if (DT == 1) { IDF_MMA_KIND("f16") } else { IDF_MMA_KIND("i8") }
+#undef IDF_MMA_KIND
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -113,6 +141,28 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16])
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+__device__ __forceinline__ void tmem_st16_zero(uint32_t taddr)
+{
+    const uint32_t z = 0;
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
+        ::"r"(taddr), "r"(z) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Position of tap row ky inside a stacked weight tile.  The Kh blocks of Ntile rows are ordered so
+// that the taps one input row uses (ky = ph, ph+stride, ...) sit next to each other with ky
+// descending: their output rows ascend, and so do the ring slots (TMEM columns) they accumulate
+// into, which lets one MMA of N = (taps)*Ntile serve several ring rows at once.
+__device__ __forceinline__ int weight_block(int ky, int Kh, int stride)
+{
+    const int ph = ky % stride;
+    int off = 0;
+    for (int p = 0; p < ph; ++p) off += (Kh - p + stride - 1) / stride;
+    const int cnt = (Kh - ph + stride - 1) / stride;
+    return off + cnt - 1 - ky / stride;
+}
+
 // shared-memory matrix descriptor, K-major operand in the canonical swizzled layout:
 // rows of `swb` bytes, 8-row groups `8*swb` bytes apart
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t swb)
@@ -125,6 +175,128 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t swb)
     d |= (uint64_t)1 << 46;                           // descriptor version of this architecture
     d |= layout << 61;
     return d;
+}
+
+
+// TMEM loads of W consecutive accumulator columns of this thread's lane
+template <int W>
+__device__ __forceinline__ void tmem_ld(uint32_t taddr, uint32_t (&v)[W])
+{
+    if (W == 16) {
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+              "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+            : "r"(taddr) : "memory");
+    } else {
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+            "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+              "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+              "=r"(v[16 % W]), "=r"(v[17 % W]), "=r"(v[18 % W]), "=r"(v[19 % W]), "=r"(v[20 % W]), "=r"(v[21 % W]),
+              "=r"(v[22 % W]), "=r"(v[23 % W]), "=r"(v[24 % W]), "=r"(v[25 % W]), "=r"(v[26 % W]), "=r"(v[27 % W]),
+              "=r"(v[28 % W]), "=r"(v[29 % W]), "=r"(v[30 % W]), "=r"(v[31 % W])
+            : "r"(taddr) : "memory");
+    }
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+template <int W>
+__device__ __forceinline__ void tmem_st_zero(uint32_t taddr)
+{
+    const uint32_t z = 0;
+    if (W == 16)
+        asm volatile(
+            "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
+            ::"r"(taddr), "r"(z) : "memory");
+    else
+        asm volatile(
+            "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, "
+            "%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
+            ::"r"(taddr), "r"(z) : "memory");
+}
+
+// Row finalisation of W accumulator columns of one (stream, x) position: add what earlier blocks
+// left in the ring, then either park the sum in the ring (row still open) or emit f(c + b) in the
+// layer's output type.
+template <int DT, int W, typename TS>
+__device__ __forceinline__ void finalise_chunk(const uint32_t (&v)[W], bool carried_in, bool emit, TS* rp,
+                                               const TS* bias_c, void* out, long long oidx, int out_elem, int relu, int shift)
+{
+    TS acc[W];
+#pragma unroll
+    for (int j = 0; j < W; ++j) acc[j] = DT == 1 ? (TS)__uint_as_float(v[j]) : (TS)(int)v[j];
+    if (carried_in) {
+        const int4* p4 = (const int4*)rp;
+#pragma unroll
+        for (int j4 = 0; j4 < W / 4; ++j4) {
+            const int4 t4 = p4[j4];
+            if (DT == 1) {
+                acc[4 * j4 + 0] += (TS)__int_as_float(t4.x); acc[4 * j4 + 1] += (TS)__int_as_float(t4.y);
+                acc[4 * j4 + 2] += (TS)__int_as_float(t4.z); acc[4 * j4 + 3] += (TS)__int_as_float(t4.w);
+            } else {
+                acc[4 * j4 + 0] += (TS)t4.x; acc[4 * j4 + 1] += (TS)t4.y;
+                acc[4 * j4 + 2] += (TS)t4.z; acc[4 * j4 + 3] += (TS)t4.w;
+            }
+        }
+    }
+    if (!emit) {
+        int4* p4 = (int4*)rp;
+#pragma unroll
+        for (int j4 = 0; j4 < W / 4; ++j4) {
+            int4 t4;
+            if (DT == 1) {
+                t4.x = __float_as_int((float)acc[4 * j4 + 0]); t4.y = __float_as_int((float)acc[4 * j4 + 1]);
+                t4.z = __float_as_int((float)acc[4 * j4 + 2]); t4.w = __float_as_int((float)acc[4 * j4 + 3]);
+            } else {
+                t4.x = (int)acc[4 * j4 + 0]; t4.y = (int)acc[4 * j4 + 1];
+                t4.z = (int)acc[4 * j4 + 2]; t4.w = (int)acc[4 * j4 + 3];
+            }
+            p4[j4] = t4;
+        }
+        return;
+    }
+    if (DT == 1) {
+        float f[W];
+#pragma unroll
+        for (int j = 0; j < W; ++j) {
+            float t = (float)acc[j] + (bias_c ? (float)bias_c[j] : 0.f);
+            f[j] = (relu && t < 0.f) ? 0.f : t;
+        }
+        if (out_elem == E_BF16) {
+            int4* op = (int4*)((__nv_bfloat16*)out + oidx);
+#pragma unroll
+            for (int j8 = 0; j8 < W / 8; ++j8) {
+                uint32_t pk[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    __nv_bfloat162 h2 = __floats2bfloat162_rn(f[8 * j8 + 2 * j], f[8 * j8 + 2 * j + 1]);
+                    pk[j] = *(uint32_t*)&h2;
+                }
+                op[j8] = make_int4((int)pk[0], (int)pk[1], (int)pk[2], (int)pk[3]);
+            }
+        } else {
+            float4* op = (float4*)((float*)out + oidx);
+#pragma unroll
+            for (int j4 = 0; j4 < W / 4; ++j4) op[j4] = make_float4(f[4 * j4], f[4 * j4 + 1], f[4 * j4 + 2], f[4 * j4 + 3]);
+        }
+    } else {
+        const int lo = relu ? 0 : -127;
+        int4* op = (int4*)((int8_t*)out + oidx);
+#pragma unroll
+        for (int j16 = 0; j16 < W / 16; ++j16) {
+            uint32_t pk[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                int t = (int)acc[16 * j16 + j] + (bias_c ? (int)bias_c[16 * j16 + j] : 0);
+                if (relu && t < 0) t = 0;
+                if (shift > 0) t = (t + (1 << (shift - 1))) >> shift;
+                t = t < lo ? lo : (t > 127 ? 127 : t);
+                pk[j >> 2] |= ((uint32_t)t & 0xffu) << (8 * (j & 3));
+            }
+            op[j16] = make_int4((int)pk[0], (int)pk[1], (int)pk[2], (int)pk[3]);
+        }
+    }
 }
 
 struct TcArgs {
@@ -150,7 +322,7 @@ template <int DT> struct Acc;
 template <> struct Acc<1> { typedef float S; };
 template <> struct Acc<2> { typedef int S; };
 
-template <int DT>
+template <int DT, int KSTEPS>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, const TcArgs a)
 {
@@ -159,7 +331,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     __shared__ int s_issued;
-    __shared__ int s_tap_ky[32], s_tap_orel[32], s_tap_first[32];   // scratch of the MMA thread
+    __shared__ int s_ph_cnt[32], s_ph_off[32];                        // scratch of the MMA thread
+    __shared__ uint32_t s_seg_col[16], s_seg_boff[16], s_seg_idesc[16];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int taps = a.Kh * a.Kw;
@@ -210,8 +383,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const int tap = ky * a.Kw + kx;
                     mbar_expect_tx(bar_w + 8u * tap, (uint32_t)a.n_kb * w_tile_bytes);
                     for (int kb = 0; kb < a.n_kb; ++kb)
-                        tma_load_2d(sW + (uint32_t)(tap * a.n_kb + kb) * w_tile_bytes, &tmW, bar_w + 8u * tap,
-                                    kb * a.KB, tap * a.Cout + n0);
+                        tma_load_2d(sW + (uint32_t)((kx * a.n_kb + kb) * a.Kh + weight_block(ky, a.Kh, a.stride)) * w_tile_bytes,
+                                    &tmW, bar_w + 8u * tap, kb * a.KB, tap * a.Cout + n0);
                 }
             int stage = 0, t = 0;
             uint32_t phase = 0;
@@ -230,74 +403,117 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ---------------------------------------------
+        // One thread issues every MMA, so the per-row bookkeeping is kept incremental: no division
+        // inside the row loop.  With t0 = base_ty + ri, the taps of input row ri are ky = ph, ph+s, ...
+        // (ph = t0 mod s); tap ky = ph + j*s reaches relative output row hi - j (hi = t0 div s).
         if (lane == 0) {
-            const uint32_t idesc = (DT == 1 ? ((1u << 4) | (1u << 7) | (1u << 10)) : ((2u << 4) | (1u << 7) | (1u << 10))) |
-                                   ((uint32_t)(a.Ntile >> 3) << 17) | ((128u >> 4) << 24);
-            const int ksteps = a.swb / 32;
+            const uint32_t idesc0 = (DT == 1 ? ((1u << 4) | (1u << 7) | (1u << 10)) : ((2u << 4) | (1u << 7) | (1u << 10))) |
+                                    ((128u >> 4) << 24);
             const uint64_t desc_hi = make_smem_desc(0, a.swb);
             const int n_kx = a.shift_mode ? a.Kw : 1;
-            uint32_t w_seen = 0;
+            const int max_rows = 256 / a.Ntile;          // ring rows one instruction can cover (N <= 256)
+            const int s = a.stride, nslot = a.nslot;
+            const uint32_t kx_bytes = a.shift_mode ? (uint32_t)a.swb >> 4 : 0u;
+            const uint32_t wtile_kx = ((uint32_t)(a.n_kb * a.Kh) * w_tile_bytes) >> 4;   // descriptor units per kx
+            const uint32_t wtile_kb = ((uint32_t)a.Kh * w_tile_bytes) >> 4;
+            // taps per phase and where their blocks start in the stacked weight tile (see weight_block)
+            for (int p = 0, off = 0; p < s; ++p) {
+                s_ph_cnt[p] = (a.Kh - p + s - 1) / s;
+                s_ph_off[p] = off;
+                off += s_ph_cnt[p];
+            }
+            bool ok = true;
+            for (int slot = 0; slot < nslot && ok; ++slot)       // every slot has been cleared once
+                ok = mbar_wait(bar_free + 8u * slot, 0, abort_flag);
+            tc_fence_after();
+            int t0 = a.base_ty;
+            int ph = t0 % s, hi = t0 / s;
+            int slot_hi = hi % nslot, u_hi = hi / nslot;
+            // the row completed by input row ri is (t0 - (Kh-1)) / s when that is a whole number >= 0
+            int of, phf;
+            {
+                const int tf = t0 - (a.Kh - 1);
+                if (tf >= 0) { of = tf / s; phf = tf - of * s; }
+                else { of = -((-tf + s - 1) / s); phf = tf - of * s; }
+            }
+            int slot_f = ((of % nslot) + nslot) % nslot;
+            for (int tap = 0; tap < taps && ok; ++tap)            // the CTA's weight slice has landed
+                ok = mbar_wait(bar_w + 8u * tap, 0, abort_flag);
+            tc_fence_after();
+            const uint64_t adesc_base = desc_hi | (uint64_t)((sA & 0x3FFFFu) >> 4);
+            const uint64_t bdesc_base = desc_hi | (uint64_t)((sW & 0x3FFFFu) >> 4);
             int stage = 0;
             uint32_t phase = 0;
-            bool ok = true;
             for (int ri = 0; ri < n_rows && ok; ++ri) {
-                // output rows this input row reaches (a handful): slot, first touch, completion
-                int n_t = 0;
-                for (int ky = 0; ky < a.Kh && ok; ++ky) {
-                    const int ty = a.base_ty + ri - ky;
-                    if (ty < 0) break;
-                    const int orel = ty / a.stride;
-                    if (orel * a.stride != ty) continue;
-                    int fr = orel * a.stride - a.base_ty;
-                    if (fr < 0) fr = 0;
-                    const int first = (ri == fr);
-                    if (first && orel >= a.nslot) {      // the slot's previous row must have been read out
-                        const int u = orel / a.nslot;
-                        if (!mbar_wait(bar_free + 8u * (orel % a.nslot), (uint32_t)((u - 1) & 1), abort_flag)) { ok = false; break; }
-                        tc_fence_after();
+                if (ri > 0 && ph == 0 && hi >= nslot) {  // a new row starts: its slot's previous row must be gone
+                    if (!mbar_wait(bar_free + 8u * slot_hi, (uint32_t)(u_hi & 1), abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                }
+                int n_t = s_ph_cnt[ph];
+                if (n_t > hi + 1) n_t = hi + 1;          // taps that would reach rows above the map drop out
+                int sl = slot_hi - (n_t - 1);
+                if (sl < 0) sl += nslot;
+                const uint32_t blk = (uint32_t)(s_ph_off[ph] + s_ph_cnt[ph] - n_t);
+                // Segments: runs of rows whose slots are consecutive TMEM column blocks (N <= 256 each).
+                // The first two live in registers; longer lists (tall 1D kernels) spill to shared memory.
+                int len0 = n_t;
+                if (len0 > nslot - sl) len0 = nslot - sl;
+                if (len0 > max_rows) len0 = max_rows;
+                const uint32_t d0 = tmem_base + (uint32_t)(sl * a.Ntile);
+                const uint64_t boff0 = (uint64_t)((blk * w_tile_bytes) >> 4);
+                const uint32_t id0 = idesc0 | ((uint32_t)((len0 * a.Ntile) >> 3) << 17);
+                int rem = n_t - len0;
+                sl += len0; if (sl == nslot) sl = 0;
+                int len1 = rem;
+                if (len1 > nslot - sl) len1 = nslot - sl;
+                if (len1 > max_rows) len1 = max_rows;
+                const bool have1 = len1 > 0;
+                const uint32_t d1 = tmem_base + (uint32_t)(sl * a.Ntile);
+                const uint64_t boff1 = boff0 + (uint64_t)(((uint32_t)len0 * w_tile_bytes) >> 4);
+                const uint32_t id1 = idesc0 | ((uint32_t)((len1 * a.Ntile) >> 3) << 17);
+                rem -= len1;
+                int n_seg = 0;
+                if (rem > 0) {
+                    uint32_t b = blk + (uint32_t)(len0 + len1);
+                    sl += len1; if (sl == nslot) sl = 0;
+                    while (rem > 0) {
+                        int len = rem;
+                        if (len > nslot - sl) len = nslot - sl;
+                        if (len > max_rows) len = max_rows;
+                        s_seg_col[n_seg] = (uint32_t)(sl * a.Ntile);
+                        s_seg_boff[n_seg] = (b * w_tile_bytes) >> 4;
+                        s_seg_idesc[n_seg] = idesc0 | ((uint32_t)((len * a.Ntile) >> 3) << 17);
+                        ++n_seg;
+                        rem -= len; b += (uint32_t)len; sl += len;
+                        if (sl == nslot) sl = 0;
                     }
-                    s_tap_ky[n_t] = ky; s_tap_orel[n_t] = orel; s_tap_first[n_t] = first;
-                    ++n_t;
                 }
                 for (int xl = 0; xl < n_xload && ok; ++xl)
-                    for (int kb = 0; kb < a.n_kb && ok; ++kb) {
+                    for (int kb = 0; kb < a.n_kb; ++kb) {
                         if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag)) { ok = false; break; }
                         tc_fence_after();
-                        const uint32_t abase = sA + (uint32_t)stage * a_stage_bytes;
-                        for (int kxi = 0; kxi < n_kx && ok; ++kxi) {
-                            const int kx = a.shift_mode ? kxi : xl;
-                            // tap kx reads the same tile kxi rows further down: the swizzle is a function of
-                            // the absolute shared-memory address, so a start address moved by whole rows
-                            // still meets the pattern the TMA wrote (base-offset field stays 0)
-                            const uint32_t aaddr = abase + (uint32_t)kxi * a.swb;
-                            const uint64_t adesc = desc_hi | (uint64_t)((aaddr & 0x3FFFFu) >> 4);
-                            const bool first_tile = (xl == 0 && kxi == 0 && kb == 0);
-                            for (int i = 0; i < n_t; ++i) {
-                                const int tap = s_tap_ky[i] * a.Kw + kx;
-                                if (!((w_seen >> tap) & 1u)) {
-                                    if (!mbar_wait(bar_w + 8u * tap, 0, abort_flag)) { ok = false; break; }
-                                    tc_fence_after();
-                                    w_seen |= 1u << tap;
-                                }
-                                const uint32_t baddr = sW + (uint32_t)(tap * a.n_kb + kb) * w_tile_bytes;
-                                const uint64_t bdesc = desc_hi | (uint64_t)((baddr & 0x3FFFFu) >> 4);
-                                const uint32_t d = tmem_base + (uint32_t)((s_tap_orel[i] % a.nslot) * a.Ntile);
-                                const uint32_t acc0 = (first_tile && s_tap_first[i]) ? 0u : 1u;
-                                umma<DT>(d, adesc, bdesc, idesc, acc0);
-                                for (int k = 1; k < ksteps; ++k)
-                                    umma<DT>(d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, 1u);
-                            }
+                        // tap kx reads the same tile kxi rows further down: the swizzle is a function of
+                        // the absolute shared-memory address, so a start address moved by whole rows
+                        // still meets the pattern the TMA wrote (base-offset field stays 0)
+                        uint64_t adesc = adesc_base + (uint64_t)(((uint32_t)stage * a_stage_bytes) >> 4);
+                        uint64_t bdesc = bdesc_base + (uint64_t)((a.shift_mode ? 0u : (uint32_t)xl) * wtile_kx + (uint32_t)kb * wtile_kb);
+                        for (int kxi = 0; kxi < n_kx; ++kxi, adesc += kx_bytes, bdesc += wtile_kx) {
+                            umma_tile<DT, KSTEPS>(d0, adesc, bdesc + boff0, id0);
+                            if (have1) umma_tile<DT, KSTEPS>(d1, adesc, bdesc + boff1, id1);
+                            for (int i = 0; i < n_seg; ++i)
+                                umma_tile<DT, KSTEPS>(tmem_base + s_seg_col[i], adesc, bdesc + (uint64_t)s_seg_boff[i], s_seg_idesc[i]);
                         }
-                        if (ok) umma_commit(bar_empty + 8u * stage);
+                        umma_commit(bar_empty + 8u * stage);
                         if (++stage == a.nstage) { stage = 0; phase ^= 1u; }
                     }
                 if (!ok) break;
-                // accumulators that this input row completed (on the block's last row: everything still open)
-                for (int i = n_t - 1; i >= 0; --i) {
-                    const int orel = s_tap_orel[i];
-                    const int fin = (orel < a.done_rel) ? orel * a.stride - a.base_ty + a.Kh - 1 : n_rows - 1;
-                    if (fin == ri) umma_commit(bar_ready + 8u * (uint32_t)(orel % a.nslot));
-                }
+                // the accumulator this input row completed; on the block's last row also everything still open
+                if (phf == 0 && of >= 0 && of < a.done_rel) umma_commit(bar_ready + 8u * (uint32_t)slot_f);
+                if (ri == n_rows - 1)
+                    for (int orel = a.done_rel; orel < a.n_orows; ++orel) umma_commit(bar_ready + 8u * (uint32_t)(orel % nslot));
+                ++t0;
+                if (++ph == s) { ph = 0; ++hi; if (++slot_hi == nslot) { slot_hi = 0; ++u_hi; } }
+                if (++phf == s) { phf = 0; ++of; if (++slot_f == nslot) slot_f = 0; }
             }
         }
         __syncwarp();
@@ -312,6 +528,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         TS* ring = (TS*)a.ring;
         const long long row_elems = (long long)a.Wout * a.Cout;
         bool ok = true;
+        // every ring slot in tensor memory starts at zero (all MMAs accumulate)
+        for (int slot = 0; slot < a.nslot; ++slot) {
+            for (int c = 0; c < a.Ntile; c += 16)
+                tmem_st16_zero(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(slot * a.Ntile + c));
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(bar_free + 8u * slot);
+        }
         for (int orel = 0; orel < a.n_orows && ok; ++orel) {
             const long long o = a.o_begin + orel;
             const int slot = orel % a.nslot, u = orel / a.nslot;
@@ -325,81 +549,27 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             TS* rp = ring + ((o % a.ring_rows) * a.S + s) * row_elems + (long long)x * a.Cout + n0;
             const long long obase = (o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride +
                                     (long long)x * a.Cout + n0;
-            for (int c = 0; c < a.Ntile; c += 16) {
-                uint32_t v[16];
-                tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(slot * a.Ntile + c), v);
-                if (!valid) continue;
-                TS acc[16];
-#pragma unroll
-                for (int j = 0; j < 16; ++j) acc[j] = DT == 1 ? (TS)__uint_as_float(v[j]) : (TS)(int)v[j];
-                if (carried_in) {
-                    const int4* p4 = (const int4*)(rp + c);
-#pragma unroll
-                    for (int j4 = 0; j4 < 4; ++j4) {
-                        const int4 t4 = p4[j4];
-                        if (DT == 1) {
-                            acc[4 * j4 + 0] += (TS)__int_as_float(t4.x); acc[4 * j4 + 1] += (TS)__int_as_float(t4.y);
-                            acc[4 * j4 + 2] += (TS)__int_as_float(t4.z); acc[4 * j4 + 3] += (TS)__int_as_float(t4.w);
-                        } else {
-                            acc[4 * j4 + 0] += (TS)t4.x; acc[4 * j4 + 1] += (TS)t4.y;
-                            acc[4 * j4 + 2] += (TS)t4.z; acc[4 * j4 + 3] += (TS)t4.w;
-                        }
-                    }
+            const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(slot * a.Ntile);
+            if ((a.Ntile & 31) == 0) {
+                for (int c = 0; c < a.Ntile; c += 32) {
+                    uint32_t v[32];
+                    tmem_ld<32>(trow + c, v);
+                    tmem_st_zero<32>(trow + c);           // the slot's next row starts from zero
+                    if (valid)
+                        finalise_chunk<DT, 32, TS>(v, carried_in, emit, rp + c, bias ? bias + n0 + c : nullptr, a.out,
+                                                   obase + c, a.out_elem, a.relu, a.shift);
                 }
-                if (!emit) {
-                    int4* p4 = (int4*)(rp + c);
-#pragma unroll
-                    for (int j4 = 0; j4 < 4; ++j4) {
-                        int4 t4;
-                        if (DT == 1) {
-                            t4.x = __float_as_int((float)acc[4 * j4 + 0]); t4.y = __float_as_int((float)acc[4 * j4 + 1]);
-                            t4.z = __float_as_int((float)acc[4 * j4 + 2]); t4.w = __float_as_int((float)acc[4 * j4 + 3]);
-                        } else {
-                            t4.x = (int)acc[4 * j4 + 0]; t4.y = (int)acc[4 * j4 + 1];
-                            t4.z = (int)acc[4 * j4 + 2]; t4.w = (int)acc[4 * j4 + 3];
-                        }
-                        p4[j4] = t4;
-                    }
-                    continue;
-                }
-                if (DT == 1) {
-                    float f[16];
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        float t = (float)acc[j] + (bias ? (float)bias[n0 + c + j] : 0.f);
-                        f[j] = (a.relu && t < 0.f) ? 0.f : t;
-                    }
-                    if (a.out_elem == E_BF16) {
-                        __nv_bfloat16* op = (__nv_bfloat16*)a.out + obase + c;
-                        uint32_t pk[8];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            __nv_bfloat162 h2 = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]);
-                            pk[j] = *(uint32_t*)&h2;
-                        }
-                        ((int4*)op)[0] = make_int4((int)pk[0], (int)pk[1], (int)pk[2], (int)pk[3]);
-                        ((int4*)op)[1] = make_int4((int)pk[4], (int)pk[5], (int)pk[6], (int)pk[7]);
-                    } else {
-                        float* op = (float*)a.out + obase + c;
-#pragma unroll
-                        for (int j4 = 0; j4 < 4; ++j4)
-                            ((float4*)op)[j4] = make_float4(f[4 * j4], f[4 * j4 + 1], f[4 * j4 + 2], f[4 * j4 + 3]);
-                    }
-                } else {
-                    uint32_t pk[4] = {0, 0, 0, 0};
-                    const int lo = a.relu ? 0 : -127;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        int t = (int)acc[j] + (bias ? (int)bias[n0 + c + j] : 0);
-                        if (a.relu && t < 0) t = 0;
-                        if (a.shift > 0) t = (t + (1 << (a.shift - 1))) >> a.shift;
-                        t = t < lo ? lo : (t > 127 ? 127 : t);
-                        pk[j >> 2] |= ((uint32_t)t & 0xffu) << (8 * (j & 3));
-                    }
-                    int8_t* op = (int8_t*)a.out + obase + c;
-                    *(int4*)op = make_int4((int)pk[0], (int)pk[1], (int)pk[2], (int)pk[3]);
+            } else {
+                for (int c = 0; c < a.Ntile; c += 16) {
+                    uint32_t v[16];
+                    tmem_ld<16>(trow + c, v);
+                    tmem_st_zero<16>(trow + c);
+                    if (valid)
+                        finalise_chunk<DT, 16, TS>(v, carried_in, emit, rp + c, bias ? bias + n0 + c : nullptr, a.out,
+                                                   obase + c, a.out_elem, a.relu, a.shift);
                 }
             }
+            tmem_st_wait();
             tc_fence_before();
             mbar_arrive(bar_free + 8u * slot);
         }
@@ -566,18 +736,21 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     t.swb = p.swb; t.nslot = p.nslot; t.nstage = p.nstage; t.tmem_cols = p.tmem_cols;
     t.BXP = p.BXP; t.shift_mode = p.shift_mode; t.a_stage_bytes = p.a_stage_bytes;
     const unsigned grid = (unsigned)(p.n_mt * p.n_nt);
-    static bool attr_set[2][64] = {};
+    typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const TcArgs);
+    static const KernelFn kernels[2][3] = {
+        {conv_tc_kernel<1, 1>, conv_tc_kernel<1, 2>, conv_tc_kernel<1, 4>},
+        {conv_tc_kernel<2, 1>, conv_tc_kernel<2, 2>, conv_tc_kernel<2, 4>}};
+    const int kidx = p.swb == 32 ? 0 : (p.swb == 64 ? 1 : 2);
+    const KernelFn fn = kernels[dtype - 1][kidx];
+    static bool attr_set[2][3][64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (!attr_set[dtype - 1][dev]) {
-        cudaError_t e = dtype == 1
-            ? cudaFuncSetAttribute(conv_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_LIMIT - 1024))
-            : cudaFuncSetAttribute(conv_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_LIMIT - 1024));
+    if (!attr_set[dtype - 1][kidx][dev]) {
+        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_LIMIT - 1024));
         if (e != cudaSuccess) return e;
-        attr_set[dtype - 1][dev] = true;
+        attr_set[dtype - 1][kidx][dev] = true;
     }
-    if (dtype == 1) conv_tc_kernel<1><<<grid, TC_THREADS, p.smem_bytes, st>>>(tmA, *(const CUtensorMap*)w_map, t);
-    else conv_tc_kernel<2><<<grid, TC_THREADS, p.smem_bytes, st>>>(tmA, *(const CUtensorMap*)w_map, t);
+    fn<<<grid, TC_THREADS, p.smem_bytes, st>>>(tmA, *(const CUtensorMap*)w_map, t);
     return cudaGetLastError();
 }
 
