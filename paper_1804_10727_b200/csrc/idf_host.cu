@@ -42,6 +42,10 @@ struct LayerPlan {
     size_t wtc_off = 0;
     alignas(64) unsigned char w_map[128];   // TMA descriptor of wtc in the workspace (made at open)
     long long tc_launches = 0;
+    // x-unfold in front of the tensor-core kernel (thin or x-strided layers): the Kw taps of every
+    // output position are laid side by side as kpad channels, the conv then has Kw = 1, stride_x = 1
+    int unfold = 0, kpad = 0, in_cap_rows = 0;
+    size_t unf_off = 0;
     // host copies of the packed parameters
     std::vector<unsigned char> w_packed;   // [Kh][Kw][Cin][Cout] float (float nets) or int8
     std::vector<unsigned char> b_packed;   // [Cout] float / int32 (empty = zero bias)
@@ -161,6 +165,7 @@ int advance_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, bo
         a.ring = net->ws + P.state_off;
         a.out = out_ptr;
         a.out_row_stride = row_stride; a.out_stream_stride = stream_stride; a.out_row_base = row_base;
+        a.out_rows_extent = last ? out_cap : P.out_cap_rows;
         a.event_counter = (unsigned long long*)(net->ws + net->counters_off) + i;
         a.S = (int)S; a.Win = P.in_w; a.Wout = P.out_w; a.Cin = P.in_c; a.Cout = P.out_c;
         a.Kh = P.l.kh; a.Kw = P.l.kw; a.stride = P.l.stride; a.pad = P.l.pad; a.relu = P.l.relu; a.shift = P.l.shift;
@@ -169,7 +174,18 @@ int advance_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, bo
         a.r0 = r0; a.r1 = r1; a.o_begin = o_begin; a.o_end = o_end; a.done_end = done_end;
         ce = cudaErrorNotSupported;
         if (P.tc.ok && !P.use_sparse && !flush && n_in > 0) {
-            ce = launch_conv_tc(a, P.tc, net->dtype, P.w_map, (int)n_in, (unsigned int*)(net->ws + net->status_off), net->stream);
+            ConvArgs t = a;
+            if (P.unfold && n_in <= P.in_cap_rows) {
+                ce = launch_unfold(a, (int)n_in, P.kpad, net->ws + P.unf_off, net->stream);
+                t.in = net->ws + P.unf_off;
+                t.Win = a.Wout; t.Cin = P.kpad; t.Kw = 1; t.stride_x = 1; t.pad_x = 0;
+                if (ce == cudaSuccess) {
+                    net->launches += 1;
+                    ce = launch_conv_tc(t, P.tc, net->dtype, P.w_map, (int)n_in, (unsigned int*)(net->ws + net->status_off), net->stream);
+                }
+            } else if (!P.unfold) {
+                ce = launch_conv_tc(t, P.tc, net->dtype, P.w_map, (int)n_in, (unsigned int*)(net->ws + net->status_off), net->stream);
+            }
             if (ce == cudaSuccess) P.tc_launches += 1;
         }
         if (ce == cudaErrorNotSupported)
@@ -327,16 +343,35 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
             }
             // tensor-core layout [tap][Cout][Cin], activation type, when the layer qualifies
             const char* no_tc = getenv("IDF_DISABLE_TC");
-            if (!P.use_sparse && !(no_tc && no_tc[0] == '1') &&
-                tc_make_plan(spec->dtype, net->n_streams, w, P.out_w, l.cin, l.cout, l.kh, l.kw, w == 1 ? 1 : l.stride,
-                             P.ring_rows, &P.tc)) {
-                const size_t es = spec->dtype == IDF_I8_I32 ? 1 : 2;
+            const int in_cap = i == 0 ? net->row_block : net->L[i - 1].out_cap_rows;
+            const bool tc_allowed = !P.use_sparse && !(no_tc && no_tc[0] == '1') && spec->dtype != IDF_F32;
+            const size_t es = spec->dtype == IDF_I8_I32 ? 1 : 2;
+            const int taps = l.kh * l.kw;
+            if (tc_allowed && tc_make_plan(spec->dtype, net->n_streams, w, P.out_w, l.cin, l.cout, l.kh, l.kw,
+                                           w == 1 ? 1 : l.stride, P.ring_rows, (int)elem_size(P.out_elem), &P.tc)) {
                 P.wtc_packed.resize(nw * es);
-                const int taps = l.kh * l.kw;
                 for (int co = 0; co < l.cout; ++co)
                     for (int k = 0; k < taps; ++k)
                         memcpy(P.wtc_packed.data() + (((size_t)k * l.cout + co) * l.cin) * es,
                                (const unsigned char*)weights[i] + (((size_t)co * taps + k) * l.cin) * es, (size_t)l.cin * es);
+            } else if (tc_allowed) {
+                // thin (Cin*Kw below a tensor-core K step) or x-strided layer: unfold x first
+                const size_t kbytes = (size_t)l.kw * l.cin * es;
+                const size_t padded = kbytes <= 32 ? 32 : (kbytes <= 64 ? 64 : (kbytes + 127) / 128 * 128);
+                const int kpad = (int)(padded / es);
+                if (padded <= 1024 &&
+                    tc_make_plan(spec->dtype, net->n_streams, P.out_w, P.out_w, kpad, l.cout, l.kh, 1, 1, P.ring_rows,
+                                 (int)elem_size(P.out_elem), &P.tc)) {
+                    P.unfold = 1;
+                    P.kpad = kpad;
+                    P.in_cap_rows = in_cap;
+                    P.wtc_packed.assign((size_t)l.kh * l.cout * kpad * es, 0);      // [ky][Cout][kx*Cin + ci], zero padded
+                    for (int co = 0; co < l.cout; ++co)
+                        for (int ky = 0; ky < l.kh; ++ky)
+                            memcpy(P.wtc_packed.data() + (((size_t)ky * l.cout + co) * kpad) * es,
+                                   (const unsigned char*)weights[i] + (((size_t)co * l.kh + ky) * l.kw * l.cin) * es,
+                                   (size_t)l.kw * l.cin * es);
+                }
             }
             if (biases && biases[i]) {
                 P.b_packed.resize((size_t)l.cout * 4);
@@ -375,6 +410,11 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
         P.out_off = off;
         off = align_up(off + (size_t)P.out_cap_rows * net->n_streams * P.out_w * P.out_c * elem_size(P.out_elem));
     }
+    for (auto& P : net->L)
+        if (P.unfold) {
+            P.unf_off = off;
+            off = align_up(off + (size_t)P.in_cap_rows * net->n_streams * P.out_w * P.kpad * elem_size(P.in_elem), 1024);
+        }
     net->counters_off = off;
     off = align_up(off + net->L.size() * sizeof(unsigned long long));
     net->status_off = off;
@@ -426,7 +466,8 @@ int idf_stream_open(idf_net* net, void* d_workspace, size_t workspace_bytes, voi
             e = cudaMemcpyAsync(net->ws + P.b_off, P.b_packed.data(), P.b_packed.size(), cudaMemcpyHostToDevice, net->stream);
         if (!P.wtc_packed.empty() && e == cudaSuccess) {
             e = cudaMemcpyAsync(net->ws + P.wtc_off, P.wtc_packed.data(), P.wtc_packed.size(), cudaMemcpyHostToDevice, net->stream);
-            if (tc_encode_weights(P.tc, net->dtype, net->ws + P.wtc_off, P.l.kh * P.l.kw, P.l.cin, P.l.cout, P.w_map) != 0)
+            if (tc_encode_weights(P.tc, net->dtype, net->ws + P.wtc_off, P.unfold ? P.l.kh : P.l.kh * P.l.kw,
+                                  P.unfold ? P.kpad : P.l.cin, P.l.cout, P.w_map) != 0)
                 P.tc.ok = 0;               // no TMA descriptor: this layer stays on the CUDA-core kernel
         }
         P.rows_in = 0; P.rows_done = 0; P.tc_launches = 0;

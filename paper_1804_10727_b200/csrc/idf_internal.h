@@ -26,6 +26,7 @@ struct ConvArgs {
     void* ring;            // [ring_rows][S][Wout][Cout] state words
     void* out;             // emitted rows
     long long out_row_stride, out_stream_stride, out_row_base;  // element strides; row o goes to (o - out_row_base)
+    long long out_rows_extent;   // rows the output buffer holds per stream
     unsigned long long* event_counter;  // sparse path: number of non-zero events applied
     int S, Win, Wout, Cin, Cout, Kh, Kw, stride, pad, relu, shift, ring_rows;
     int stride_x, pad_x;   // x axis: equal to stride/pad, except 1 and 0 on width-1 (1D) maps
@@ -58,14 +59,19 @@ struct TcPlan {
     int nslot = 0;           // ring rows resident in tensor memory at once (>= ring rows + 1)
     int nstage = 0;          // Δ-row tiles in flight
     int tmem_cols = 0;
+    int out_esize = 0, out_pwb = 0, out_panels = 0, out_stage_bytes = 0;   // staging of emitted rows for the TMA store
     size_t smem_bytes = 0;
     size_t w_bytes = 0;      // device weights for this path: [tap][Cout][Cin] in the activation type
 };
 bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh, int Kw, int stride_x, int ring_rows,
-                  TcPlan* p);
+                  int out_esize, TcPlan* p);
 int tc_encode_weights(const TcPlan& p, int dtype, const void* d_w, int taps, int Cin, int Cout, void* map_out);
 cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const void* w_map, int n_in_rows,
                            unsigned int* status, cudaStream_t st);
+
+// x-unfold: out[row][s][x'][kx*Cin + ci] = in[row][s][x'*stride_x - pad_x + kx][ci] (0 outside the row or
+// beyond Kw*Cin), kpad channels per position, in the activation type
+cudaError_t launch_unfold(const ConvArgs& a, int n_rows, int kpad, void* out, cudaStream_t st);
 
 // CUDA-core kernels (every type, every shape)
 cudaError_t launch_conv_simple(const ConvArgs& a, int dtype, cudaStream_t st);

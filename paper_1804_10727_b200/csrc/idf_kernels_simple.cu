@@ -280,6 +280,56 @@ cudaError_t launch_conv_sparse(const ConvArgs& a, int dtype, cudaStream_t st)
 }
 
 // ------------------------------------------------------------------------------------------------
+// x-unfold in front of the tensor-core kernel for thin or x-strided layers: every output position
+// gets its Kw*Cin input values side by side (zero padded to kpad), so that the channel contraction
+// has a K the tensor cores accept and needs no stride in x.  One thread writes 16 bytes.
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) unfold_rows_kernel(const T* __restrict__ in, T* __restrict__ out, long long n_pos,
+                                                          int Win, int Wout, int Cin, int Kw, int stride_x, int pad_x, int kpad)
+{
+    constexpr int V = 16 / (int)sizeof(T);
+    const int vecs = kpad / V;
+    const long long total = n_pos * vecs;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int v = (int)(idx % vecs);
+        const long long p = idx / vecs;              // (row, stream, x') flattened
+        const int xo = (int)(p % Wout);
+        const long long rs = p / Wout;               // (row, stream)
+        const T* row = in + rs * (long long)Win * Cin;
+        __align__(16) T vals[V];
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            const int k = v * V + j;
+            const int kx = k / Cin, ci = k - kx * Cin;
+            const int ix = xo * stride_x - pad_x + kx;
+            vals[j] = (kx < Kw && ix >= 0 && ix < Win) ? row[(long long)ix * Cin + ci] : (T)0;
+        }
+        *(int4*)(out + p * kpad + (long long)v * V) = *(const int4*)vals;
+    }
+}
+
+cudaError_t launch_unfold(const ConvArgs& a, int n_rows, int kpad, void* out, cudaStream_t st)
+{
+    const long long n_pos = (long long)n_rows * a.S * a.Wout;
+    if (n_pos == 0) return cudaSuccess;
+    const int esize = a.in_elem == E_BF16 ? 2 : 1;
+    const long long total = n_pos * (kpad * esize / 16);
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148LL * 32) blocks = 148LL * 32;
+    if (a.in_elem == E_BF16)
+        unfold_rows_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)a.in, (__nv_bfloat16*)out, n_pos,
+                                                                          a.Win, a.Wout, a.Cin, a.Kw, a.stride_x, a.pad_x, kpad);
+    else if (a.in_elem == E_I8)
+        unfold_rows_kernel<int8_t><<<(unsigned)blocks, 256, 0, st>>>((const int8_t*)a.in, (int8_t*)out, n_pos, a.Win, a.Wout,
+                                                                   a.Cin, a.Kw, a.stride_x, a.pad_x, kpad);
+    else
+        return cudaErrorInvalidValue;
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
 // Max-pool fold: the x-pair is reduced at once; the first row of a y-pair waits in a one-row
 // running maximum; the second row emits.  Width-1 maps pool over rows only.
 // ------------------------------------------------------------------------------------------------

@@ -15,7 +15,8 @@
 //     accumulator, add what the ring held from earlier blocks and the bias, apply f, round or
 //     requantise, and write the row for the next layer; rows still open at the end of the block go
 //     back to the ring in global memory.
-// Warp roles: warp 0 = TMA producer, warp 1 = TMEM owner and MMA issuer, warps 2-5 = epilogue.
+// Warp roles: warp 0 = TMA producer and row scheduler, warp 1 = TMEM owner and MMA issuer,
+// warps 2-9 = epilogue (two per TMEM lane quarter).
 // Every wait is bounded; on expiry the kernel records IDF_ERR_TIMEOUT in the status word and leaves.
 #include "idf_internal.h"
 
@@ -26,7 +27,8 @@ namespace idf {
 
 namespace {
 
-constexpr int TC_THREADS = 192;
+constexpr int TC_THREADS = 320;
+constexpr int ROWQ = 16;                     // row-schedule queue entries (more than the stages in flight)
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr size_t SMEM_LIMIT = 232448;        // 227 KB per CTA
 
@@ -216,12 +218,49 @@ __device__ __forceinline__ void tmem_st_zero(uint32_t taddr)
             ::"r"(taddr), "r"(z) : "memory");
 }
 
+
+// Where an emitted row goes first: a shared-memory tile [tile row][panel of pwb bytes], written in
+// the swizzle the output tensor map expects, from which one thread sends it out with a TMA store.
+struct StageSink {
+    uint32_t row_base;     // shared address of this thread's tile row in panel 0
+    uint32_t panel_bytes;  // bytes of one panel (128 rows * pwb)
+    uint32_t pwb_log2;     // log2(panel row bytes)
+    uint32_t phase;        // swizzle phase of this row (XORed into the 16-byte chunk index)
+};
+__device__ __forceinline__ void stage_store16(const StageSink& k, uint32_t col_byte, int4 v)
+{
+    const uint32_t panel = col_byte >> k.pwb_log2;
+    const uint32_t within = col_byte & ((1u << k.pwb_log2) - 1u);
+    const uint32_t addr = k.row_base + panel * k.panel_bytes + ((((within >> 4) ^ k.phase)) << 4);
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(tm), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void named_bar_sync(int id, int count)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+// barrier among `count` threads that also tells everyone whether all of them passed `pred`
+__device__ __forceinline__ bool named_bar_and(int id, int count, bool pred)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %3, 0;\n\t"
+        "bar.red.and.pred q, %1, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"(id), "r"(count), "r"((uint32_t)pred) : "memory");
+    return r != 0;
+}
+
 // Row finalisation of W accumulator columns of one (stream, x) position: add what earlier blocks
 // left in the ring, then either park the sum in the ring (row still open) or emit f(c + b) in the
 // layer's output type.
 template <int DT, int W, typename TS>
 __device__ __forceinline__ void finalise_chunk(const uint32_t (&v)[W], bool carried_in, bool emit, TS* rp,
-                                               const TS* bias_c, void* out, long long oidx, int out_elem, int relu, int shift)
+                                               const TS* bias_c, const StageSink& sink, uint32_t col_byte, int out_elem,
+                                               int relu, int shift)
 {
     TS acc[W];
 #pragma unroll
@@ -264,7 +303,6 @@ __device__ __forceinline__ void finalise_chunk(const uint32_t (&v)[W], bool carr
             f[j] = (relu && t < 0.f) ? 0.f : t;
         }
         if (out_elem == E_BF16) {
-            int4* op = (int4*)((__nv_bfloat16*)out + oidx);
 #pragma unroll
             for (int j8 = 0; j8 < W / 8; ++j8) {
                 uint32_t pk[4];
@@ -273,16 +311,17 @@ __device__ __forceinline__ void finalise_chunk(const uint32_t (&v)[W], bool carr
                     __nv_bfloat162 h2 = __floats2bfloat162_rn(f[8 * j8 + 2 * j], f[8 * j8 + 2 * j + 1]);
                     pk[j] = *(uint32_t*)&h2;
                 }
-                op[j8] = make_int4((int)pk[0], (int)pk[1], (int)pk[2], (int)pk[3]);
+                stage_store16(sink, col_byte + 16u * j8, make_int4((int)pk[0], (int)pk[1], (int)pk[2], (int)pk[3]));
             }
         } else {
-            float4* op = (float4*)((float*)out + oidx);
 #pragma unroll
-            for (int j4 = 0; j4 < W / 4; ++j4) op[j4] = make_float4(f[4 * j4], f[4 * j4 + 1], f[4 * j4 + 2], f[4 * j4 + 3]);
+            for (int j4 = 0; j4 < W / 4; ++j4)
+                stage_store16(sink, col_byte + 16u * j4,
+                              make_int4(__float_as_int(f[4 * j4]), __float_as_int(f[4 * j4 + 1]), __float_as_int(f[4 * j4 + 2]),
+                                        __float_as_int(f[4 * j4 + 3])));
         }
     } else {
         const int lo = relu ? 0 : -127;
-        int4* op = (int4*)((int8_t*)out + oidx);
 #pragma unroll
         for (int j16 = 0; j16 < W / 16; ++j16) {
             uint32_t pk[4] = {0, 0, 0, 0};
@@ -294,7 +333,7 @@ __device__ __forceinline__ void finalise_chunk(const uint32_t (&v)[W], bool carr
                 t = t < lo ? lo : (t > 127 ? 127 : t);
                 pk[j >> 2] |= ((uint32_t)t & 0xffu) << (8 * (j & 3));
             }
-            op[j16] = make_int4((int)pk[0], (int)pk[1], (int)pk[2], (int)pk[3]);
+            stage_store16(sink, col_byte + 16u * j16, make_int4((int)pk[0], (int)pk[1], (int)pk[2], (int)pk[3]));
         }
     }
 }
@@ -316,6 +355,9 @@ struct TcArgs {
     int BX, BXP, BS, n_xt, Ntile, n_nt, KB, n_kb, swb, nslot, nstage, tmem_cols;
     int shift_mode;              // 1: one box per (row, K block) holds the kx halo, taps address it at row offsets
     int a_stage_bytes;
+    int out_esize, out_pwb, out_panels, out_stage_bytes;   // emitted rows: staging panels of out_pwb-byte rows
+    int out_row_dim;             // position of the row coordinate in the output tensor map (2 or 3)
+    int out_row_first;           // tensor-map row index of relative output row 0
 };
 
 template <int DT> struct Acc;
@@ -324,7 +366,8 @@ template <> struct Acc<2> { typedef int S; };
 
 template <int DT, int KSTEPS>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, const TcArgs a)
+conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+               const __grid_constant__ CUtensorMap tmO, const TcArgs a)
 {
     typedef typename Acc<DT>::S TS;
     extern __shared__ unsigned char smem_raw[];
@@ -332,7 +375,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __shared__ int s_abort;
     __shared__ int s_issued;
     __shared__ int s_ph_cnt[32], s_ph_off[32];                        // scratch of the MMA thread
-    __shared__ uint32_t s_seg_col[16], s_seg_boff[16], s_seg_idesc[16];
+    __shared__ __align__(16) uint32_t s_rowq[ROWQ][16];                // per input row: what the MMA thread must do
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int taps = a.Kh * a.Kw;
@@ -344,7 +387,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sW = base;
     const uint32_t sA = (sW + (uint32_t)taps * a.n_kb * w_tile_bytes + 1023u) & ~1023u;
-    const uint32_t bars = sA + (uint32_t)a.nstage * a_stage_bytes;
+    const uint32_t sOut = sA + (uint32_t)a.nstage * a_stage_bytes;               // one staging tile per epilogue group
+    const uint32_t bars = sOut + 2u * (uint32_t)a.out_stage_bytes;
     const uint32_t bar_full = bars;
     const uint32_t bar_empty = bar_full + 8u * a.nstage;
     const uint32_t bar_w = bar_empty + 8u * a.nstage;
@@ -376,7 +420,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int n_rows = a.n_rows;
 
     if (warp == 0) {
-        // ------------------------------ TMA producer -------------------------------------------
+        // ------------------------------ TMA producer + row scheduler ---------------------------
+        // One thread issues every MMA and the tensor pipe runs only a couple of instructions ahead
+        // of it, so that thread must do as little else as possible.  This thread, which mostly waits
+        // for free stages, therefore also works out for every input row which accumulators it feeds
+        // and leaves the answer in a small queue next to the data (published by the stage's barrier).
+        // With t0 = base_ty + ri the taps of input row ri are ky = ph, ph+s, ... (ph = t0 mod s), and
+        // tap ky = ph + j*s reaches relative output row hi - j (hi = t0 div s).  All incremental.
         if (lane == 0) {
             for (int kx = 0; kx < a.Kw; ++kx)
                 for (int ky = 0; ky < a.Kh; ++ky) {
@@ -386,46 +436,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         tma_load_2d(sW + (uint32_t)((kx * a.n_kb + kb) * a.Kh + weight_block(ky, a.Kh, a.stride)) * w_tile_bytes,
                                     &tmW, bar_w + 8u * tap, kb * a.KB, tap * a.Cout + n0);
                 }
-            int stage = 0, t = 0;
-            uint32_t phase = 0;
-            bool ok = true;
-            for (int ri = 0; ri < n_rows && ok; ++ri)
-                for (int xl = 0; xl < n_xload && ok; ++xl)
-                    for (int kb = 0; kb < a.n_kb; ++kb) {
-                        if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-                        mbar_expect_tx(bar_full + 8u * stage, a_box_bytes);
-                        tma_load_4d(sA + (uint32_t)stage * a_stage_bytes, &tmA, bar_full + 8u * stage,
-                                    kb * a.KB, x0 - a.pad_x + xl, s0, ri);
-                        s_issued = ++t;
-                        if (++stage == a.nstage) { stage = 0; phase ^= 1u; }
-                    }
-        }
-        __syncwarp();
-    } else if (warp == 1) {
-        // ------------------------------ MMA issuer ---------------------------------------------
-        // One thread issues every MMA, so the per-row bookkeeping is kept incremental: no division
-        // inside the row loop.  With t0 = base_ty + ri, the taps of input row ri are ky = ph, ph+s, ...
-        // (ph = t0 mod s); tap ky = ph + j*s reaches relative output row hi - j (hi = t0 div s).
-        if (lane == 0) {
             const uint32_t idesc0 = (DT == 1 ? ((1u << 4) | (1u << 7) | (1u << 10)) : ((2u << 4) | (1u << 7) | (1u << 10))) |
                                     ((128u >> 4) << 24);
-            const uint64_t desc_hi = make_smem_desc(0, a.swb);
-            const int n_kx = a.shift_mode ? a.Kw : 1;
             const int max_rows = 256 / a.Ntile;          // ring rows one instruction can cover (N <= 256)
             const int s = a.stride, nslot = a.nslot;
-            const uint32_t kx_bytes = a.shift_mode ? (uint32_t)a.swb >> 4 : 0u;
-            const uint32_t wtile_kx = ((uint32_t)(a.n_kb * a.Kh) * w_tile_bytes) >> 4;   // descriptor units per kx
-            const uint32_t wtile_kb = ((uint32_t)a.Kh * w_tile_bytes) >> 4;
             // taps per phase and where their blocks start in the stacked weight tile (see weight_block)
             for (int p = 0, off = 0; p < s; ++p) {
                 s_ph_cnt[p] = (a.Kh - p + s - 1) / s;
                 s_ph_off[p] = off;
                 off += s_ph_cnt[p];
             }
-            bool ok = true;
-            for (int slot = 0; slot < nslot && ok; ++slot)       // every slot has been cleared once
-                ok = mbar_wait(bar_free + 8u * slot, 0, abort_flag);
-            tc_fence_after();
             int t0 = a.base_ty;
             int ph = t0 % s, hi = t0 / s;
             int slot_hi = hi % nslot, u_hi = hi / nslot;
@@ -437,6 +457,61 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 else { of = -((-tf + s - 1) / s); phf = tf - of * s; }
             }
             int slot_f = ((of % nslot) + nslot) % nslot;
+            int stage = 0, t = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int ri = 0; ri < n_rows && ok; ++ri) {
+                uint32_t* q = s_rowq[ri & (ROWQ - 1)];
+                // a new output row starts when ph == 0: its slot's previous row must have been read out
+                const bool fresh = (ri > 0 && ph == 0 && hi >= nslot);
+                q[0] = fresh ? bar_free + 8u * (uint32_t)slot_hi : 0u;
+                q[1] = (uint32_t)(u_hi & 1);
+                q[3] = (phf == 0 && of >= 0 && of < a.done_rel) ? bar_ready + 8u * (uint32_t)slot_f : 0u;
+                int n_t = s_ph_cnt[ph];
+                if (n_t > hi + 1) n_t = hi + 1;          // taps that would reach rows above the map drop out
+                int sl = slot_hi - (n_t - 1);
+                if (sl < 0) sl += nslot;
+                uint32_t blk = (uint32_t)(s_ph_off[ph] + s_ph_cnt[ph] - n_t);
+                // segments: runs of rows whose slots are consecutive TMEM column blocks (N <= 256 each)
+                int n_seg = 0;
+                for (int rem = n_t; rem > 0 && n_seg < 4; ++n_seg) {
+                    int len = rem;
+                    if (len > nslot - sl) len = nslot - sl;
+                    if (len > max_rows) len = max_rows;
+                    q[4 + 3 * n_seg] = tmem_base + (uint32_t)(sl * a.Ntile);
+                    q[5 + 3 * n_seg] = (blk * w_tile_bytes) >> 4;
+                    q[6 + 3 * n_seg] = idesc0 | ((uint32_t)((len * a.Ntile) >> 3) << 17);
+                    rem -= len; blk += (uint32_t)len; sl += len;
+                    if (sl == nslot) sl = 0;
+                }
+                q[2] = (uint32_t)n_seg;
+                for (int xl = 0; xl < n_xload && ok; ++xl)
+                    for (int kb = 0; kb < a.n_kb; ++kb) {
+                        if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                        mbar_expect_tx(bar_full + 8u * stage, a_box_bytes);
+                        tma_load_4d(sA + (uint32_t)stage * a_stage_bytes, &tmA, bar_full + 8u * stage,
+                                    kb * a.KB, x0 - a.pad_x + xl, s0, ri);
+                        s_issued = ++t;
+                        if (++stage == a.nstage) { stage = 0; phase ^= 1u; }
+                    }
+                ++t0;
+                if (++ph == s) { ph = 0; ++hi; if (++slot_hi == nslot) { slot_hi = 0; ++u_hi; } }
+                if (++phf == s) { phf = 0; ++of; if (++slot_f == nslot) slot_f = 0; }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ---------------------------------------------
+        if (lane == 0) {
+            const uint64_t desc_hi = make_smem_desc(0, a.swb);
+            const int n_kx = a.shift_mode ? a.Kw : 1;
+            const int nslot = a.nslot;
+            const uint32_t kx_bytes = a.shift_mode ? (uint32_t)a.swb >> 4 : 0u;
+            const uint32_t wtile_kx = ((uint32_t)(a.n_kb * a.Kh) * w_tile_bytes) >> 4;   // descriptor units per kx
+            const uint32_t wtile_kb = ((uint32_t)a.Kh * w_tile_bytes) >> 4;
+            bool ok = true;
+            for (int slot = 0; slot < nslot && ok; ++slot)       // every slot has been cleared once
+                ok = mbar_wait(bar_free + 8u * slot, 0, abort_flag);
             for (int tap = 0; tap < taps && ok; ++tap)            // the CTA's weight slice has landed
                 ok = mbar_wait(bar_w + 8u * tap, 0, abort_flag);
             tc_fence_after();
@@ -445,134 +520,132 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int stage = 0;
             uint32_t phase = 0;
             for (int ri = 0; ri < n_rows && ok; ++ri) {
-                if (ri > 0 && ph == 0 && hi >= nslot) {  // a new row starts: its slot's previous row must be gone
-                    if (!mbar_wait(bar_free + 8u * slot_hi, (uint32_t)(u_hi & 1), abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                }
-                int n_t = s_ph_cnt[ph];
-                if (n_t > hi + 1) n_t = hi + 1;          // taps that would reach rows above the map drop out
-                int sl = slot_hi - (n_t - 1);
-                if (sl < 0) sl += nslot;
-                const uint32_t blk = (uint32_t)(s_ph_off[ph] + s_ph_cnt[ph] - n_t);
-                // Segments: runs of rows whose slots are consecutive TMEM column blocks (N <= 256 each).
-                // The first two live in registers; longer lists (tall 1D kernels) spill to shared memory.
-                int len0 = n_t;
-                if (len0 > nslot - sl) len0 = nslot - sl;
-                if (len0 > max_rows) len0 = max_rows;
-                const uint32_t d0 = tmem_base + (uint32_t)(sl * a.Ntile);
-                const uint64_t boff0 = (uint64_t)((blk * w_tile_bytes) >> 4);
-                const uint32_t id0 = idesc0 | ((uint32_t)((len0 * a.Ntile) >> 3) << 17);
-                int rem = n_t - len0;
-                sl += len0; if (sl == nslot) sl = 0;
-                int len1 = rem;
-                if (len1 > nslot - sl) len1 = nslot - sl;
-                if (len1 > max_rows) len1 = max_rows;
-                const bool have1 = len1 > 0;
-                const uint32_t d1 = tmem_base + (uint32_t)(sl * a.Ntile);
-                const uint64_t boff1 = boff0 + (uint64_t)(((uint32_t)len0 * w_tile_bytes) >> 4);
-                const uint32_t id1 = idesc0 | ((uint32_t)((len1 * a.Ntile) >> 3) << 17);
-                rem -= len1;
-                int n_seg = 0;
-                if (rem > 0) {
-                    uint32_t b = blk + (uint32_t)(len0 + len1);
-                    sl += len1; if (sl == nslot) sl = 0;
-                    while (rem > 0) {
-                        int len = rem;
-                        if (len > nslot - sl) len = nslot - sl;
-                        if (len > max_rows) len = max_rows;
-                        s_seg_col[n_seg] = (uint32_t)(sl * a.Ntile);
-                        s_seg_boff[n_seg] = (b * w_tile_bytes) >> 4;
-                        s_seg_idesc[n_seg] = idesc0 | ((uint32_t)((len * a.Ntile) >> 3) << 17);
-                        ++n_seg;
-                        rem -= len; b += (uint32_t)len; sl += len;
-                        if (sl == nslot) sl = 0;
-                    }
-                }
+                uint4 hdr = make_uint4(0, 0, 0, 0), sa = hdr, sb = hdr, sc = hdr;
                 for (int xl = 0; xl < n_xload && ok; ++xl)
                     for (int kb = 0; kb < a.n_kb; ++kb) {
                         if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag)) { ok = false; break; }
                         tc_fence_after();
+                        if (xl == 0 && kb == 0) {        // the row's schedule came with its first tile
+                            const uint4* q = (const uint4*)s_rowq[ri & (ROWQ - 1)];
+                            hdr = q[0]; sa = q[1]; sb = q[2]; sc = q[3];
+                            if (hdr.x) {
+                                if (!mbar_wait(hdr.x, hdr.y, abort_flag)) { ok = false; break; }
+                                tc_fence_after();
+                            }
+                        }
                         // tap kx reads the same tile kxi rows further down: the swizzle is a function of
                         // the absolute shared-memory address, so a start address moved by whole rows
                         // still meets the pattern the TMA wrote (base-offset field stays 0)
                         uint64_t adesc = adesc_base + (uint64_t)(((uint32_t)stage * a_stage_bytes) >> 4);
                         uint64_t bdesc = bdesc_base + (uint64_t)((a.shift_mode ? 0u : (uint32_t)xl) * wtile_kx + (uint32_t)kb * wtile_kb);
                         for (int kxi = 0; kxi < n_kx; ++kxi, adesc += kx_bytes, bdesc += wtile_kx) {
-                            umma_tile<DT, KSTEPS>(d0, adesc, bdesc + boff0, id0);
-                            if (have1) umma_tile<DT, KSTEPS>(d1, adesc, bdesc + boff1, id1);
-                            for (int i = 0; i < n_seg; ++i)
-                                umma_tile<DT, KSTEPS>(tmem_base + s_seg_col[i], adesc, bdesc + (uint64_t)s_seg_boff[i], s_seg_idesc[i]);
+                            umma_tile<DT, KSTEPS>(sa.x, adesc, bdesc + (uint64_t)sa.y, sa.z);
+                            if (hdr.z > 1) umma_tile<DT, KSTEPS>(sa.w, adesc, bdesc + (uint64_t)sb.x, sb.y);
+                            if (hdr.z > 2) umma_tile<DT, KSTEPS>(sb.z, adesc, bdesc + (uint64_t)sb.w, sc.x);
+                            if (hdr.z > 3) umma_tile<DT, KSTEPS>(sc.y, adesc, bdesc + (uint64_t)sc.z, sc.w);
                         }
                         umma_commit(bar_empty + 8u * stage);
                         if (++stage == a.nstage) { stage = 0; phase ^= 1u; }
                     }
                 if (!ok) break;
                 // the accumulator this input row completed; on the block's last row also everything still open
-                if (phf == 0 && of >= 0 && of < a.done_rel) umma_commit(bar_ready + 8u * (uint32_t)slot_f);
+                if (hdr.w) umma_commit(hdr.w);
                 if (ri == n_rows - 1)
                     for (int orel = a.done_rel; orel < a.n_orows; ++orel) umma_commit(bar_ready + 8u * (uint32_t)(orel % nslot));
-                ++t0;
-                if (++ph == s) { ph = 0; ++hi; if (++slot_hi == nslot) { slot_hi = 0; ++u_hi; } }
-                if (++phf == s) { phf = 0; ++of; if (++slot_f == nslot) slot_f = 0; }
             }
         }
         __syncwarp();
     } else {
         // ------------------------------ epilogue: row finalisation -----------------------------
+        // Two groups of four warps (one warp per TMEM lane quarter) take the output rows in turn.
+        // An emitted row is first laid out in the group's shared-memory tile (each thread writes its
+        // own tile row, swizzled), then one thread hands the tile to a TMA store, which writes whole
+        // lines and clips whatever lies outside the map.
         const int q = warp & 3;                          // TMEM lane quarter this warp may read
+        const int grp = (warp - 2) >> 2;
+        const bool leader = (warp - 2) == grp * 4 && lane == 0;
         const int m = q * 32 + lane;                     // row of the tile = TMEM lane
         const int bs = m / a.BXP, bx = m - bs * a.BXP;
         const int s = s0 + bs, x = x0 + bx;
-        const bool valid = (bs < a.BS) && (bx < a.BX) && (s < a.S) && (x < a.Wout);
-        const TS* bias = (const TS*)a.bias;
-        TS* ring = (TS*)a.ring;
+        const bool in_tile = (bs < a.BS) && (bx < a.BX);
+        const bool valid = in_tile && (s < a.S) && (x < a.Wout);
+        const bool wide = (a.Ntile & 31) == 0;
+        const TS* bias = a.bias ? (const TS*)a.bias + n0 : nullptr;
         const long long row_elems = (long long)a.Wout * a.Cout;
+        TS* ring_pos = (TS*)a.ring + (long long)s * row_elems + (long long)x * a.Cout + n0;   // + ring slot * S * row_elems
+        const long long ring_slot_stride = (long long)a.S * row_elems;
+        const uint32_t tlane = tmem_base + ((uint32_t)(q * 32) << 16);
+        const int md = bs * a.BX + bx;                   // row of the dense output tile
+        StageSink sink;
+        sink.pwb_log2 = 31u - (uint32_t)__clz(a.out_pwb);
+        sink.panel_bytes = 128u * (uint32_t)a.out_pwb;
+        sink.row_base = sOut + (uint32_t)grp * a.out_stage_bytes + (uint32_t)md * a.out_pwb;
+        sink.phase = a.out_pwb == 128 ? (uint32_t)(md & 7) : (a.out_pwb == 64 ? (uint32_t)((md >> 1) & 3)
+                   : (a.out_pwb == 32 ? (uint32_t)((md >> 2) & 1) : 0u));
+        const uint32_t stg = sOut + (uint32_t)grp * a.out_stage_bytes;
+        const int panel_cols = a.out_pwb / a.out_esize;
         bool ok = true;
         // every ring slot in tensor memory starts at zero (all MMAs accumulate)
-        for (int slot = 0; slot < a.nslot; ++slot) {
-            for (int c = 0; c < a.Ntile; c += 16)
-                tmem_st16_zero(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(slot * a.Ntile + c));
-            tmem_st_wait();
-            tc_fence_before();
-            mbar_arrive(bar_free + 8u * slot);
-        }
-        for (int orel = 0; orel < a.n_orows && ok; ++orel) {
-            const long long o = a.o_begin + orel;
-            const int slot = orel % a.nslot, u = orel / a.nslot;
+        if (grp == 0)
+            for (int slot = 0; slot < a.nslot; ++slot) {
+                for (int c = 0; c < a.Ntile; c += 16) tmem_st16_zero(tlane + (uint32_t)(slot * a.Ntile + c));
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(bar_free + 8u * slot);
+            }
+        for (int orel = grp; orel < a.n_orows && ok; orel += 2) {
+            const int slot = orel % a.nslot;
+            const uint32_t par = (uint32_t)((orel / a.nslot) & 1);
+            const bool emit = orel < a.done_rel;
             int got = 0;
-            if (lane == 0) got = mbar_wait(bar_ready + 8u * slot, (uint32_t)(u & 1), abort_flag) ? 1 : 0;
+            if (lane == 0) got = mbar_wait(bar_ready + 8u * slot, par, abort_flag) ? 1 : 0;
             got = __shfl_sync(0xffffffffu, got, 0);
-            if (!got) { ok = false; break; }
+            // the tile must have been drained by the group's previous store before anyone writes it again;
+            // the barrier also makes the whole group leave together if any of its waits ran out
+            if (emit && leader) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            if (!named_bar_and(1 + grp, 128, got != 0)) { ok = false; break; }
             tc_fence_after();
             const bool carried_in = a.r0_positive && (orel * a.stride - a.base_ty < 0);
-            const bool emit = orel < a.done_rel;
-            TS* rp = ring + ((o % a.ring_rows) * a.S + s) * row_elems + (long long)x * a.Cout + n0;
-            const long long obase = (o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride +
-                                    (long long)x * a.Cout + n0;
-            const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(slot * a.Ntile);
-            if ((a.Ntile & 31) == 0) {
+            TS* rp = ring_pos + (long long)((a.o_begin + orel) % a.ring_rows) * ring_slot_stride;
+            const uint32_t trow = tlane + (uint32_t)(slot * a.Ntile);
+            if (wide) {
                 for (int c = 0; c < a.Ntile; c += 32) {
                     uint32_t v[32];
                     tmem_ld<32>(trow + c, v);
                     tmem_st_zero<32>(trow + c);           // the slot's next row starts from zero
-                    if (valid)
-                        finalise_chunk<DT, 32, TS>(v, carried_in, emit, rp + c, bias ? bias + n0 + c : nullptr, a.out,
-                                                   obase + c, a.out_elem, a.relu, a.shift);
+                    if (emit ? in_tile : valid)
+                        finalise_chunk<DT, 32, TS>(v, carried_in && valid, emit, rp + c, bias ? bias + c : nullptr, sink,
+                                                   (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift);
                 }
             } else {
                 for (int c = 0; c < a.Ntile; c += 16) {
                     uint32_t v[16];
                     tmem_ld<16>(trow + c, v);
                     tmem_st_zero<16>(trow + c);
-                    if (valid)
-                        finalise_chunk<DT, 16, TS>(v, carried_in, emit, rp + c, bias ? bias + n0 + c : nullptr, a.out,
-                                                   obase + c, a.out_elem, a.relu, a.shift);
+                    if (emit ? in_tile : valid)
+                        finalise_chunk<DT, 16, TS>(v, carried_in && valid, emit, rp + c, bias ? bias + c : nullptr, sink,
+                                                   (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift);
                 }
             }
             tmem_st_wait();
             tc_fence_before();
             mbar_arrive(bar_free + 8u * slot);
+            if (emit) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                named_bar_sync(1 + grp, 128);
+                if (leader) {
+                    const int orow = a.out_row_first + orel;
+                    for (int pnl = 0; pnl < a.out_panels; ++pnl) {
+                        if (a.out_row_dim == 3)
+                            tma_store_4d(&tmO, stg + (uint32_t)pnl * sink.panel_bytes, n0 + pnl * panel_cols, x0, s0, orow);
+                        else
+                            tma_store_4d(&tmO, stg + (uint32_t)pnl * sink.panel_bytes, n0 + pnl * panel_cols, x0, orow, s0);
+                    }
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+            }
         }
+        if (leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     tc_fence_before();
@@ -627,7 +700,7 @@ CUtensorMapSwizzle swizzle_of(int swb)
 }  // namespace
 
 bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh, int Kw, int stride_x, int ring_rows,
-                  TcPlan* p)
+                  int out_esize, TcPlan* p)
 {
     *p = TcPlan{};
     if (dtype != 1 && dtype != 2) return false;
@@ -663,8 +736,9 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     for (int nt = 256; nt >= 16; nt >>= 1) {
         if (Cout % nt) continue;
         if ((ring_rows + 1) * nt > 512) continue;
+        if ((ring_rows + 256 / nt - 1) / (256 / nt) + 1 > 4) continue;   // at most 4 MMA segments per input row
         const size_t wb = (size_t)taps * p->n_kb * nt * p->swb;
-        if (wb + 3 * a_stage + 4096 > SMEM_LIMIT) continue;
+        if (wb + 3 * a_stage + 2 * 128 * (size_t)nt * out_esize + 6144 > SMEM_LIMIT) continue;
         const int units = p->n_mt * (Cout / nt);
         if (units >= 120) { best = nt; break; }          // enough CTAs for the 148 SMs: take the widest such tile
         if (units > best_units) { best_units = units; best = nt; }
@@ -679,12 +753,16 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     while (cols < p->nslot * best) cols <<= 1;
     p->tmem_cols = cols;
     const size_t wb = ((size_t)taps * p->n_kb * best * p->swb + 1023) / 1024 * 1024;
-    const size_t room = SMEM_LIMIT - 2048 - wb - 1024;
+    p->out_esize = out_esize;
+    p->out_pwb = best * out_esize >= 128 ? 128 : best * out_esize;
+    p->out_panels = best * out_esize / p->out_pwb;
+    p->out_stage_bytes = p->out_panels * 128 * p->out_pwb;
+    const size_t room = SMEM_LIMIT - 4096 - wb - 1024 - 2 * (size_t)p->out_stage_bytes;   // static shared memory and alignment slack stay free
     int nstage = (int)(room / a_stage);
     if (nstage > 8) nstage = 8;
     if (nstage < 2) return false;
     p->nstage = nstage;
-    p->smem_bytes = 1024 + wb + (size_t)nstage * a_stage + 8 * (2 * nstage + taps + 2 * p->nslot) + 64;
+    p->smem_bytes = 1024 + wb + (size_t)nstage * a_stage + 2 * (size_t)p->out_stage_bytes + 8 * (2 * nstage + taps + 2 * p->nslot) + 64;
     p->w_bytes = (size_t)taps * Cout * Cin * esize;
     p->ok = 1;
     return true;
@@ -725,6 +803,28 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
                      CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorNotSupported;
 
+    // emitted rows leave through a TMA store: [channel][x][stream][row] or [channel][x][row][stream]
+    CUtensorMap tmO;
+    const int row_dim = a.out_row_stride > a.out_stream_stride ? 3 : 2;
+    {
+        const int oes = p.out_esize;
+        cuuint64_t od[4] = {(cuuint64_t)a.Cout, (cuuint64_t)a.Wout, 0, 0};
+        cuuint64_t os[3] = {(cuuint64_t)a.Cout * oes, 0, 0};
+        cuuint32_t ob[4] = {(cuuint32_t)(p.out_pwb / oes), (cuuint32_t)p.BX, 1, 1};
+        od[row_dim] = (cuuint64_t)a.out_rows_extent; od[5 - row_dim] = (cuuint64_t)a.S;
+        os[row_dim - 1] = (cuuint64_t)a.out_row_stride * oes; os[4 - row_dim] = (cuuint64_t)a.out_stream_stride * oes;
+        ob[5 - row_dim] = (cuuint32_t)p.BS;
+        if (((uintptr_t)a.out & 15) != 0 || a.out_rows_extent < 1) return cudaErrorNotSupported;
+        const CUtensorMapDataType odt = a.out_elem == E_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                      : (a.out_elem == E_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
+        const CUtensorMapSwizzle osw = p.out_pwb == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                     : (p.out_pwb == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                     : (p.out_pwb == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE));
+        CUresult ro = enc(&tmO, odt, 4, a.out, od, os, ob, es, CU_TENSOR_MAP_INTERLEAVE_NONE, osw,
+                          CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (ro != CUDA_SUCCESS) return cudaErrorNotSupported;
+    }
+
     TcArgs t{};
     t.bias = a.bias; t.ring = a.ring; t.out = a.out; t.status = status;
     t.out_row_stride = a.out_row_stride; t.out_stream_stride = a.out_stream_stride; t.out_row_base = a.out_row_base;
@@ -735,8 +835,10 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     t.BX = p.BX; t.BS = p.BS; t.n_xt = p.n_xt; t.Ntile = p.Ntile; t.n_nt = p.n_nt; t.KB = p.KB; t.n_kb = p.n_kb;
     t.swb = p.swb; t.nslot = p.nslot; t.nstage = p.nstage; t.tmem_cols = p.tmem_cols;
     t.BXP = p.BXP; t.shift_mode = p.shift_mode; t.a_stage_bytes = p.a_stage_bytes;
+    t.out_esize = p.out_esize; t.out_pwb = p.out_pwb; t.out_panels = p.out_panels; t.out_stage_bytes = p.out_stage_bytes;
+    t.out_row_dim = row_dim; t.out_row_first = (int)(a.o_begin - a.out_row_base);
     const unsigned grid = (unsigned)(p.n_mt * p.n_nt);
-    typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const TcArgs);
+    typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const TcArgs);
     static const KernelFn kernels[2][3] = {
         {conv_tc_kernel<1, 1>, conv_tc_kernel<1, 2>, conv_tc_kernel<1, 4>},
         {conv_tc_kernel<2, 1>, conv_tc_kernel<2, 2>, conv_tc_kernel<2, 4>}};
@@ -746,11 +848,11 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!attr_set[dtype - 1][kidx][dev]) {
-        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_LIMIT - 1024));
+        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_LIMIT - 2048));
         if (e != cudaSuccess) return e;
         attr_set[dtype - 1][kidx][dev] = true;
     }
-    fn<<<grid, TC_THREADS, p.smem_bytes, st>>>(tmA, *(const CUtensorMap*)w_map, t);
+    fn<<<grid, TC_THREADS, p.smem_bytes, st>>>(tmA, *(const CUtensorMap*)w_map, tmO, t);
     return cudaGetLastError();
 }
 

@@ -46,6 +46,14 @@ CASES = [
     ("bf16_16ch", "bf16", (conv(16, 32, 3, pad=1),), 12, 24, 6),
     ("bf16_two_layers", "bf16", (conv(64, 64, 3, pad=1), POOL, conv(64, 128, 3, pad=1)), 16, 24, 5),
     ("bf16_k5", "bf16", (conv(64, 32, 5, pad=2),), 14, 33, 4),
+    # thin or x-strided layers reach the tensor cores through the x-unfold pre-pass
+    ("bf16_3ch_unfold", "bf16", (conv(3, 64, 3, pad=1),), 13, 40, 5),
+    ("bf16_1ch_1d_unfold", "bf16", (conv(1, 32, 9, stride=2, one_d=True),), 70, 1, 150),
+    ("bf16_stride2_unfold", "bf16", (conv(64, 64, 3, stride=2, pad=1),), 15, 31, 4),
+    ("bf16_5ch_k5_unfold", "bf16", (conv(5, 16, 5, stride=2, pad=2),), 17, 29, 3),
+    ("i8_16ch_unfold", "i8", (conv(16, 32, 3),), 12, 26, 7),
+    ("i8_stride2_unfold", "i8", (conv(32, 64, 3, stride=2),), 21, 33, 5),
+    ("i8_2ch_unfold", "i8", (conv(2, 32, 3, path=1),), 12, 30, 6),     # forced dense: AUTO would scatter events
     ("i8_64", "i8", (conv(64, 64, 3),), 12, 30, 6),
     ("i8_32", "i8", (conv(32, 64, 3),), 12, 30, 6),
     ("i8_128", "i8", (conv(128, 32, 3, pad=1),), 9, 20, 7),
