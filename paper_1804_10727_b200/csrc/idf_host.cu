@@ -108,7 +108,7 @@ long long conv_rows_at_flush(const idf_layer& l, long long rows_in)
 // Returns the number of rows it emits; enqueues nothing when `dry` is set.
 int advance_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, bool flush, bool dry,
                   void* final_out, long long out_cap, long long* n_out_p, long long* rows_in_sim,
-                  long long* rows_done_sim)
+                  long long* rows_done_sim, long long out_slot_offset = 0)
 {
     LayerPlan& P = net->L[i];
     const bool last = (i + 1 == net->L.size());
@@ -130,7 +130,7 @@ int advance_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, bo
     rows_done_sim[i] = done_end;
     if (last && done_end > out_cap)
         return fail(IDF_ERR_CAPACITY, "output row %lld does not fit out_capacity_rows=%lld", done_end - 1, out_cap);
-    if (!last && n_out > P.out_cap_rows)
+    if (!last && n_out + out_slot_offset > P.out_cap_rows)
         return fail(IDF_ERR_CAPACITY, "internal: layer %zu emits %lld rows into a %d-row buffer", i, n_out, P.out_cap_rows);
     if (dry || (n_in == 0 && n_out == 0)) return IDF_OK;
 
@@ -146,7 +146,7 @@ int advance_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, bo
         out_ptr = net->ws + P.out_off;
         stream_stride = (long long)P.out_w * P.out_c;
         row_stride = S * stream_stride;
-        row_base = o_begin;
+        row_base = o_begin - out_slot_offset;      // rows of one block are appended slot after slot
     }
     cudaError_t ce;
     cudaEvent_t ev_a = nullptr, ev_b = nullptr;
@@ -217,7 +217,18 @@ int run_block(idf_net* net, const void* d_seg, long long n_seg, bool flush, bool
     long long n_in = n_seg;
     for (size_t i = 0; i < net->L.size(); ++i) {
         long long n_out = 0;
-        int rc = advance_layer(net, i, in_ptr, n_in, flush, dry, d_out, out_cap, &n_out, rows_in_sim, rows_done_sim);
+        int rc;
+        if (flush && n_in > 0) {
+            // End of input with rows still arriving from below: first an ordinary update with those
+            // rows (so they take the layer's fast path), then the padding-only completion of the rest.
+            long long n1 = 0, n2 = 0;
+            rc = advance_layer(net, i, in_ptr, n_in, false, dry, d_out, out_cap, &n1, rows_in_sim, rows_done_sim);
+            if (rc == IDF_OK)
+                rc = advance_layer(net, i, nullptr, 0, true, dry, d_out, out_cap, &n2, rows_in_sim, rows_done_sim, n1);
+            n_out = n1 + n2;
+        } else {
+            rc = advance_layer(net, i, in_ptr, n_in, flush, dry, d_out, out_cap, &n_out, rows_in_sim, rows_done_sim);
+        }
         if (rc != IDF_OK) return rc;
         if (i + 1 == net->L.size()) *emitted += n_out;
         if (n_out == 0 && !flush) break;    // nothing travels further up in this block

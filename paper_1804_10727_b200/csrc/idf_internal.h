@@ -59,6 +59,7 @@ struct TcPlan {
     int nslot = 0;           // ring rows resident in tensor memory at once (>= ring rows + 1)
     int nstage = 0;          // Δ-row tiles in flight
     int tmem_cols = 0;
+    int out_groups = 0;
     int out_esize = 0, out_pwb = 0, out_panels = 0, out_stage_bytes = 0;   // staging of emitted rows for the TMA store
     size_t smem_bytes = 0;
     size_t w_bytes = 0;      // device weights for this path: [tap][Cout][Cin] in the activation type

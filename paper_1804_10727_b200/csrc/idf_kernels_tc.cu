@@ -356,6 +356,7 @@ struct TcArgs {
     int shift_mode;              // 1: one box per (row, K block) holds the kx halo, taps address it at row offsets
     int a_stage_bytes;
     int out_esize, out_pwb, out_panels, out_stage_bytes;   // emitted rows: staging panels of out_pwb-byte rows
+    int out_groups;              // epilogue groups at work (1 or 2), each with its own staging tile
     int out_row_dim;             // position of the row coordinate in the output tensor map (2 or 3)
     int out_row_first;           // tensor-map row index of relative output row 0
 };
@@ -388,7 +389,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t sW = base;
     const uint32_t sA = (sW + (uint32_t)taps * a.n_kb * w_tile_bytes + 1023u) & ~1023u;
     const uint32_t sOut = sA + (uint32_t)a.nstage * a_stage_bytes;               // one staging tile per epilogue group
-    const uint32_t bars = sOut + 2u * (uint32_t)a.out_stage_bytes;
+    const uint32_t bars = sOut + (uint32_t)a.out_groups * (uint32_t)a.out_stage_bytes;
     const uint32_t bar_full = bars;
     const uint32_t bar_empty = bar_full + 8u * a.nstage;
     const uint32_t bar_w = bar_empty + 8u * a.nstage;
@@ -593,7 +594,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 tc_fence_before();
                 mbar_arrive(bar_free + 8u * slot);
             }
-        for (int orel = grp; orel < a.n_orows && ok; orel += 2) {
+        for (int orel = grp; orel < a.n_orows && ok && grp < a.out_groups; orel += a.out_groups) {
             const int slot = orel % a.nslot;
             const uint32_t par = (uint32_t)((orel / a.nslot) & 1);
             const bool emit = orel < a.done_rel;
@@ -738,7 +739,7 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
         if ((ring_rows + 1) * nt > 512) continue;
         if ((ring_rows + 256 / nt - 1) / (256 / nt) + 1 > 4) continue;   // at most 4 MMA segments per input row
         const size_t wb = (size_t)taps * p->n_kb * nt * p->swb;
-        if (wb + 3 * a_stage + 2 * 128 * (size_t)nt * out_esize + 6144 > SMEM_LIMIT) continue;
+        if (wb + 3 * a_stage + 128 * (size_t)nt * out_esize + 6144 > SMEM_LIMIT) continue;   // one staging tile at least
         const int units = p->n_mt * (Cout / nt);
         if (units >= 120) { best = nt; break; }          // enough CTAs for the 148 SMs: take the widest such tile
         if (units > best_units) { best_units = units; best = nt; }
@@ -757,12 +758,14 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     p->out_pwb = best * out_esize >= 128 ? 128 : best * out_esize;
     p->out_panels = best * out_esize / p->out_pwb;
     p->out_stage_bytes = p->out_panels * 128 * p->out_pwb;
-    const size_t room = SMEM_LIMIT - 4096 - wb - 1024 - 2 * (size_t)p->out_stage_bytes;   // static shared memory and alignment slack stay free
+    // two epilogue groups (two staging tiles) when that still leaves three Δ-row stages, else one
+    p->out_groups = (wb + 3 * a_stage + 2 * (size_t)p->out_stage_bytes + 6144 <= SMEM_LIMIT) ? 2 : 1;
+    const size_t room = SMEM_LIMIT - 4096 - wb - 1024 - (size_t)p->out_groups * p->out_stage_bytes;   // static shared memory and alignment slack stay free
     int nstage = (int)(room / a_stage);
     if (nstage > 8) nstage = 8;
     if (nstage < 2) return false;
     p->nstage = nstage;
-    p->smem_bytes = 1024 + wb + (size_t)nstage * a_stage + 2 * (size_t)p->out_stage_bytes + 8 * (2 * nstage + taps + 2 * p->nslot) + 64;
+    p->smem_bytes = 1024 + wb + (size_t)nstage * a_stage + (size_t)p->out_groups * p->out_stage_bytes + 8 * (2 * nstage + taps + 2 * p->nslot) + 64;
     p->w_bytes = (size_t)taps * Cout * Cin * esize;
     p->ok = 1;
     return true;
@@ -835,7 +838,7 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     t.BX = p.BX; t.BS = p.BS; t.n_xt = p.n_xt; t.Ntile = p.Ntile; t.n_nt = p.n_nt; t.KB = p.KB; t.n_kb = p.n_kb;
     t.swb = p.swb; t.nslot = p.nslot; t.nstage = p.nstage; t.tmem_cols = p.tmem_cols;
     t.BXP = p.BXP; t.shift_mode = p.shift_mode; t.a_stage_bytes = p.a_stage_bytes;
-    t.out_esize = p.out_esize; t.out_pwb = p.out_pwb; t.out_panels = p.out_panels; t.out_stage_bytes = p.out_stage_bytes;
+    t.out_esize = p.out_esize; t.out_pwb = p.out_pwb; t.out_panels = p.out_panels; t.out_stage_bytes = p.out_stage_bytes; t.out_groups = p.out_groups;
     t.out_row_dim = row_dim; t.out_row_first = (int)(a.o_begin - a.out_row_base);
     const unsigned grid = (unsigned)(p.n_mt * p.n_nt);
     typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const TcArgs);
