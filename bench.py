@@ -282,10 +282,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="vgg2d", choices=list(workloads.NAMES))
     ap.add_argument("--streams", type=int, default=None, help="streams per GPU (default: the workload's)")
+    ap.add_argument("--rows", type=int, default=None, help="segments per stream (default: the workload's; shorter runs are for profiling)")
     ap.add_argument("--row-block", type=int, default=0)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     args = ap.parse_args()
-    w = workloads.get(args.workload, n_streams=args.streams)
+    w = workloads.get(args.workload, n_streams=args.streams, H=args.rows)
     if args.impl == "reference":
         run_reference(args, w)
     else:

@@ -376,11 +376,68 @@ __global__ void __launch_bounds__(256) pool_rows_kernel(PoolArgs a)
     }
 }
 
+// 16 bytes of channels per thread (the layout is channels-innermost, so a position's channels are
+// contiguous): the same fold, vectorised.  Used when C * sizeof(T) is a multiple of 16.
+template <typename T>
+__global__ void __launch_bounds__(256) pool_rows_vec_kernel(PoolArgs a)
+{
+    constexpr int V = 16 / (int)sizeof(T);
+    const T* __restrict__ in = (const T*)a.in;
+    T* state = (T*)a.state;
+    T* out = (T*)a.out;
+    const int px = (a.Win == 1) ? 1 : 2;
+    const int cv = a.C / V;
+    const long long n_o = a.o_end - a.o_begin;
+    const long long total = n_o * a.S * a.Wout * cv;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(idx % cv) * V;
+        long long t = idx / cv;
+        const int ox = (int)(t % a.Wout);
+        t /= a.Wout;
+        const int s = (int)(t % a.S);
+        const long long o = a.o_begin + t / a.S;
+        const long long sidx = ((long long)s * a.Wout + ox) * a.C + c;
+        __align__(16) T m[V];
+        bool have = false;
+        if (2 * o < a.r0) { *(int4*)m = *(const int4*)(state + sidx); have = true; }
+        for (int dy = 0; dy < 2; ++dy) {
+            const long long r = 2 * o + dy;
+            if (r < a.r0 || r >= a.r1) continue;
+            const T* row = in + ((r - a.r0) * a.S + s) * (long long)a.Win * a.C;
+            for (int dx = 0; dx < px; ++dx) {
+                __align__(16) T v[V];
+                *(int4*)v = *(const int4*)(row + (long long)(px * ox + dx) * a.C + c);
+#pragma unroll
+                for (int j = 0; j < V; ++j) m[j] = have ? max_of(m[j], v[j]) : v[j];
+                have = true;
+            }
+        }
+        if (o < a.done_end)
+            *(int4*)(out + (o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride +
+                     (long long)ox * a.C + c) = *(const int4*)m;
+        else
+            *(int4*)(state + sidx) = *(const int4*)m;
+    }
+}
+
 template <typename T>
 static cudaError_t launch_pool_t(const PoolArgs& a, cudaStream_t st)
 {
     const long long total = (long long)a.S * a.Wout * a.C;
     if (total == 0 || a.o_end <= a.o_begin) return cudaSuccess;
+    constexpr int V = 16 / (int)sizeof(T);
+    const bool aligned = (a.C % V == 0) && (((uintptr_t)a.in | (uintptr_t)a.out | (uintptr_t)a.state) & 15) == 0 &&
+                         ((a.out_row_stride | a.out_stream_stride) % V == 0);
+    // each output row has its own thread in the vector kernel, so it needs every row pair to be
+    // independent: true as long as at most one visited row is carried in or out (always the case)
+    if (aligned) {
+        const long long tv = (a.o_end - a.o_begin) * a.S * a.Wout * (a.C / V);
+        long long blocks = (tv + 255) / 256;
+        if (blocks > 148LL * 64) blocks = 148LL * 64;
+        pool_rows_vec_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(a);
+        return cudaGetLastError();
+    }
     long long blocks = (total + 255) / 256;
     if (blocks > 148LL * 32) blocks = 148LL * 32;
     pool_rows_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(a);

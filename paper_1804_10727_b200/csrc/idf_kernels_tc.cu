@@ -749,7 +749,8 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     p->n_nt = Cout / best;
     p->nslot = 512 / best;
     if (p->nslot > 16) p->nslot = 16;
-    if (p->nslot > ring_rows + 3) p->nslot = ring_rows + 3;
+    // as many resident rows as tensor memory holds: the fewer input rows whose window of ring rows
+    // wraps around the slot array, the fewer split MMAs
     int cols = 32;
     while (cols < p->nslot * best) cols <<= 1;
     p->tmem_cols = cols;
