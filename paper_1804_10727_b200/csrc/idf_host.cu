@@ -56,6 +56,8 @@ struct LayerPlan {
     int out_cap_rows = 0;                  // capacity of the buffer this layer emits into
     // progress (identical for all streams)
     long long rows_in = 0, rows_done = 0;
+    long long pending = 0;                 // rows waiting in this layer's input buffer
+    int fire_rows = 0;                     // the layer runs once this many rows wait (or when a push ends)
 };
 
 enum Phase { CREATED = 0, OPEN = 1, FINISHED = 2 };
@@ -104,15 +106,25 @@ long long conv_rows_at_flush(const idf_layer& l, long long rows_in)
     return q < 0 ? 0 : q / l.stride + 1;
 }
 
-// One layer takes n_in new input rows (and, when flushing, learns that the input has ended).
-// Returns the number of rows it emits; enqueues nothing when `dry` is set.
-int advance_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, bool flush, bool dry,
-                  void* final_out, long long out_cap, long long* n_out_p, long long* rows_in_sim,
-                  long long* rows_done_sim, long long out_slot_offset = 0)
+long long layer_done_after(const LayerPlan& P, long long rows_in)
+{
+    return P.l.kind == IDF_CONV ? conv_done_after(P.l, rows_in) : rows_in / 2;
+}
+long long layer_rows_at_flush(const LayerPlan& P, long long rows_in)
+{
+    return P.l.kind == IDF_CONV ? conv_rows_at_flush(P.l, rows_in) : rows_in / 2;
+}
+
+// Enqueue one layer on n_in input rows found at in_ptr (slots 0..n_in-1).  With `flush` (n_in == 0)
+// the layer learns that its input has ended and completes the rows that wait only for bottom padding.
+// Rows it emits go to the next layer's buffer starting at slot `out_slot` (or to the caller's output
+// at their absolute row index).  Updates the layer's row counters; *n_out_p = rows emitted.
+int launch_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, bool flush, void* final_out,
+                 long long out_cap, long long out_slot, long long* n_out_p)
 {
     LayerPlan& P = net->L[i];
     const bool last = (i + 1 == net->L.size());
-    const long long r0 = rows_in_sim[i], r1 = r0 + n_in;
+    const long long r0 = P.rows_in, r1 = r0 + n_in;
     long long done_end, o_end;
     if (P.l.kind == IDF_CONV) {
         done_end = flush ? conv_rows_at_flush(P.l, r1) : conv_done_after(P.l, r1);
@@ -122,17 +134,18 @@ int advance_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, bo
         done_end = r1 / 2;
         o_end = (r1 + 1) / 2;
     }
-    const long long o_begin = rows_done_sim[i];
+    const long long o_begin = P.rows_done;
     if (done_end < o_begin) done_end = o_begin;
     const long long n_out = done_end - o_begin;
     *n_out_p = n_out;
-    rows_in_sim[i] = r1;
-    rows_done_sim[i] = done_end;
     if (last && done_end > out_cap)
         return fail(IDF_ERR_CAPACITY, "output row %lld does not fit out_capacity_rows=%lld", done_end - 1, out_cap);
-    if (!last && n_out + out_slot_offset > P.out_cap_rows)
-        return fail(IDF_ERR_CAPACITY, "internal: layer %zu emits %lld rows into a %d-row buffer", i, n_out, P.out_cap_rows);
-    if (dry || (n_in == 0 && n_out == 0)) return IDF_OK;
+    if (!last && n_out + out_slot > P.out_cap_rows)
+        return fail(IDF_ERR_CAPACITY, "internal: layer %zu emits %lld rows at slot %lld of a %d-row buffer", i, n_out,
+                    out_slot, P.out_cap_rows);
+    P.rows_in = r1;
+    P.rows_done = done_end;
+    if (n_in == 0 && n_out == 0) return IDF_OK;
 
     const long long S = net->n_streams;
     void* out_ptr;
@@ -146,7 +159,7 @@ int advance_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, bo
         out_ptr = net->ws + P.out_off;
         stream_stride = (long long)P.out_w * P.out_c;
         row_stride = S * stream_stride;
-        row_base = o_begin - out_slot_offset;      // rows of one block are appended slot after slot
+        row_base = o_begin - out_slot;             // emitted rows are appended slot after slot
     }
     cudaError_t ce;
     cudaEvent_t ev_a = nullptr, ev_b = nullptr;
@@ -209,31 +222,44 @@ int advance_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, bo
     return IDF_OK;
 }
 
-// Depth-first pass of one block of segments (or of the end-of-input flush) through all layers.
-int run_block(idf_net* net, const void* d_seg, long long n_seg, bool flush, bool dry, void* d_out,
-              long long out_cap, long long* rows_in_sim, long long* rows_done_sim, long long* emitted)
+// Depth-first schedule.  Rows a layer emits wait in the next layer's buffer; that layer runs ("fires")
+// once a block's worth of rows (fire_rows) has gathered, when a push ends, or when its buffer could not
+// take what is about to arrive.  So a pooled, narrower layer runs less often on as many rows, and a
+// push of one segment still walks every layer it can reach before the call returns.
+int fire(idf_net* net, size_t i, const void* in_ptr, long long n_in, bool flush, void* d_out, long long out_cap,
+         long long* emitted);
+
+int ensure_space(idf_net* net, size_t m, long long need, void* d_out, long long out_cap, long long* emitted)
 {
-    const void* in_ptr = d_seg;
-    long long n_in = n_seg;
-    for (size_t i = 0; i < net->L.size(); ++i) {
-        long long n_out = 0;
-        int rc;
-        if (flush && n_in > 0) {
-            // End of input with rows still arriving from below: first an ordinary update with those
-            // rows (so they take the layer's fast path), then the padding-only completion of the rest.
-            long long n1 = 0, n2 = 0;
-            rc = advance_layer(net, i, in_ptr, n_in, false, dry, d_out, out_cap, &n1, rows_in_sim, rows_done_sim);
-            if (rc == IDF_OK)
-                rc = advance_layer(net, i, nullptr, 0, true, dry, d_out, out_cap, &n2, rows_in_sim, rows_done_sim, n1);
-            n_out = n1 + n2;
-        } else {
-            rc = advance_layer(net, i, in_ptr, n_in, flush, dry, d_out, out_cap, &n_out, rows_in_sim, rows_done_sim);
-        }
+    LayerPlan& Q = net->L[m];
+    if (Q.pending + need <= net->L[m - 1].out_cap_rows) return IDF_OK;
+    return fire(net, m, net->ws + net->L[m - 1].out_off, Q.pending, false, d_out, out_cap, emitted);
+}
+
+int fire(idf_net* net, size_t i, const void* in_ptr, long long n_in, bool flush, void* d_out, long long out_cap,
+         long long* emitted)
+{
+    LayerPlan& P = net->L[i];
+    const bool last = (i + 1 == net->L.size());
+    const long long r1 = P.rows_in + n_in;
+    const long long n1 = std::max(0LL, layer_done_after(P, r1) - P.rows_done);
+    const long long n2 = flush ? std::max(0LL, layer_rows_at_flush(P, r1) - std::max(P.rows_done, layer_done_after(P, r1))) : 0;
+    if (!last) {
+        int rc = ensure_space(net, i + 1, n1 + n2, d_out, out_cap, emitted);
         if (rc != IDF_OK) return rc;
-        if (i + 1 == net->L.size()) *emitted += n_out;
-        if (n_out == 0 && !flush) break;    // nothing travels further up in this block
-        in_ptr = net->ws + net->L[i].out_off;
-        n_in = n_out;
+    }
+    if (i > 0) P.pending = 0;
+    long long got = 0;
+    if (n_in > 0) {
+        int rc = launch_layer(net, i, in_ptr, n_in, false, d_out, out_cap, last ? 0 : net->L[i + 1].pending, &got);
+        if (rc != IDF_OK) return rc;
+        if (last) *emitted += got; else net->L[i + 1].pending += got;
+    }
+    if (flush) {
+        // the arriving rows took the ordinary path above; what is left is the padding-only completion
+        int rc = launch_layer(net, i, nullptr, 0, true, d_out, out_cap, last ? 0 : net->L[i + 1].pending, &got);
+        if (rc != IDF_OK) return rc;
+        if (last) *emitted += got; else net->L[i + 1].pending += got;
     }
     return IDF_OK;
 }
@@ -242,28 +268,30 @@ int run_segments(idf_net* net, const void* d_segments, long long n_seg, bool flu
                  long long out_cap, long long* emitted)
 {
     const size_t nl = net->L.size();
-    std::vector<long long> rin(nl), rdone(nl);
+    // capacity of the caller's output first: the rows complete after this call do not depend on the schedule
+    {
+        long long r = net->L[0].rows_in + n_seg;
+        for (size_t i = 0; i < nl; ++i) r = flush ? layer_rows_at_flush(net->L[i], r) : layer_done_after(net->L[i], r);
+        if (r > out_cap)
+            return fail(IDF_ERR_CAPACITY, "output row %lld does not fit out_capacity_rows=%lld", r - 1, out_cap);
+    }
     const size_t seg_bytes = (size_t)net->n_streams * net->in_w * net->in_c * elem_size(net->L[0].in_elem);
-    for (int pass = 0; pass < 2; ++pass) {       // pass 0: dry run (capacity check), pass 1: enqueue
-        const bool dry = (pass == 0);
-        for (size_t i = 0; i < nl; ++i) { rin[i] = net->L[i].rows_in; rdone[i] = net->L[i].rows_done; }
-        long long em = 0;
-        for (long long s0 = 0; s0 < n_seg; s0 += net->row_block) {
-            const long long n = std::min<long long>(net->row_block, n_seg - s0);
-            int rc = run_block(net, (const unsigned char*)d_segments + (size_t)s0 * seg_bytes, n, false, dry, d_out,
-                               out_cap, rin.data(), rdone.data(), &em);
-            if (rc != IDF_OK) return rc;
-        }
-        if (flush) {
-            int rc = run_block(net, nullptr, 0, true, dry, d_out, out_cap, rin.data(), rdone.data(), &em);
-            if (rc != IDF_OK) return rc;
-        }
-        if (!dry) {
-            for (size_t i = 0; i < nl; ++i) { net->L[i].rows_in = rin[i]; net->L[i].rows_done = rdone[i]; }
-            *emitted = em;
+    int rc = IDF_OK;
+    for (long long s0 = 0; s0 < n_seg && rc == IDF_OK; s0 += net->row_block) {
+        const long long n = std::min<long long>(net->row_block, n_seg - s0);
+        rc = fire(net, 0, (const unsigned char*)d_segments + (size_t)s0 * seg_bytes, n, false, d_out, out_cap, emitted);
+        const bool last_block = s0 + n >= n_seg;
+        for (size_t i = 1; i < nl && rc == IDF_OK; ++i) {
+            LayerPlan& P = net->L[i];
+            if (P.pending > 0 && (P.pending >= P.fire_rows || last_block))
+                rc = fire(net, i, net->ws + net->L[i - 1].out_off, P.pending, false, d_out, out_cap, emitted);
         }
     }
-    return IDF_OK;
+    if (flush)
+        for (size_t i = 0; i < nl && rc == IDF_OK; ++i)
+            rc = fire(net, i, i ? net->ws + net->L[i - 1].out_off : nullptr, i ? net->L[i].pending : 0, true, d_out, out_cap, emitted);
+    if (rc != IDF_OK) net->phase = FINISHED;      // counters and buffers are no longer consistent: reopen to go on
+    return rc;
 }
 
 }  // namespace
@@ -329,7 +357,7 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
             P.use_sparse = l.path == IDF_PATH_SPARSE ||
                            (l.path == IDF_PATH_AUTO && i == 0 && spec->dtype == IDF_I8_I32 && l.cin <= 4);
             P.state_bytes_stream = (size_t)P.ring_rows * P.out_w * P.out_c * state_word;
-            cap = (cap + l.stride - 1) / l.stride + 1 + P.ring_rows;
+            cap = std::max(2 * net->row_block + 8, (cap + l.stride - 1) / l.stride + 1 + P.ring_rows);
             // parameters -> [Kh][Kw][Cin][Cout]
             const size_t nw = (size_t)l.cout * l.kh * l.kw * l.cin;
             if (spec->dtype == IDF_I8_I32) {
@@ -396,12 +424,13 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
             P.out_elem = elem;
             P.use_sparse = 0;
             P.state_bytes_stream = (size_t)P.out_w * P.out_c * elem_size(elem);
-            cap = cap / 2 + 1;
+            cap = std::max(2 * net->row_block + 8, cap / 2 + 1);
         } else {
             delete net;
             return fail(IDF_ERR_SPEC, "layer %d: unknown kind %d", i, l.kind);
         }
-        P.out_cap_rows = cap;
+        P.out_cap_rows = cap;      // rows the buffer behind this layer holds: a block in waiting plus one arrival
+        P.fire_rows = net->row_block;
         P.state_bytes_all = P.state_bytes_stream * (size_t)net->n_streams;
         net->state_bytes_stream += P.state_bytes_stream;
         w = P.out_w; c = P.out_c; elem = P.out_elem;
@@ -481,7 +510,7 @@ int idf_stream_open(idf_net* net, void* d_workspace, size_t workspace_bytes, voi
                                   P.unfold ? P.kpad : P.l.cin, P.l.cout, P.w_map) != 0)
                 P.tc.ok = 0;               // no TMA descriptor: this layer stays on the CUDA-core kernel
         }
-        P.rows_in = 0; P.rows_done = 0; P.tc_launches = 0;
+        P.rows_in = 0; P.rows_done = 0; P.tc_launches = 0; P.pending = 0;
     }
     if (e == cudaSuccess) e = cudaMemsetAsync(net->ws + net->status_off, 0, sizeof(unsigned int), net->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(net->ws + net->state_region_off, 0, net->state_region_bytes, net->stream);
