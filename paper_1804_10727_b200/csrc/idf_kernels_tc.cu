@@ -29,7 +29,7 @@ namespace idf {
 namespace {
 
 constexpr int TC_THREADS = 320;
-constexpr int ROWQ = 16;                     // row-schedule queue entries (more than the stages in flight)
+constexpr int ROWQ = 64;                     // row-schedule queue: two chunks of 32 rows
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr size_t SMEM_LIMIT = 232448;        // 227 KB per CTA
 
@@ -376,7 +376,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     __shared__ int s_issued;
-    __shared__ int s_ph_cnt[32], s_ph_off[32];                        // scratch of the MMA thread
     __shared__ __align__(16) uint32_t s_rowq[ROWQ][16];                // per input row: what the MMA thread must do
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its own prologue
@@ -441,70 +440,71 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // for free stages, therefore also works out for every input row which accumulators it feeds
         // and leaves the answer in a small queue next to the data (published by the stage's barrier).
         // With t0 = base_ty + ri the taps of input row ri are ky = ph, ph+s, ... (ph = t0 mod s), and
-        // tap ky = ph + j*s reaches relative output row hi - j (hi = t0 div s).  All incremental.
-        if (lane == 0) {
-            const uint32_t idesc0 = (DT == 1 ? ((1u << 4) | (1u << 7) | (1u << 10)) : ((2u << 4) | (1u << 7) | (1u << 10))) |
-                                    ((128u >> 4) << 24);
-            const int max_rows = 256 / a.Ntile;          // ring rows one instruction can cover (N <= 256)
-            const int s = a.stride, nslot = a.nslot;
-            // taps per phase and where their blocks start in the stacked weight tile (see weight_block)
-            for (int p = 0, off = 0; p < s; ++p) {
-                s_ph_cnt[p] = (a.Kh - p + s - 1) / s;
-                s_ph_off[p] = off;
-                off += s_ph_cnt[p];
-            }
-            int t0 = a.base_ty;
-            int ph = t0 % s, hi = t0 / s;
-            int slot_hi = hi % nslot, u_hi = hi / nslot;
-            // the row completed by input row ri is (t0 - (Kh-1)) / s when that is a whole number >= 0
-            int of, phf;
+        // tap ky = ph + j*s reaches relative output row hi - j (hi = t0 div s).
+        // The 32 lanes work out the schedule of 32 rows at a time (one row each, closed form), then
+        // lane 0 issues those rows' copies.
+        const uint32_t idesc0 = (DT == 1 ? ((1u << 4) | (1u << 7) | (1u << 10)) : ((2u << 4) | (1u << 7) | (1u << 10))) |
+                                ((128u >> 4) << 24);
+        const int max_rows = 256 / a.Ntile;              // ring rows one instruction can cover (N <= 256)
+        const int s = a.stride, nslot = a.nslot;
+        int stage = 0, t = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int r_chunk = 0; r_chunk < n_rows && ok; r_chunk += 32) {
             {
-                const int tf = t0 - (a.Kh - 1);
-                if (tf >= 0) { of = tf / s; phf = tf - of * s; }
-                else { of = -((-tf + s - 1) / s); phf = tf - of * s; }
-            }
-            int slot_f = ((of % nslot) + nslot) % nslot;
-            int stage = 0, t = 0;
-            uint32_t phase = 0;
-            bool ok = true;
-            for (int ri = 0; ri < n_rows && ok; ++ri) {
-                uint32_t* q = s_rowq[ri & (ROWQ - 1)];
-                // a new output row starts when ph == 0: its slot's previous row must have been read out
-                const bool fresh = (ri > 0 && ph == 0 && hi >= nslot);
-                q[0] = fresh ? bar_free + 8u * (uint32_t)slot_hi : 0u;
-                q[1] = (uint32_t)(u_hi & 1);
-                q[3] = (phf == 0 && of >= 0 && of < a.done_rel) ? bar_ready + 8u * (uint32_t)slot_f : 0u;
-                int n_t = s_ph_cnt[ph];
-                if (n_t > hi + 1) n_t = hi + 1;          // taps that would reach rows above the map drop out
-                int sl = slot_hi - (n_t - 1);
-                if (sl < 0) sl += nslot;
-                uint32_t blk = (uint32_t)(s_ph_off[ph] + s_ph_cnt[ph] - n_t);
-                // segments: runs of rows whose slots are consecutive TMEM column blocks (N <= 256 each)
-                int n_seg = 0;
-                for (int rem = n_t; rem > 0 && n_seg < 4; ++n_seg) {
-                    int len = rem;
-                    if (len > nslot - sl) len = nslot - sl;
-                    if (len > max_rows) len = max_rows;
-                    q[4 + 3 * n_seg] = tmem_base + (uint32_t)(sl * a.Ntile);
-                    q[5 + 3 * n_seg] = (blk * w_tile_bytes) >> 4;
-                    q[6 + 3 * n_seg] = idesc0 | ((uint32_t)((len * a.Ntile) >> 3) << 17);
-                    rem -= len; blk += (uint32_t)len; sl += len;
-                    if (sl == nslot) sl = 0;
-                }
-                q[2] = (uint32_t)n_seg;
-                for (int xl = 0; xl < n_xload && ok; ++xl)
-                    for (int kb = 0; kb < a.n_kb; ++kb) {
-                        if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-                        mbar_expect_tx(bar_full + 8u * stage, a_box_bytes);
-                        tma_load_4d(sA + (uint32_t)stage * a_stage_bytes, &tmA, bar_full + 8u * stage,
-                                    kb * a.KB, x0 - a.pad_x + xl, s0, ri);
-                        s_issued = ++t;
-                        if (++stage == a.nstage) { stage = 0; phase ^= 1u; }
+                const int ri = r_chunk + lane;
+                if (ri < n_rows) {
+                    uint32_t* q = s_rowq[ri & (ROWQ - 1)];
+                    const int t0 = a.base_ty + ri;
+                    const int hi = t0 / s, ph = t0 - hi * s;
+                    const int slot_hi = hi % nslot, u_hi = hi / nslot;
+                    // a new output row starts when ph == 0: its slot's previous row must have been read out
+                    const bool fresh = (ri > 0 && ph == 0 && hi >= nslot);
+                    q[0] = fresh ? bar_free + 8u * (uint32_t)slot_hi : 0u;
+                    q[1] = (uint32_t)(u_hi & 1);
+                    // the row completed by input row ri is (t0 - (Kh-1)) / s when that is a whole number >= 0
+                    const int tf = t0 - (a.Kh - 1);
+                    const int of = tf >= 0 ? tf / s : -1;
+                    q[3] = (tf >= 0 && of * s == tf && of < a.done_rel) ? bar_ready + 8u * (uint32_t)(of % nslot) : 0u;
+                    // taps ky = ph, ph+s, ... < Kh; those that would reach rows above the map drop out
+                    const int cnt = (a.Kh - ph + s - 1) / s;
+                    int n_t = cnt;
+                    if (n_t > hi + 1) n_t = hi + 1;
+                    int sl = slot_hi - (n_t - 1);
+                    if (sl < 0) sl += nslot;
+                    int poff = 0;
+                    for (int p = 0; p < ph; ++p) poff += (a.Kh - p + s - 1) / s;
+                    uint32_t blk = (uint32_t)(poff + cnt - n_t);
+                    // segments: runs of rows whose slots are consecutive TMEM column blocks (N <= 256 each)
+                    int n_seg = 0;
+                    for (int rem = n_t; rem > 0 && n_seg < 4; ++n_seg) {
+                        int len = rem;
+                        if (len > nslot - sl) len = nslot - sl;
+                        if (len > max_rows) len = max_rows;
+                        q[4 + 3 * n_seg] = tmem_base + (uint32_t)(sl * a.Ntile);
+                        q[5 + 3 * n_seg] = (blk * w_tile_bytes) >> 4;
+                        q[6 + 3 * n_seg] = idesc0 | ((uint32_t)((len * a.Ntile) >> 3) << 17);
+                        rem -= len; blk += (uint32_t)len; sl += len;
+                        if (sl == nslot) sl = 0;
                     }
-                ++t0;
-                if (++ph == s) { ph = 0; ++hi; if (++slot_hi == nslot) { slot_hi = 0; ++u_hi; } }
-                if (++phf == s) { phf = 0; ++of; if (++slot_f == nslot) slot_f = 0; }
+                    q[2] = (uint32_t)n_seg;
+                }
             }
+            __syncwarp();
+            if (lane == 0) {
+                const int r_end = r_chunk + 32 < n_rows ? r_chunk + 32 : n_rows;
+                for (int ri = r_chunk; ri < r_end && ok; ++ri)
+                    for (int xl = 0; xl < n_xload && ok; ++xl)
+                        for (int kb = 0; kb < a.n_kb; ++kb) {
+                            if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                            mbar_expect_tx(bar_full + 8u * stage, a_box_bytes);
+                            tma_load_4d(sA + (uint32_t)stage * a_stage_bytes, &tmA, bar_full + 8u * stage,
+                                        kb * a.KB, x0 - a.pad_x + xl, s0, ri);
+                            s_issued = ++t;
+                            if (++stage == a.nstage) { stage = 0; phase ^= 1u; }
+                        }
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -615,28 +615,46 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const bool carried_in = a.r0_positive && (orel * a.stride - a.base_ty < 0);
             TS* rp = ring_pos + (long long)((a.o_begin + orel) % a.ring_rows) * ring_slot_stride;
             const uint32_t trow = tlane + (uint32_t)(slot * a.Ntile);
-            if (wide) {
-                for (int c = 0; c < a.Ntile; c += 32) {
-                    uint32_t v[32];
-                    tmem_ld<32>(trow + c, v);
-                    tmem_st_zero<32>(trow + c);           // the slot's next row starts from zero
-                    if (emit ? in_tile : valid)
-                        finalise_chunk<DT, 32, TS>(v, carried_in && valid, emit, rp + c, bias ? bias + c : nullptr, sink,
-                                                   (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift);
+            if (a.Ntile == 64 || a.Ntile == 32) {
+                // the whole row fits in registers: take it, clear and release the slot at once, then finalise
+                uint32_t v0[32], v1[32];
+                tmem_ld<32>(trow, v0);
+                if (a.Ntile == 64) tmem_ld<32>(trow + 32, v1);
+                tmem_st_zero<32>(trow);
+                if (a.Ntile == 64) tmem_st_zero<32>(trow + 32);
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(bar_free + 8u * slot);
+                if (emit ? in_tile : valid) {
+                    finalise_chunk<DT, 32, TS>(v0, carried_in && valid, emit, rp, bias, sink, 0u, a.out_elem, a.relu, a.shift);
+                    if (a.Ntile == 64)
+                        finalise_chunk<DT, 32, TS>(v1, carried_in && valid, emit, rp + 32, bias ? bias + 32 : nullptr, sink,
+                                                   (uint32_t)(32 * a.out_esize), a.out_elem, a.relu, a.shift);
                 }
             } else {
-                for (int c = 0; c < a.Ntile; c += 16) {
-                    uint32_t v[16];
-                    tmem_ld<16>(trow + c, v);
-                    tmem_st_zero<16>(trow + c);
-                    if (emit ? in_tile : valid)
-                        finalise_chunk<DT, 16, TS>(v, carried_in && valid, emit, rp + c, bias ? bias + c : nullptr, sink,
-                                                   (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift);
+                if (wide) {
+                    for (int c = 0; c < a.Ntile; c += 32) {
+                        uint32_t v[32];
+                        tmem_ld<32>(trow + c, v);
+                        tmem_st_zero<32>(trow + c);           // the slot's next row starts from zero
+                        if (emit ? in_tile : valid)
+                            finalise_chunk<DT, 32, TS>(v, carried_in && valid, emit, rp + c, bias ? bias + c : nullptr, sink,
+                                                       (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift);
+                    }
+                } else {
+                    for (int c = 0; c < a.Ntile; c += 16) {
+                        uint32_t v[16];
+                        tmem_ld<16>(trow + c, v);
+                        tmem_st_zero<16>(trow + c);
+                        if (emit ? in_tile : valid)
+                            finalise_chunk<DT, 16, TS>(v, carried_in && valid, emit, rp + c, bias ? bias + c : nullptr, sink,
+                                                       (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift);
+                    }
                 }
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(bar_free + 8u * slot);
             }
-            tmem_st_wait();
-            tc_fence_before();
-            mbar_arrive(bar_free + 8u * slot);
             if (emit) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 named_bar_sync(1 + grp, 128);
@@ -745,7 +763,7 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
         if ((ring_rows + 1) * nt > 512) continue;
         if ((ring_rows + 256 / nt - 1) / (256 / nt) + 1 > 4) continue;   // at most 4 MMA segments per input row
         const size_t wb = (size_t)taps * p->n_kb * nt * p->swb;
-        if (wb + 3 * a_stage + 128 * (size_t)nt * out_esize + 6144 > SMEM_LIMIT) continue;   // one staging tile at least
+        if (wb + 3 * a_stage + 128 * (size_t)nt * out_esize + 10240 > SMEM_LIMIT) continue;   // one staging tile at least
         const int units = p->n_mt * (Cout / nt);
         if (units >= 120) { best = nt; break; }          // enough CTAs for the 148 SMs: take the widest such tile
         if (units > best_units) { best_units = units; best = nt; }
@@ -766,8 +784,8 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     p->out_panels = best * out_esize / p->out_pwb;
     p->out_stage_bytes = p->out_panels * 128 * p->out_pwb;
     // two epilogue groups (two staging tiles) when that still leaves three Δ-row stages, else one
-    p->out_groups = (wb + 3 * a_stage + 2 * (size_t)p->out_stage_bytes + 6144 <= SMEM_LIMIT) ? 2 : 1;
-    const size_t room = SMEM_LIMIT - 4096 - wb - 1024 - (size_t)p->out_groups * p->out_stage_bytes;   // static shared memory and alignment slack stay free
+    p->out_groups = (wb + 3 * a_stage + 2 * (size_t)p->out_stage_bytes + 10240 <= SMEM_LIMIT) ? 2 : 1;
+    const size_t room = SMEM_LIMIT - 8192 - wb - 1024 - (size_t)p->out_groups * p->out_stage_bytes;   // static shared memory and alignment slack stay free
     int nstage = (int)(room / a_stage);
     if (nstage > 8) nstage = 8;
     if (nstage < 2) return false;
@@ -858,7 +876,7 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!attr_set[dtype - 1][kidx][dev]) {
-        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_LIMIT - 2048));
+        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_LIMIT - 6144));
         if (e != cudaSuccess) return e;
         attr_set[dtype - 1][kidx][dev] = true;
     }
