@@ -299,22 +299,35 @@ __device__ __forceinline__ void finalise_chunk(const uint32_t (&v)[W], bool carr
     if (DT == 1) {
         float f[W];
 #pragma unroll
-        for (int j = 0; j < W; ++j) {
-            float t = (float)acc[j] + (bias_c ? (float)bias_c[j] : 0.f);
-            f[j] = (relu && t < 0.f) ? 0.f : t;
+        for (int j = 0; j < W; ++j) f[j] = (float)acc[j];
+        if (bias_c) {
+#pragma unroll
+            for (int j4 = 0; j4 < W / 4; ++j4) {
+                const float4 b4 = ((const float4*)bias_c)[j4];
+                f[4 * j4] += b4.x; f[4 * j4 + 1] += b4.y; f[4 * j4 + 2] += b4.z; f[4 * j4 + 3] += b4.w;
+            }
         }
         if (out_elem == E_BF16) {
+            // two values per instruction: round to nearest even, with the ReLU folded into the conversion
+            uint32_t pk[W / 2];
+            if (relu) {
 #pragma unroll
-            for (int j8 = 0; j8 < W / 8; ++j8) {
-                uint32_t pk[4];
+                for (int j = 0; j < W / 2; ++j)
+                    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(pk[j]) : "f"(f[2 * j + 1]), "f"(f[2 * j]));
+            } else {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    __nv_bfloat162 h2 = __floats2bfloat162_rn(f[8 * j8 + 2 * j], f[8 * j8 + 2 * j + 1]);
-                    pk[j] = *(uint32_t*)&h2;
-                }
-                stage_store16(sink, col_byte + 16u * j8, make_int4((int)pk[0], (int)pk[1], (int)pk[2], (int)pk[3]));
+                for (int j = 0; j < W / 2; ++j)
+                    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk[j]) : "f"(f[2 * j + 1]), "f"(f[2 * j]));
             }
+#pragma unroll
+            for (int j8 = 0; j8 < W / 8; ++j8)
+                stage_store16(sink, col_byte + 16u * j8,
+                              make_int4((int)pk[4 * j8], (int)pk[4 * j8 + 1], (int)pk[4 * j8 + 2], (int)pk[4 * j8 + 3]));
         } else {
+            if (relu) {
+#pragma unroll
+                for (int j = 0; j < W; ++j) f[j] = fmaxf(f[j], 0.f);
+            }
 #pragma unroll
             for (int j4 = 0; j4 < W / 4; ++j4)
                 stage_store16(sink, col_byte + 16u * j4,
