@@ -16,7 +16,7 @@
 //     requantise, and write the row for the next layer; rows still open at the end of the block go
 //     back to the ring in global memory.
 // Warp roles: warp 0 = TMA producer and row scheduler, warp 1 = TMEM owner and MMA issuer,
-// warps 2-9 = epilogue (two per TMEM lane quarter).
+// warps 2.. = epilogue groups of four warps (one warp per TMEM lane quarter) that take output rows in turn.
 // Every wait is bounded; on expiry the kernel records IDF_ERR_TIMEOUT in the status word and leaves.
 #include "idf_internal.h"
 
@@ -28,7 +28,8 @@ namespace idf {
 
 namespace {
 
-constexpr int TC_THREADS = 320;
+constexpr int MAX_GROUPS = 4;                // epilogue groups (four warps each) taking output rows in turn
+constexpr int TC_THREADS = 64 + 128 * MAX_GROUPS;
 constexpr int ROWQ = 64;                     // row-schedule queue: two chunks of 32 rows
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr size_t SMEM_LIMIT = 232448;        // 227 KB per CTA
@@ -577,7 +578,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         __syncwarp();
     } else {
         // ------------------------------ epilogue: row finalisation -----------------------------
-        // Two groups of four warps (one warp per TMEM lane quarter) take the output rows in turn.
+        // Groups of four warps (one warp per TMEM lane quarter) take the output rows in turn.
         // An emitted row is first laid out in the group's shared-memory tile (each thread writes its
         // own tile row, swizzled), then one thread hands the tile to a TMA store, which writes whole
         // lines and clips whatever lies outside the map.
@@ -613,7 +614,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 tc_fence_before();
                 mbar_arrive(bar_free + 8u * slot);
             }
-        for (int orel = grp; orel < a.n_orows && ok && grp < a.out_groups; orel += a.out_groups) {
+        // Rows that exchange state with the ring in global memory (those begun by an earlier block and
+        // those left open by this one) may share a ring slot; group 0 takes them all, in order, so a
+        // slot is read before it is rewritten.  The other rows go round the groups.
+        const int n_cin = a.r0_positive ? (a.base_ty + a.stride - 1) / a.stride : 0;
+        for (int orel = 0; orel < a.n_orows && ok && grp < a.out_groups; ++orel) {
+            const int owner = (orel < n_cin || orel >= a.done_rel) ? 0 : orel % a.out_groups;
+            if (owner != grp) continue;
             const int slot = orel % a.nslot;
             const uint32_t par = (uint32_t)((orel / a.nslot) & 1);
             const bool emit = orel < a.done_rel;
@@ -796,8 +803,10 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     p->out_pwb = best * out_esize >= 128 ? 128 : best * out_esize;
     p->out_panels = best * out_esize / p->out_pwb;
     p->out_stage_bytes = p->out_panels * 128 * p->out_pwb;
-    // two epilogue groups (two staging tiles) when that still leaves three Δ-row stages, else one
-    p->out_groups = (wb + 3 * a_stage + 2 * (size_t)p->out_stage_bytes + 10240 <= SMEM_LIMIT) ? 2 : 1;
+    // as many epilogue groups (one staging tile each) as still leave three Δ-row stages
+    p->out_groups = 1;
+    for (int g = MAX_GROUPS; g > 1; --g)
+        if (wb + 3 * a_stage + (size_t)g * p->out_stage_bytes + 10240 <= SMEM_LIMIT) { p->out_groups = g; break; }
     const size_t room = SMEM_LIMIT - 8192 - wb - 1024 - (size_t)p->out_groups * p->out_stage_bytes;   // static shared memory and alignment slack stay free
     int nstage = (int)(room / a_stage);
     if (nstage > 8) nstage = 8;
@@ -900,9 +909,8 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    // Opt-in (IDF_PDL=1): with it one end-to-end parity case fails intermittently, cause not found yet;
-    // without the attribute the griddepcontrol instructions in the kernels are no-ops.
-    static const bool use_pdl = getenv("IDF_PDL") != nullptr;
+    // (IDF_NO_PDL=1 turns it off; the griddepcontrol instructions in the kernels are then no-ops)
+    static const bool use_pdl = getenv("IDF_NO_PDL") == nullptr;
     cfg.attrs = attr; cfg.numAttrs = use_pdl ? 1 : 0;
     cudaError_t le = cudaLaunchKernelEx(&cfg, fn, tmA, *(const CUtensorMap*)w_map, tmO, t);
     if (le != cudaSuccess) return le;
