@@ -318,7 +318,8 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
     idf_net* net = new (std::nothrow) idf_net();
     if (!net) return fail(IDF_ERR_ARG, "out of host memory");
     net->dtype = spec->dtype; net->in_w = spec->in_w; net->in_c = spec->in_c; net->n_streams = spec->n_streams;
-    net->row_block = spec->row_block > 0 ? spec->row_block : 32;
+    // default: about 8192 positions per stream and block (32 rows of a 224-wide image, 1024 samples of a 1D signal)
+    net->row_block = spec->row_block > 0 ? spec->row_block : std::min(1024, std::max(32, 8192 / spec->in_w));
     const int act_elem = spec->dtype == IDF_F32 ? E_F32 : (spec->dtype == IDF_BF16_F32 ? E_BF16 : E_I8);
     const size_t state_word = 4;
 

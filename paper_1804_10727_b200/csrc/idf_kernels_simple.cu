@@ -212,6 +212,7 @@ __global__ void __launch_bounds__(SPARSE_THREADS) conv_sparse_kernel(ConvArgs a)
 
     const int n_comp = a.Win * a.Cin;
     const int taps = a.Kh * a.Kw;
+    const int slot0 = (int)(a.o_begin % a.ring_rows);     // ring slot of the first visited row
     long long done = a.o_begin;                      // rows below `done` have been emitted
     for (long long r = a.r0; r <= a.r1; ++r) {
         // r == r1 is the flush pass: no input, only rows up to done_end are finalised
@@ -239,24 +240,25 @@ __global__ void __launch_bounds__(SPARSE_THREADS) conv_sparse_kernel(ConvArgs a)
                 __syncthreads();
                 const int n_ev = ev_count;
                 if (tid == 0) ev_total += (unsigned long long)n_ev;
-                // scatter: item = (event, tap, co); consecutive threads differ in co
-                const long long items = (long long)n_ev * taps * a.Cout;
-                for (long long it = tid; it < items; it += SPARSE_THREADS) {
-                    const int co = (int)(it % a.Cout);
-                    const int t2 = (int)(it / a.Cout);
+                // scatter: item = (event, tap, co); consecutive threads differ in co.  All index
+                // arithmetic in 32 bits: for every tap row ky the target ring slot is worked out once.
+                const int items = n_ev * taps * a.Cout;
+                // relative target row of tap ky: (r + pad - ky) / stride when whole and not below o_begin
+                for (int it = tid; it < items; it += SPARSE_THREADS) {
+                    const int co = it % a.Cout;
+                    const int t2 = it / a.Cout;
                     const int tap = t2 % taps, e = t2 / taps;
                     const int ky = tap / a.Kw, kx = tap - ky * a.Kw;
                     const int pos = ev_pos[e];
                     const int x = pos / a.Cin, ci = pos - x * a.Cin;
-                    const long long ty = r + a.pad - ky;
+                    const int ty = (int)(r - a.o_begin * a.stride) + a.pad - ky;    // relative to row o_begin
                     const int tx = x + a.pad_x - kx;
-                    if (ty < 0 || tx < 0 || ty % a.stride || tx % a.stride_x) continue;
-                    const long long o = ty / a.stride;
-                    const int ox = tx / a.stride_x;
-                    if (ox >= a.Wout || o < a.o_begin) continue;
-                    const TS wv = (TS)to_acc(w[((long long)(ky * a.Kw + kx) * a.Cin + ci) * a.Cout + co]);
-                    atomic_add(&ring[ring_base + (o % a.ring_rows) * slot_stride + (long long)ox * a.Cout + co],
-                               ev_val[e] * wv);
+                    if (ty < 0 || tx < 0) continue;
+                    const int orel = ty / a.stride, ox = tx / a.stride_x;
+                    if (orel * a.stride != ty || ox * a.stride_x != tx || ox >= a.Wout) continue;
+                    const int slot = (slot0 + orel) % a.ring_rows;
+                    const TS wv = (TS)to_acc(w[((ky * a.Kw + kx) * a.Cin + ci) * a.Cout + co]);
+                    atomic_add(&ring[ring_base + slot * slot_stride + ox * a.Cout + co], ev_val[e] * wv);
                 }
                 __syncthreads();
             }
@@ -272,13 +274,30 @@ __global__ void __launch_bounds__(SPARSE_THREADS) conv_sparse_kernel(ConvArgs a)
         }
         for (; done < upto; ++done) {
             const long long slot = done % a.ring_rows;
-            for (int i = tid; i < row_elems; i += SPARSE_THREADS) {
-                TS* p = &ring[ring_base + slot * slot_stride + i];
-                const TS c = *p;
-                *p = 0;
-                const int co = i % a.Cout;
-                out[(done - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride + i] =
-                    Emit<TO, TS>::run(c, bias ? bias[co] : (TS)0, a.relu, a.shift);
+            TO* orow = out + (done - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride;
+            if (sizeof(TO) == 1 && (a.Cout & 3) == 0 && (((uintptr_t)orow) & 3) == 0) {
+                // int8 rows: four channels per thread, one 4-byte store
+                for (int i = tid * 4; i < row_elems; i += SPARSE_THREADS * 4) {
+                    TS* p = &ring[ring_base + slot * slot_stride + i];
+                    const int co = i % a.Cout;
+                    uint32_t pk = 0;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const TS c = p[j];
+                        p[j] = 0;
+                        const TO v = Emit<TO, TS>::run(c, bias ? bias[co + j] : (TS)0, a.relu, a.shift);
+                        pk |= ((uint32_t)(*(const unsigned char*)&v)) << (8 * j);
+                    }
+                    *(uint32_t*)(orow + i) = pk;
+                }
+            } else {
+                for (int i = tid; i < row_elems; i += SPARSE_THREADS) {
+                    TS* p = &ring[ring_base + slot * slot_stride + i];
+                    const TS c = *p;
+                    *p = 0;
+                    const int co = i % a.Cout;
+                    orow[i] = Emit<TO, TS>::run(c, bias ? bias[co] : (TS)0, a.relu, a.shift);
+                }
             }
         }
         __syncthreads();
