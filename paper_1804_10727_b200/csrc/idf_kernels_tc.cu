@@ -58,6 +58,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// Non-blocking look at a barrier phase (the result may be consumed much later: the round trip to the
+// barrier then overlaps whatever is issued in between).
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
 // Bounded wait: false if the limit ran out or another role has given up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
@@ -67,6 +79,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             __nanosleep(32);
         }
+    }
+    *abort_flag = 1;
+    return false;
+}
+// The same for roles that are not on the critical path (producer waiting for a free stage, epilogue
+// waiting for a finished row): sleep between polls, so the polling warp leaves the issue slots of its
+// scheduler to the MMA-issuing warp that shares it.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(200);
+        if ((i & 15u) == 15u && *abort_flag) return false;
     }
     *abort_flag = 1;
     return false;
@@ -83,6 +108,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+
+// true in exactly one lane of a converged warp
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -421,7 +454,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         s_issued = 0;
         for (int i = 0; i < a.nstage; ++i) { mbar_init(bar_full + 8u * i, 1); mbar_init(bar_empty + 8u * i, 1); }
         for (int i = 0; i < taps; ++i) mbar_init(bar_w + 8u * i, 1);
-        for (int i = 0; i < a.nslot; ++i) { mbar_init(bar_ready + 8u * i, 1); mbar_init(bar_free + 8u * i, 128); }
+        for (int i = 0; i < a.nslot; ++i) { mbar_init(bar_ready + 8u * i, 1); mbar_init(bar_free + 8u * i, 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         // The weights do not depend on earlier kernels of the stream: fetch them before waiting for
         // the previous kernel (programmatic dependent launch), so the fetch overlaps its tail.
@@ -507,72 +540,116 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             __syncwarp();
             if (lane == 0) {
                 const int r_end = r_chunk + 32 < n_rows ? r_chunk + 32 : n_rows;
-                for (int ri = r_chunk; ri < r_end && ok; ++ri)
+                for (int ri = r_chunk; ri < r_end && ok; ++ri) {
+                    // A row that starts a new output row needs that row's slot read out and cleared.  Waiting
+                    // here, before the row's first copy, means the MMA thread learns it from the copy's
+                    // barrier and has one barrier less to look at.
+                    const uint32_t* qr = s_rowq[ri & (ROWQ - 1)];
+                    if (qr[0] && !mbar_wait(qr[0], qr[1], abort_flag)) { ok = false; break; }
                     for (int xl = 0; xl < n_xload && ok; ++xl)
                         for (int kb = 0; kb < a.n_kb; ++kb) {
                             if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                             mbar_expect_tx(bar_full + 8u * stage, a_box_bytes);
                             tma_load_4d(sA + (uint32_t)stage * a_stage_bytes, &tmA, bar_full + 8u * stage,
                                         kb * a.KB, x0 - a.pad_x + xl, s0, ri);
-                            s_issued = ++t;
+                            ++t;
                             if (++stage == a.nstage) { stage = 0; phase ^= 1u; }
                         }
+                }
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         }
+        if (lane == 0) s_issued = t;     // copies in flight, for the clean-up after a failed wait
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ---------------------------------------------
-        if (lane == 0) {
+        // The whole warp runs this loop in step (every value in it is the same in all lanes) and one
+        // elected lane issues the tensor-core instructions.  The tensor pipe runs only a few instructions
+        // behind the issuing lane, so every cycle spent here on anything but issuing is a cycle the pipe
+        // idles.  Hence: the barrier of the NEXT tile is looked at (non-blocking) before the current
+        // tile's MMAs are issued and the answer is read after them, the next row's schedule entry is
+        // fetched the same way, and the wait for a free accumulator slot is the producer's (a tile of a
+        // row only arrives once its slot is free).
+        {
             const uint64_t desc_hi = make_smem_desc(0, a.swb);
             const int n_kx = a.shift_mode ? a.Kw : 1;
             const int nslot = a.nslot;
             const uint32_t kx_bytes = a.shift_mode ? (uint32_t)a.swb >> 4 : 0u;
             const uint32_t wtile_kx = ((uint32_t)(a.n_kb * a.Kh) * w_tile_bytes) >> 4;   // descriptor units per kx
             const uint32_t wtile_kb = ((uint32_t)a.Kh * w_tile_bytes) >> 4;
+            const uint32_t a_stage_units = a_stage_bytes >> 4;
+            const int nstage = a.nstage, n_kb = a.n_kb;
             bool ok = true;
             for (int slot = 0; slot < nslot && ok; ++slot)       // every slot has been cleared once
                 ok = mbar_wait(bar_free + 8u * slot, 0, abort_flag);
             for (int tap = 0; tap < taps && ok; ++tap)            // the CTA's weight slice has landed
                 ok = mbar_wait(bar_w + 8u * tap, 0, abort_flag);
-            tc_fence_after();
             const uint64_t adesc_base = desc_hi | (uint64_t)((sA & 0x3FFFFu) >> 4);
             const uint64_t bdesc_base = desc_hi | (uint64_t)((sW & 0x3FFFFu) >> 4);
+            const int n_st = n_xload * n_kb;                     // tiles per input row
+            const bool issuer = elect_one();                     // the lane that issues (the warp stays converged)
             int stage = 0;
             uint32_t phase = 0;
+            uint64_t adesc_stage = adesc_base;                   // descriptor of the current stage's tile
+            ok = ok && mbar_wait(bar_full, 0, abort_flag);       // first tile of the first row
+            tc_fence_after();
+            uint4 hdr = make_uint4(0, 0, 0, 0), sa = hdr, sb = hdr, sc = hdr;
+            if (ok) {
+                const uint4* q = (const uint4*)s_rowq[0];
+                hdr = q[0]; sa = q[1]; sb = q[2]; sc = q[3];
+            }
             for (int ri = 0; ri < n_rows && ok; ++ri) {
-                uint4 hdr = make_uint4(0, 0, 0, 0), sa = hdr, sb = hdr, sc = hdr;
+                const bool last_row = ri == n_rows - 1;
+                // schedule entries are published 32 rows at a time, ahead of the first copy of those rows
+                const bool early_info = !last_row && ((ri + 1) & 31) != 0;
+                const uint4* qn = (const uint4*)s_rowq[(ri + 1) & (ROWQ - 1)];
+                uint4 nh = make_uint4(0, 0, 0, 0), na = nh, nb = nh, nc = nh;
+                int st = 0;
                 for (int xl = 0; xl < n_xload && ok; ++xl)
-                    for (int kb = 0; kb < a.n_kb; ++kb) {
-                        if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag)) { ok = false; break; }
-                        tc_fence_after();
-                        if (xl == 0 && kb == 0) {        // the row's schedule came with its first tile
-                            const uint4* q = (const uint4*)s_rowq[ri & (ROWQ - 1)];
-                            hdr = q[0]; sa = q[1]; sb = q[2]; sc = q[3];
-                            if (hdr.x) {
-                                if (!mbar_wait(hdr.x, hdr.y, abort_flag)) { ok = false; break; }
-                                tc_fence_after();
-                            }
-                        }
+                    for (int kb = 0; kb < n_kb; ++kb, ++st) {
+                        const bool row_end = st == n_st - 1;
+                        int nstage_i = stage + 1;
+                        uint32_t nphase = phase;
+                        uint64_t adesc_next = adesc_stage + a_stage_units;
+                        if (nstage_i == nstage) { nstage_i = 0; nphase ^= 1u; adesc_next = adesc_base; }
                         // tap kx reads the same tile kxi rows further down: the swizzle is a function of
                         // the absolute shared-memory address, so a start address moved by whole rows
                         // still meets the pattern the TMA wrote (base-offset field stays 0)
-                        uint64_t adesc = adesc_base + (uint64_t)(((uint32_t)stage * a_stage_bytes) >> 4);
+                        uint64_t adesc = adesc_stage;
                         uint64_t bdesc = bdesc_base + (uint64_t)((a.shift_mode ? 0u : (uint32_t)xl) * wtile_kx + (uint32_t)kb * wtile_kb);
+                        uint32_t next_ok = 1u;
                         for (int kxi = 0; kxi < n_kx; ++kxi, adesc += kx_bytes, bdesc += wtile_kx) {
-                            umma_tile<DT, KSTEPS>(sa.x, adesc, bdesc + (uint64_t)sa.y, sa.z);
-                            if (hdr.z > 1) umma_tile<DT, KSTEPS>(sa.w, adesc, bdesc + (uint64_t)sb.x, sb.y);
-                            if (hdr.z > 2) umma_tile<DT, KSTEPS>(sb.z, adesc, bdesc + (uint64_t)sb.w, sc.x);
-                            if (hdr.z > 3) umma_tile<DT, KSTEPS>(sc.y, adesc, bdesc + (uint64_t)sc.z, sc.w);
+                            if (issuer) {
+                                umma_tile<DT, KSTEPS>(sa.x, adesc, bdesc + (uint64_t)sa.y, sa.z);
+                                if (hdr.z > 1) {
+                                    umma_tile<DT, KSTEPS>(sa.w, adesc, bdesc + (uint64_t)sb.x, sb.y);
+                                    if (hdr.z > 2) umma_tile<DT, KSTEPS>(sb.z, adesc, bdesc + (uint64_t)sb.w, sc.x);
+                                    if (hdr.z > 3) umma_tile<DT, KSTEPS>(sc.y, adesc, bdesc + (uint64_t)sc.z, sc.w);
+                                }
+                            }
+                            if (kxi == 0) {
+                                // with the first MMAs of the tile queued: look at the next tile's barrier and
+                                // fetch the next row's schedule entry
+                                if (!(last_row && row_end)) next_ok = mbar_test(bar_full + 8u * nstage_i, nphase);
+                                if (row_end && early_info) { nh = qn[0]; na = qn[1]; nb = qn[2]; nc = qn[3]; }
+                            }
                         }
-                        umma_commit(bar_empty + 8u * stage);
-                        if (++stage == a.nstage) { stage = 0; phase ^= 1u; }
+                        if (issuer) {
+                            umma_commit(bar_empty + 8u * stage);
+                            if (row_end) {
+                                // the accumulator this input row completed; on the block's last row also everything still open
+                                if (hdr.w) umma_commit(hdr.w);
+                                if (last_row)
+                                    for (int orel = a.done_rel; orel < a.n_orows; ++orel) umma_commit(bar_ready + 8u * (uint32_t)(orel % nslot));
+                            }
+                        }
+                        if (!next_ok && !mbar_wait(bar_full + 8u * nstage_i, nphase, abort_flag)) { ok = false; break; }
+                        stage = nstage_i; phase = nphase; adesc_stage = adesc_next;
                     }
-                if (!ok) break;
-                // the accumulator this input row completed; on the block's last row also everything still open
-                if (hdr.w) umma_commit(hdr.w);
-                if (ri == n_rows - 1)
-                    for (int orel = a.done_rel; orel < a.n_orows; ++orel) umma_commit(bar_ready + 8u * (uint32_t)(orel % nslot));
+                if (!ok || last_row) break;
+                if (!early_info) { nh = qn[0]; na = qn[1]; nb = qn[2]; nc = qn[3]; }
+                hdr = nh; sa = na; sb = nb; sc = nc;
+                tc_fence_after();                                // the next row may start on a slot the epilogue has just cleared
             }
         }
         __syncwarp();
@@ -612,7 +689,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 for (int c = 0; c < a.Ntile; c += 16) tmem_st16_zero(tlane + (uint32_t)(slot * a.Ntile + c));
                 tmem_st_wait();
                 tc_fence_before();
-                mbar_arrive(bar_free + 8u * slot);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_free + 8u * slot);   // one arrival per warp
             }
         // Rows that exchange state with the ring in global memory (those begun by an earlier block and
         // those left open by this one) may share a ring slot; group 0 takes them all, in order, so a
@@ -624,9 +702,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int slot = orel % a.nslot;
             const uint32_t par = (uint32_t)((orel / a.nslot) & 1);
             const bool emit = orel < a.done_rel;
-            int got = 0;
-            if (lane == 0) got = mbar_wait(bar_ready + 8u * slot, par, abort_flag) ? 1 : 0;
-            got = __shfl_sync(0xffffffffu, got, 0);
+            // one thread of the group polls the barrier; the named barrier below releases the other warps
+            int got = 1;
+            if (leader) got = mbar_wait_relaxed(bar_ready + 8u * slot, par, abort_flag) ? 1 : 0;
             // the tile must have been drained by the group's previous store before anyone writes it again;
             // the barrier also makes the whole group leave together if any of its waits ran out
             if (emit && leader) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -644,7 +722,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (a.Ntile == 64) tmem_st_zero<32>(trow + 32);
                 tmem_st_wait();
                 tc_fence_before();
-                mbar_arrive(bar_free + 8u * slot);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_free + 8u * slot);   // one arrival per warp
                 if (emit ? in_tile : valid) {
                     finalise_chunk<DT, 32, TS>(v0, carried_in && valid, emit, rp, bias, sink, 0u, a.out_elem, a.relu, a.shift);
                     if (a.Ntile == 64)
@@ -673,7 +752,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
                 tmem_st_wait();
                 tc_fence_before();
-                mbar_arrive(bar_free + 8u * slot);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_free + 8u * slot);   // one arrival per warp
             }
             if (emit) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
