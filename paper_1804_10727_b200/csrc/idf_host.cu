@@ -186,7 +186,7 @@ int launch_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, boo
         a.ring_rows = P.ring_rows; a.in_elem = P.in_elem; a.out_elem = P.out_elem;
         a.r0 = r0; a.r1 = r1; a.o_begin = o_begin; a.o_end = o_end; a.done_end = done_end;
         ce = cudaErrorNotSupported;
-        if (P.tc.ok && !P.use_sparse && !flush && n_in > 0) {
+        if (P.tc.ok && !P.use_sparse && n_in > 0) {
             ConvArgs t = a;
             if (P.unfold && n_in <= P.in_cap_rows) {
                 ce = launch_unfold(a, (int)n_in, P.kpad, net->ws + P.unf_off, net->stream);
@@ -251,9 +251,13 @@ int fire(idf_net* net, size_t i, const void* in_ptr, long long n_in, bool flush,
     if (i > 0) P.pending = 0;
     long long got = 0;
     if (n_in > 0) {
-        int rc = launch_layer(net, i, in_ptr, n_in, false, d_out, out_cap, last ? 0 : net->L[i + 1].pending, &got);
+        // When the end of input comes with the layer's last rows, one launch of a dense layer does both:
+        // it applies the rows and completes what then only waits for bottom padding.
+        const bool fused = flush && P.l.kind == IDF_CONV && !P.use_sparse;
+        int rc = launch_layer(net, i, in_ptr, n_in, fused, d_out, out_cap, last ? 0 : net->L[i + 1].pending, &got);
         if (rc != IDF_OK) return rc;
         if (last) *emitted += got; else net->L[i + 1].pending += got;
+        if (fused) flush = false;
     }
     if (flush) {
         // the arriving rows took the ordinary path above; what is left is the padding-only completion
@@ -279,15 +283,16 @@ int run_segments(idf_net* net, const void* d_segments, long long n_seg, bool flu
     int rc = IDF_OK;
     for (long long s0 = 0; s0 < n_seg && rc == IDF_OK; s0 += net->row_block) {
         const long long n = std::min<long long>(net->row_block, n_seg - s0);
-        rc = fire(net, 0, (const unsigned char*)d_segments + (size_t)s0 * seg_bytes, n, false, d_out, out_cap, emitted);
         const bool last_block = s0 + n >= n_seg;
+        const bool fin = flush && last_block;          // the input ends with this block: every layer also flushes
+        rc = fire(net, 0, (const unsigned char*)d_segments + (size_t)s0 * seg_bytes, n, fin, d_out, out_cap, emitted);
         for (size_t i = 1; i < nl && rc == IDF_OK; ++i) {
             LayerPlan& P = net->L[i];
-            if (P.pending > 0 && (P.pending >= P.fire_rows || last_block))
-                rc = fire(net, i, net->ws + net->L[i - 1].out_off, P.pending, false, d_out, out_cap, emitted);
+            if (fin || (P.pending > 0 && (P.pending >= P.fire_rows || last_block)))
+                rc = fire(net, i, net->ws + net->L[i - 1].out_off, P.pending, fin, d_out, out_cap, emitted);
         }
     }
-    if (flush)
+    if (flush && n_seg == 0)
         for (size_t i = 0; i < nl && rc == IDF_OK; ++i)
             rc = fire(net, i, i ? net->ws + net->L[i - 1].out_off : nullptr, i ? net->L[i].pending : 0, true, d_out, out_cap, emitted);
     if (rc != IDF_OK) net->phase = FINISHED;      // counters and buffers are no longer consistent: reopen to go on
@@ -318,8 +323,9 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
     idf_net* net = new (std::nothrow) idf_net();
     if (!net) return fail(IDF_ERR_ARG, "out of host memory");
     net->dtype = spec->dtype; net->in_w = spec->in_w; net->in_c = spec->in_c; net->n_streams = spec->n_streams;
-    // default: about 8192 positions per stream and block (32 rows of a 224-wide image, 1024 samples of a 1D signal)
-    net->row_block = spec->row_block > 0 ? spec->row_block : std::min(1024, std::max(32, 8192 / spec->in_w));
+    // default: about 25 000 positions per stream and block (112 rows of a 224-wide image, 1024 samples of a 1D
+    // signal): long enough that a launch's fixed cost (weights into shared memory, ring rows in and out) is small
+    net->row_block = spec->row_block > 0 ? spec->row_block : std::min(1024, std::max(32, 25088 / spec->in_w));
     const int act_elem = spec->dtype == IDF_F32 ? E_F32 : (spec->dtype == IDF_BF16_F32 ? E_BF16 : E_I8);
     const size_t state_word = 4;
 
@@ -511,12 +517,21 @@ int idf_stream_open(idf_net* net, void* d_workspace, size_t workspace_bytes, voi
                                   P.unfold ? P.kpad : P.l.cin, P.l.cout, P.w_map) != 0)
                 P.tc.ok = 0;               // no TMA descriptor: this layer stays on the CUDA-core kernel
         }
-        P.rows_in = 0; P.rows_done = 0; P.tc_launches = 0; P.pending = 0;
     }
-    if (e == cudaSuccess) e = cudaMemsetAsync(net->ws + net->status_off, 0, sizeof(unsigned int), net->stream);
+    if (e != cudaSuccess) { net->phase = CREATED; return fail(IDF_ERR_CUDA, "stream_open: %s", cudaGetErrorString(e)); }
+    net->phase = FINISHED;                 // a bound workspace with uploaded parameters: ready for a reset
+    return idf_stream_reset(net);
+}
+
+int idf_stream_reset(idf_net* net)
+{
+    if (!net) return fail(IDF_ERR_ARG, "net must not be NULL");
+    if (net->phase == CREATED) return fail(IDF_ERR_STATE, "reset before stream_open");
+    for (auto& P : net->L) { P.rows_in = 0; P.rows_done = 0; P.tc_launches = 0; P.pending = 0; }
+    cudaError_t e = cudaMemsetAsync(net->ws + net->status_off, 0, sizeof(unsigned int), net->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(net->ws + net->state_region_off, 0, net->state_region_bytes, net->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(net->ws + net->counters_off, 0, net->L.size() * sizeof(unsigned long long), net->stream);
-    if (e != cudaSuccess) { net->phase = CREATED; return fail(IDF_ERR_CUDA, "stream_open: %s", cudaGetErrorString(e)); }
+    if (e != cudaSuccess) { net->phase = CREATED; return fail(IDF_ERR_CUDA, "stream_reset: %s", cudaGetErrorString(e)); }
     net->phase = OPEN;
     net->launches = 0;
     net->out_rows_total = 0;
@@ -554,6 +569,22 @@ int idf_stream_finish(idf_net* net, void* d_out, long long out_capacity_rows, lo
     return IDF_OK;
 }
 
+int idf_stream_push_last(idf_net* net, const void* d_segments, int n_seg, void* d_out, long long out_capacity_rows,
+                         long long* total_rows)
+{
+    if (!net) return fail(IDF_ERR_ARG, "net must not be NULL");
+    if (net->phase != OPEN) return fail(IDF_ERR_STATE, net->phase == CREATED ? "push before stream_open" : "push after stream_finish");
+    if (n_seg < 0 || out_capacity_rows < 0) return fail(IDF_ERR_ARG, "negative count");
+    if (!d_out || (n_seg > 0 && !d_segments)) return fail(IDF_ERR_ARG, "d_segments and d_out must not be NULL");
+    long long em = 0;
+    int rc = run_segments(net, d_segments, n_seg, true, d_out, out_capacity_rows, &em);
+    if (rc != IDF_OK) return rc;
+    net->out_rows_total += em;
+    net->phase = FINISHED;
+    if (total_rows) *total_rows = net->out_rows_total;
+    return IDF_OK;
+}
+
 int idf_run_host(idf_net* net, const void* h_segments, int n_seg, void* d_segments, void* h_out, void* d_out,
                  long long out_capacity_rows, long long* total_rows)
 {
@@ -563,10 +594,8 @@ int idf_run_host(idf_net* net, const void* h_segments, int n_seg, void* d_segmen
     const size_t in_bytes = (size_t)n_seg * net->n_streams * net->in_w * net->in_c * elem_size(net->L[0].in_elem);
     cudaError_t e = cudaMemcpyAsync(d_segments, h_segments, in_bytes, cudaMemcpyHostToDevice, net->stream);
     if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "run_host h2d: %s", cudaGetErrorString(e));
-    int rc = idf_stream_push(net, d_segments, n_seg, d_out, out_capacity_rows, nullptr);
-    if (rc != IDF_OK) return rc;
     long long tot = 0;
-    rc = idf_stream_finish(net, d_out, out_capacity_rows, &tot);
+    int rc = idf_stream_push_last(net, d_segments, n_seg, d_out, out_capacity_rows, &tot);
     if (rc != IDF_OK) return rc;
     const LayerPlan& P = net->L.back();
     const size_t out_bytes = (size_t)net->n_streams * out_capacity_rows * P.out_w * P.out_c * elem_size(P.out_elem);

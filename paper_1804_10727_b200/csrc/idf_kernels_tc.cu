@@ -397,6 +397,8 @@ struct TcArgs {
     int n_rows;                  // input rows in this block
     int n_orows;                 // visited output rows: o_begin + [0, n_orows)
     int done_rel;                // rows with relative index < done_rel are emitted, the others go back to the ring
+    int sched_rel;               // rows below it are completed by an input row of this block; rows in [sched_rel, done_rel)
+                                 // wait only for bottom padding and are completed by the block's last row (end of input)
     int base_ty;                 // r0 + pad - o_begin*stride: input row ri reaches relative output row
                                  // (base_ty + ri - ky) / stride through tap ky when that is a whole number >= 0
     int S, Wout, Cout, Kh, Kw, stride, pad_x, relu, shift, ring_rows, out_elem;
@@ -512,7 +514,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     // the row completed by input row ri is (t0 - (Kh-1)) / s when that is a whole number >= 0
                     const int tf = t0 - (a.Kh - 1);
                     const int of = tf >= 0 ? tf / s : -1;
-                    q[3] = (tf >= 0 && of * s == tf && of < a.done_rel) ? bar_ready + 8u * (uint32_t)(of % nslot) : 0u;
+                    q[3] = (tf >= 0 && of * s == tf && of < a.sched_rel) ? bar_ready + 8u * (uint32_t)(of % nslot) : 0u;
                     // taps ky = ph, ph+s, ... < Kh; those that would reach rows above the map drop out
                     const int cnt = (a.Kh - ph + s - 1) / s;
                     int n_t = cnt;
@@ -638,9 +640,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             umma_commit(bar_empty + 8u * stage);
                             if (row_end) {
                                 // the accumulator this input row completed; on the block's last row also everything still open
+                                // (to be parked in the ring, or emitted if only bottom padding was missing)
                                 if (hdr.w) umma_commit(hdr.w);
                                 if (last_row)
-                                    for (int orel = a.done_rel; orel < a.n_orows; ++orel) umma_commit(bar_ready + 8u * (uint32_t)(orel % nslot));
+                                    for (int orel = a.sched_rel; orel < a.n_orows; ++orel) umma_commit(bar_ready + 8u * (uint32_t)(orel % nslot));
                             }
                         }
                         if (!next_ok && !mbar_wait(bar_full + 8u * nstage_i, nphase, abort_flag)) { ok = false; break; }
@@ -959,7 +962,16 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     t.bias = a.bias; t.ring = a.ring; t.out = a.out; t.status = status;
     t.out_row_stride = a.out_row_stride; t.out_stream_stride = a.out_stream_stride; t.out_row_base = a.out_row_base;
     t.o_begin = a.o_begin; t.r0_positive = a.r0 > 0; t.n_rows = (int)(a.r1 - a.r0); t.n_orows = (int)(a.o_end - a.o_begin);
-    t.done_rel = (int)(a.done_end - a.o_begin); t.base_ty = (int)(a.r0 + a.pad - a.o_begin * a.stride);
+    t.done_rel = (int)(a.done_end - a.o_begin);
+    {
+        // rows whose last tap is a real input row of this block (the others below done_end end on bottom padding)
+        const long long q = a.r1 + a.pad - a.Kh;
+        long long sched = q < 0 ? 0 : q / a.stride + 1;
+        if (sched < a.o_begin) sched = a.o_begin;
+        if (sched > a.done_end) sched = a.done_end;
+        t.sched_rel = (int)(sched - a.o_begin);
+    }
+    t.base_ty = (int)(a.r0 + a.pad - a.o_begin * a.stride);
     t.S = a.S; t.Wout = a.Wout; t.Cout = a.Cout; t.Kh = a.Kh; t.Kw = a.Kw; t.stride = a.stride;
     t.pad_x = a.pad_x; t.relu = a.relu; t.shift = a.shift; t.ring_rows = a.ring_rows; t.out_elem = a.out_elem;
     t.BX = p.BX; t.BS = p.BS; t.n_xt = p.n_xt; t.Ntile = p.Ntile; t.n_nt = p.n_nt; t.KB = p.KB; t.n_kb = p.n_kb;

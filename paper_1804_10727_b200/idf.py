@@ -26,7 +26,7 @@ OK, ERR_ARG, ERR_SPEC, ERR_STATE, ERR_CAPACITY, ERR_UNSUPPORTED, ERR_CUDA, ERR_T
 
 EXPORTS = (
     "idf_net_create", "idf_net_destroy", "idf_net_state_bytes", "idf_net_workspace_bytes", "idf_out_shape",
-    "idf_stream_open", "idf_stream_push", "idf_stream_finish", "idf_run_host", "idf_event_counts",
+    "idf_stream_open", "idf_stream_reset", "idf_stream_push", "idf_stream_push_last", "idf_stream_finish", "idf_run_host", "idf_event_counts",
     "idf_launch_count", "idf_stream_status", "idf_set_timing", "idf_layer_times", "idf_conv_rows_noalloc", "idf_last_error",
 )
 
@@ -63,8 +63,10 @@ def lib():
         L.idf_net_workspace_bytes.argtypes = [vp]; L.idf_net_workspace_bytes.restype = sz
         L.idf_out_shape.argtypes = [vp, ll, ctypes.POINTER(ll), ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
         L.idf_stream_open.argtypes = [vp, vp, sz, vp]
+        L.idf_stream_reset.argtypes = [vp]
         L.idf_stream_push.argtypes = [vp, vp, ctypes.c_int, vp, ll, ctypes.POINTER(ctypes.c_int)]
         L.idf_stream_finish.argtypes = [vp, vp, ll, ctypes.POINTER(ll)]
+        L.idf_stream_push_last.argtypes = [vp, vp, ctypes.c_int, vp, ll, ctypes.POINTER(ll)]
         L.idf_run_host.argtypes = [vp, vp, ctypes.c_int, vp, vp, vp, ll, ctypes.POINTER(ll)]
         L.idf_event_counts.argtypes = [vp, ctypes.POINTER(ll)]
         L.idf_launch_count.argtypes = [vp]; L.idf_launch_count.restype = ll
@@ -192,6 +194,10 @@ class Net:
         st = stream.cuda_stream if stream is not None else torch.cuda.current_stream(workspace.device).cuda_stream
         _check(lib().idf_stream_open(self._h, aligned, nbytes, st))
 
+    def reset(self):
+        """New streams on the workspace of the last open(): state and counters to zero, parameters stay."""
+        _check(lib().idf_stream_reset(self._h))
+
     def alloc_out(self, in_rows: int, device="cuda:0") -> torch.Tensor:
         r, w, c = self.out_shape(in_rows)
         return torch.zeros((self.n_streams, max(r, 1), w, c), dtype=self.out_torch_dtype, device=device)
@@ -205,6 +211,16 @@ class Net:
         _check(lib().idf_stream_push(self._h, segments.data_ptr(), segments.shape[0], out.data_ptr(), out.shape[1],
                                      ctypes.byref(em)))
         return int(em.value)
+
+    def push_last(self, segments: torch.Tensor, out: torch.Tensor) -> int:
+        """The last segments and the end of input in one call; returns the total number of output rows."""
+        assert segments.is_cuda and segments.is_contiguous() and out.is_cuda and out.is_contiguous()
+        assert segments.dtype == self.act_torch_dtype and out.dtype == self.out_torch_dtype
+        assert tuple(segments.shape[1:]) == (self.n_streams, self.in_w, self.in_c), segments.shape
+        tot = ctypes.c_longlong()
+        _check(lib().idf_stream_push_last(self._h, segments.data_ptr(), segments.shape[0], out.data_ptr(), out.shape[1],
+                                          ctypes.byref(tot)))
+        return int(tot.value)
 
     def finish(self, out: torch.Tensor) -> int:
         tot = ctypes.c_longlong()
@@ -246,22 +262,31 @@ def net_from_workload(w, weights, biases, n_streams: Optional[int] = None, row_b
     return Net(w.dtype, w.layers, w.W, w.C, n_streams or w.n_streams, weights, biases, row_block=row_block)
 
 
-def infer(net: Net, x: np.ndarray, chunks: Optional[Sequence[int]] = None, device="cuda:0") -> np.ndarray:
+def infer(net: Net, x: np.ndarray, chunks: Optional[Sequence[int]] = None, device="cuda:0", last: bool = False) -> np.ndarray:
     """Run whole maps x [n_streams][H][W][C] through the net; ``chunks`` gives the number of
-    segments per push (default: one push).  Returns the output map as a numpy array."""
+    segments per push (default: one push).  With ``last`` the final group of segments and the end
+    of input go through ``push_last`` instead of ``push`` + ``finish``.  Returns the output map as
+    a numpy array."""
     seg = segments_from_maps(x, net.dtype).to(device)
     H = seg.shape[0]
     out = net.alloc_out(H, device)
     net.open(device)
-    pos = 0
+    groups, pos = [], 0
     for n in (chunks or [H]):
         n = min(n, H - pos)
         if n > 0:
-            net.push(seg[pos:pos + n], out)
+            groups.append((pos, pos + n))
         pos += n
     if pos < H:
-        net.push(seg[pos:], out)
-    rows = net.finish(out)
+        groups.append((pos, H))
+    rows = None
+    for k, (a, b) in enumerate(groups):
+        if last and k == len(groups) - 1:
+            rows = net.push_last(seg[a:b], out)
+        else:
+            net.push(seg[a:b], out)
+    if rows is None:
+        rows = net.finish(out)
     net.status()
     torch.cuda.synchronize()
     assert rows == net.out_shape(H)[0], (rows, net.out_shape(H))

@@ -1,5 +1,5 @@
 """Parity at the workloads' full sizes, in the launch configuration bench.py times (all streams of
-the batch, one push + finish with the default row block).  Streams are independent, so the oracle
+the batch, all segments and the end of input in one push_last with the default row block).  Streams are independent, so the oracle
 is run only on a sample of streams and compared with exactly those streams of the device result;
 the rest is covered by properties that hold at any size (shape, finiteness, batch-mate independence)."""
 import numpy as np
@@ -26,8 +26,7 @@ def test_full_size_sampled_streams_match_oracle(orc, name, sample):
     seg = idf.segments_from_maps(x, w.dtype).cuda()
     out = net.alloc_out(w.H)
     net.open()
-    net.push(seg, out)
-    rows = net.finish(out)
+    rows = net.push_last(seg, out)
     tc = net.status()
     assert rows == net.out_shape(w.H)[0]
     got_all = out[:, :rows]

@@ -105,6 +105,8 @@ def test_bad_arguments_and_call_order():
     # push / finish before open: refused on the host, nothing is enqueued
     assert L.idf_stream_push(net._h, 256, 1, 256, 4, ctypes.byref(em)) == idf.ERR_STATE
     assert L.idf_stream_finish(net._h, 256, 4, None) == idf.ERR_STATE
+    assert L.idf_stream_push_last(net._h, 256, 1, 256, 4, None) == idf.ERR_STATE
+    assert L.idf_stream_reset(net._h) == idf.ERR_STATE
     assert b"before stream_open" in L.idf_last_error()
     assert L.idf_stream_open(net._h, None, 0, None) == idf.ERR_ARG
     assert L.idf_stream_open(net._h, 256, 16, None) == idf.ERR_CAPACITY

@@ -11,11 +11,11 @@ from helpers import (SMALL_NETS, assert_close, assert_equal, rand_net, small_dim
 pytestmark = pytest.mark.gpu
 
 
-def _run(mode, layers, x, ws, bs, chunks=None, row_block=0):
+def _run(mode, layers, x, ws, bs, chunks=None, row_block=0, last=False):
     S, H, W, C = x.shape
     net = idf.Net(mode, layers, W, C, S, ws, bs, row_block=row_block)
     try:
-        return idf.infer(net, x, chunks=chunks), net
+        return idf.infer(net, x, chunks=chunks, last=last), net
     finally:
         pass
 
@@ -59,6 +59,57 @@ def test_small_nets_match_oracle(orc, name, mode):
     for chunks, rb in ((None, 0), ([1] * H, 0), (_random_chunks(H, 1), 3), (None, 1), ([H], 64)):
         got, _ = _run(mode, layers, x, ws, bs, chunks=chunks, row_block=rb)
         _compare(mode, got, want, f"{name}/{mode}/chunks={chunks and len(chunks)}/rb={rb}")
+
+
+# ---- the end of input given with the last segments (push_last) equals push + finish -------------
+@pytest.mark.parametrize("name", list(SMALL_NETS))
+@pytest.mark.parametrize("mode", ["f32", "i8"])
+def test_push_last_equals_push_then_finish(orc, name, mode):
+    layers = SMALL_NETS[name]
+    if mode == "i8":
+        layers = with_shifts(layers, 8)
+    H, W = small_dims(name)
+    C0 = next(l.cin for l in layers if l.kind == "conv")
+    x, ws, bs = rand_net(mode, layers, H, W, C0, S=4, seed=7 + len(name))
+    want = orc.forward(mode, layers, x, ws, bs)
+    for chunks, rb in ((None, 0), ([H - 1], 0), (_random_chunks(H, 2), 3), ([1] * H, 1), (None, 2)):
+        got, _ = _run(mode, layers, x, ws, bs, chunks=chunks, row_block=rb, last=True)
+        _compare(mode, got, want, f"push_last {name}/{mode}/chunks={chunks and len(chunks)}/rb={rb}")
+
+
+def test_push_last_on_tensor_core_layers_matches_oracle(orc):
+    # same-padded dense int8 layers wide enough for the tensor-core kernel: the rows that end on bottom
+    # padding are completed by the launch that applies the last input rows
+    layers = with_shifts((conv(16, 32, 3, pad=1), conv(32, 32, 3, pad=1), POOL, conv(32, 16, 3, pad=1)), 8)
+    x, ws, bs = rand_net("i8", layers, 21, 40, 16, S=5, seed=11)
+    want = orc.forward("i8", layers, x, ws, bs)
+    for chunks, rb in ((None, 0), ([20], 0), ([7, 7], 4), (None, 5)):
+        got, net = _run("i8", layers, x, ws, bs, chunks=chunks, row_block=rb, last=True)
+        assert_equal(got, want, f"push_last tc chunks={chunks} rb={rb}")
+        assert any(t > 0 for t in net.status()), "no layer took the tensor-core path"
+    net = idf.Net("i8", layers, 40, 16, 5, ws, bs)
+    seg = idf.segments_from_maps(x, "i8").cuda()
+    out = net.alloc_out(21)
+    net.open()
+    assert net.push_last(seg, out) == want.shape[1]
+    with pytest.raises(idf.IdfError) as e:                      # the stream has ended
+        net.push(seg, out)
+    assert e.value.code == idf.ERR_STATE
+    net.open()
+    net.push(seg, out)
+    assert net.push_last(seg[:0], out) == want.shape[1]         # no segments: the same as finish
+    assert_equal(out.cpu().numpy(), want, "push + empty push_last")
+    out.zero_()
+    net.reset()                                                 # new streams, parameters kept
+    assert net.push_last(seg, out) == want.shape[1]
+    assert_equal(out.cpu().numpy(), want, "reset + push_last")
+    net.reset()
+    net.push(seg[:9], out)                                      # abandoned half way ...
+    net.reset()                                                 # ... and started again
+    out.zero_()
+    net.push(seg[:13], out)
+    net.push_last(seg[13:], out)
+    assert_equal(out.cpu().numpy(), want, "reset in the middle of streams")
 
 
 @pytest.mark.parametrize("mode", ["f32", "i8"])
