@@ -41,6 +41,8 @@ struct LayerPlan {
     std::vector<unsigned char> wtc_packed;  // [tap][Cout][Cin] in the activation type
     size_t wtc_off = 0;
     alignas(64) unsigned char w_map[128];   // TMA descriptor of wtc in the workspace (made at open)
+    TcPlan tc_pool;                         // plan of the launches that also emit the following max-pool's rows
+    alignas(64) unsigned char w_map_pool[128];
     long long tc_launches = 0;
     // x-unfold in front of the tensor-core kernel (thin or x-strided layers): the Kw taps of every
     // output position are laid side by side as kpad channels, the conv then has Kw = 1, stride_x = 1
@@ -58,6 +60,7 @@ struct LayerPlan {
     long long rows_in = 0, rows_done = 0;
     long long pending = 0;                 // rows waiting in this layer's input buffer
     int fire_rows = 0;                     // the layer runs once this many rows wait (or when a push ends)
+    int fuse_pool = 0;                     // conv layer whose tensor-core launch may emit the following 2x2 max-pool's rows
 };
 
 enum Phase { CREATED = 0, OPEN = 1, FINISHED = 2 };
@@ -222,6 +225,91 @@ int launch_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, boo
     return IDF_OK;
 }
 
+// A conv layer followed by a 2x2 max-pool, as ONE tensor-core launch that emits the pooled rows (into the
+// buffer behind the pool layer, or the caller's output).  Both layers' row counters advance as if the
+// two had run one after the other; a trailing unpaired row waits x-pooled in the pool layer's state,
+// exactly as the stand-alone pool kernel leaves it, so fused and unfused launches may alternate.
+// Returns 1 (no row counter changed) when this launch cannot take the fused path.
+int launch_conv_pool(idf_net* net, size_t i, const void* in_ptr, long long n_in, bool flush, void* final_out,
+                     long long out_cap, long long out_slot, long long* n_out_p)
+{
+    LayerPlan& P = net->L[i];
+    LayerPlan& Q = net->L[i + 1];
+    const bool last = (i + 2 == net->L.size());
+    if (!P.fuse_pool || !P.tc_pool.ok || n_in <= 0 || (P.unfold && n_in > P.in_cap_rows) || Q.rows_in != P.rows_done) return 1;
+    const long long r0 = P.rows_in, r1 = r0 + n_in;
+    long long done_end = flush ? conv_rows_at_flush(P.l, r1) : conv_done_after(P.l, r1);
+    const long long started = (r1 - 1 + P.l.pad) / P.l.stride + 1;
+    const long long o_begin = P.rows_done;
+    if (done_end < o_begin) done_end = o_begin;
+    const long long o_end = std::max(started, done_end);
+    const long long q_begin = Q.rows_done, q_done = done_end / 2;
+    const long long n_out = q_done - q_begin;
+    if (last && q_done > out_cap)
+        return fail(IDF_ERR_CAPACITY, "output row %lld does not fit out_capacity_rows=%lld", q_done - 1, out_cap);
+    if (!last && n_out + out_slot > Q.out_cap_rows)
+        return fail(IDF_ERR_CAPACITY, "internal: layer %zu emits %lld rows at slot %lld of a %d-row buffer", i + 1, n_out,
+                    out_slot, Q.out_cap_rows);
+    const long long S = net->n_streams;
+    ConvArgs a{};
+    a.in = in_ptr;
+    a.w = net->ws + P.w_off;
+    a.bias = P.b_packed.empty() ? nullptr : net->ws + P.b_off;
+    a.ring = net->ws + P.state_off;
+    if (last) {
+        a.out = final_out;
+        a.out_row_stride = (long long)Q.out_w * Q.out_c;
+        a.out_stream_stride = out_cap * a.out_row_stride;
+        a.out_row_base = 0;
+        a.out_rows_extent = out_cap;
+    } else {
+        a.out = net->ws + Q.out_off;
+        a.out_stream_stride = (long long)Q.out_w * Q.out_c;
+        a.out_row_stride = S * a.out_stream_stride;
+        a.out_row_base = q_begin - out_slot;
+        a.out_rows_extent = Q.out_cap_rows;
+    }
+    a.event_counter = (unsigned long long*)(net->ws + net->counters_off) + i;
+    a.S = (int)S; a.Win = P.in_w; a.Wout = P.out_w; a.Cin = P.in_c; a.Cout = P.out_c;
+    a.Kh = P.l.kh; a.Kw = P.l.kw; a.stride = P.l.stride; a.pad = P.l.pad; a.relu = P.l.relu; a.shift = P.l.shift;
+    a.stride_x = P.l.stride; a.pad_x = P.l.pad;
+    a.ring_rows = P.ring_rows; a.in_elem = P.in_elem; a.out_elem = P.out_elem;
+    a.r0 = r0; a.r1 = r1; a.o_begin = o_begin; a.o_end = o_end; a.done_end = done_end;
+    a.pool_fused = 1; a.pool_keep = flush ? 0 : 1; a.pool_state = net->ws + Q.state_off;
+    if (a.out_rows_extent < 1) return 1;
+    cudaEvent_t ev_a = nullptr, ev_b = nullptr;
+    if (net->timing) {
+        for (cudaEvent_t* e : {&ev_a, &ev_b}) {
+            if (!net->event_pool.empty()) { *e = net->event_pool.back(); net->event_pool.pop_back(); }
+            else if (cudaEventCreate(e) != cudaSuccess) return fail(IDF_ERR_CUDA, "cudaEventCreate failed");
+        }
+        cudaEventRecord(ev_a, net->stream);
+    }
+    cudaError_t ce;
+    ConvArgs t = a;
+    if (P.unfold) {
+        // (if the conv launch below declines, this pass has only filled its own buffer: harmless)
+        ce = launch_unfold(a, (int)n_in, P.kpad, net->ws + P.unf_off, net->stream);
+        if (ce != cudaSuccess) return fail(IDF_ERR_CUDA, "kernel launch failed at layer %zu: %s", i, cudaGetErrorString(ce));
+        net->launches += 1;
+        t.in = net->ws + P.unf_off;
+        t.Win = a.Wout; t.Cin = P.kpad; t.Kw = 1; t.stride_x = 1; t.pad_x = 0;
+    }
+    ce = launch_conv_tc(t, P.tc_pool, net->dtype, P.w_map_pool, (int)n_in, (unsigned int*)(net->ws + net->status_off), net->stream);
+    if (net->timing) {
+        cudaEventRecord(ev_b, net->stream);
+        net->timed.push_back({(int)i, ev_a, ev_b});
+    }
+    if (ce == cudaErrorNotSupported) return 1;
+    if (ce != cudaSuccess) return fail(IDF_ERR_CUDA, "kernel launch failed at layer %zu: %s", i, cudaGetErrorString(ce));
+    net->launches += 1;
+    P.tc_launches += 1;
+    P.rows_in = r1; P.rows_done = done_end;
+    Q.rows_in = done_end; Q.rows_done = q_done;
+    *n_out_p = n_out;
+    return IDF_OK;
+}
+
 // Depth-first schedule.  Rows a layer emits wait in the next layer's buffer; that layer runs ("fires")
 // once a block's worth of rows (fire_rows) has gathered, when a push ends, or when its buffer could not
 // take what is about to arrive.  So a pooled, narrower layer runs less often on as many rows, and a
@@ -244,6 +332,24 @@ int fire(idf_net* net, size_t i, const void* in_ptr, long long n_in, bool flush,
     const long long r1 = P.rows_in + n_in;
     const long long n1 = std::max(0LL, layer_done_after(P, r1) - P.rows_done);
     const long long n2 = flush ? std::max(0LL, layer_rows_at_flush(P, r1) - std::max(P.rows_done, layer_done_after(P, r1))) : 0;
+    if (P.fuse_pool && n_in > 0 && net->L[i + 1].pending == 0 && net->L[i + 1].rows_in == P.rows_done) {
+        // conv + pool in one launch: the pooled rows go straight to the buffer behind the pool layer
+        LayerPlan& Q = net->L[i + 1];
+        const bool qlast = (i + 2 == net->L.size());
+        const long long n_pool = (P.rows_done + n1 + n2) / 2 - Q.rows_done;
+        if (!qlast) {
+            int rc = ensure_space(net, i + 2, n_pool, d_out, out_cap, emitted);
+            if (rc != IDF_OK) return rc;
+        }
+        long long got = 0;
+        int rc = launch_conv_pool(net, i, in_ptr, n_in, flush, d_out, out_cap, qlast ? 0 : net->L[i + 2].pending, &got);
+        if (rc < 0) return rc;
+        if (rc == IDF_OK) {
+            if (i > 0) P.pending = 0;
+            if (qlast) *emitted += got; else net->L[i + 2].pending += got;
+            return IDF_OK;
+        }
+    }
     if (!last) {
         int rc = ensure_space(net, i + 1, n1 + n2, d_out, out_cap, emitted);
         if (rc != IDF_OK) return rc;
@@ -393,8 +499,12 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
             const bool tc_allowed = !P.use_sparse && !(no_tc && no_tc[0] == '1') && spec->dtype != IDF_F32;
             const size_t es = spec->dtype == IDF_I8_I32 ? 1 : 2;
             const int taps = l.kh * l.kw;
+            const bool pool_next = i + 1 < spec->n_layers && spec->layers[i + 1].kind == IDF_MAXPOOL2;
             if (tc_allowed && tc_make_plan(spec->dtype, net->n_streams, w, P.out_w, l.cin, l.cout, l.kh, l.kw,
-                                           w == 1 ? 1 : l.stride, P.ring_rows, (int)elem_size(P.out_elem), &P.tc)) {
+                                           w == 1 ? 1 : l.stride, P.ring_rows, (int)elem_size(P.out_elem), 0, &P.tc)) {
+                if (pool_next)
+                    tc_make_plan(spec->dtype, net->n_streams, w, P.out_w, l.cin, l.cout, l.kh, l.kw, w == 1 ? 1 : l.stride,
+                                 P.ring_rows, (int)elem_size(P.out_elem), 1, &P.tc_pool);
                 P.wtc_packed.resize(nw * es);
                 for (int co = 0; co < l.cout; ++co)
                     for (int k = 0; k < taps; ++k)
@@ -407,7 +517,10 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
                 const int kpad = (int)(padded / es);
                 if (padded <= 1024 &&
                     tc_make_plan(spec->dtype, net->n_streams, P.out_w, P.out_w, kpad, l.cout, l.kh, 1, 1, P.ring_rows,
-                                 (int)elem_size(P.out_elem), &P.tc)) {
+                                 (int)elem_size(P.out_elem), 0, &P.tc)) {
+                    if (pool_next)
+                        tc_make_plan(spec->dtype, net->n_streams, P.out_w, P.out_w, kpad, l.cout, l.kh, 1, 1, P.ring_rows,
+                                     (int)elem_size(P.out_elem), 1, &P.tc_pool);
                     P.unfold = 1;
                     P.kpad = kpad;
                     P.in_cap_rows = in_cap;
@@ -441,6 +554,15 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
         P.state_bytes_all = P.state_bytes_stream * (size_t)net->n_streams;
         net->state_bytes_stream += P.state_bytes_stream;
         w = P.out_w; c = P.out_c; elem = P.out_elem;
+    }
+    // a dense tensor-core conv layer directly followed by a 2x2 max-pool emits the pooled rows itself
+    {
+        const char* no_fuse = getenv("IDF_NO_POOL_FUSION");
+        for (size_t i = 0; i + 1 < net->L.size(); ++i) {
+            LayerPlan& P = net->L[i];
+            P.fuse_pool = P.l.kind == IDF_CONV && net->L[i + 1].l.kind == IDF_MAXPOOL2 && P.tc.ok && P.tc_pool.ok && !P.use_sparse &&
+                          P.out_w >= 2 && (P.tc_pool.BX % 2) == 0 && !(no_fuse && no_fuse[0] == '1');
+        }
     }
     // workspace: [parameters][state of all streams][rows travelling between layers][counters]
     size_t off = 0;
@@ -516,6 +638,9 @@ int idf_stream_open(idf_net* net, void* d_workspace, size_t workspace_bytes, voi
             if (tc_encode_weights(P.tc, net->dtype, net->ws + P.wtc_off, P.unfold ? P.l.kh : P.l.kh * P.l.kw,
                                   P.unfold ? P.kpad : P.l.cin, P.l.cout, P.w_map) != 0)
                 P.tc.ok = 0;               // no TMA descriptor: this layer stays on the CUDA-core kernel
+            if (P.tc_pool.ok && tc_encode_weights(P.tc_pool, net->dtype, net->ws + P.wtc_off, P.unfold ? P.l.kh : P.l.kh * P.l.kw,
+                                                  P.unfold ? P.kpad : P.l.cin, P.l.cout, P.w_map_pool) != 0)
+                P.tc_pool.ok = 0;
         }
     }
     if (e != cudaSuccess) { net->phase = CREATED; return fail(IDF_ERR_CUDA, "stream_open: %s", cudaGetErrorString(e)); }

@@ -34,6 +34,11 @@ struct ConvArgs {
     long long r0, r1;      // input rows [r0, r1) arrive in this block
     long long o_begin, o_end;  // output rows [o_begin, o_end) are visited
     long long done_end;    // rows o < done_end are complete after this block: emit them, free their slots
+    // Tensor-core kernel only: 2x2 max-pooling folded into the emission.  `out` and its strides, row base and
+    // row extent then describe the POOLED rows (pooled row p = o / 2 goes to p - out_row_base).
+    int pool_fused;        // 1: emit pooled rows
+    int pool_keep;         // 1: more input may follow (a trailing first row of a pair waits in pool_state); 0: end of input
+    void* pool_state;      // the pool layer's state: [S][Wout/2][Cout] in the output type
 };
 
 struct PoolArgs {
@@ -61,11 +66,12 @@ struct TcPlan {
     int tmem_cols = 0;
     int out_groups = 0;
     int out_esize = 0, out_pwb = 0, out_panels = 0, out_stage_bytes = 0;   // staging of emitted rows for the TMA store
+    int out_stage_rows = 0;  // rows of one staging panel: 128, or 64 in a plan for launches that emit pooled rows
     size_t smem_bytes = 0;
     size_t w_bytes = 0;      // device weights for this path: [tap][Cout][Cin] in the activation type
 };
 bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh, int Kw, int stride_x, int ring_rows,
-                  int out_esize, TcPlan* p);
+                  int out_esize, int pooled, TcPlan* p);
 int tc_encode_weights(const TcPlan& p, int dtype, const void* d_w, int taps, int Cin, int Cout, void* map_out);
 cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const void* w_map, int n_in_rows,
                            unsigned int* status, cudaStream_t st);

@@ -28,7 +28,7 @@ namespace idf {
 
 namespace {
 
-constexpr int MAX_GROUPS = 4;                // epilogue groups (four warps each) taking output rows in turn
+constexpr int MAX_GROUPS = 3;                // epilogue groups (four warps each) taking output rows in turn
 constexpr int TC_THREADS = 64 + 128 * MAX_GROUPS;
 constexpr int ROWQ = 64;                     // row-schedule queue: two chunks of 32 rows
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
@@ -258,7 +258,7 @@ __device__ __forceinline__ void tmem_st_zero(uint32_t taddr)
 // the swizzle the output tensor map expects, from which one thread sends it out with a TMA store.
 struct StageSink {
     uint32_t row_base;     // shared address of this thread's tile row in panel 0
-    uint32_t panel_bytes;  // bytes of one panel (128 rows * pwb)
+    uint32_t panel_bytes;  // bytes of one panel (staged rows * pwb)
     uint32_t pwb_log2;     // log2(panel row bytes)
     uint32_t phase;        // swizzle phase of this row (XORed into the 16-byte chunk index)
 };
@@ -268,6 +268,63 @@ __device__ __forceinline__ void stage_store16(const StageSink& k, uint32_t col_b
     const uint32_t within = col_byte & ((1u << k.pwb_log2) - 1u);
     const uint32_t addr = k.row_base + panel * k.panel_bytes + ((((within >> 4) ^ k.phase)) << 4);
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ int4 stage_load16(const StageSink& k, uint32_t col_byte)
+{
+    const uint32_t panel = col_byte >> k.pwb_log2;
+    const uint32_t within = col_byte & ((1u << k.pwb_log2) - 1u);
+    const uint32_t addr = k.row_base + panel * k.panel_bytes + ((((within >> 4) ^ k.phase)) << 4);
+    int4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+// element-wise maximum of two 32-bit words holding OP = 0: two bf16, 1: one fp32, 2: four int8
+template <int OP>
+__device__ __forceinline__ uint32_t word_max(uint32_t x, uint32_t y)
+{
+    if (OP == 0) { uint32_t r; asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(y)); return r; }
+    if (OP == 1) return __float_as_uint(fmaxf(__uint_as_float(x), __uint_as_float(y)));
+    return __vmaxs4(x, y);
+}
+// 2x2 max-pooling folded into the emission of a conv layer's rows.  A thread owns one (stream, x)
+// position; its x neighbour is the next lane.  The x-pooled first row of a pair waits in the group's
+// staging tile (or, across launches, in the pool layer's state in global memory) until the second
+// row arrives; the pooled row then leaves through the TMA store.
+struct PoolCtx {
+    int on;            // pooling is folded into this launch
+    int writer;        // this thread holds the pooled value of an in-tile position (even x)
+    int second;        // the row at hand is the second of its pair
+    int from_state;    // ... and the first one was emitted by an earlier launch
+    int to_state;      // the row at hand is a first row whose partner comes with a later launch
+    int drop;          // a first row at the end of input: never completed, nothing is kept
+    StageSink sink;    // pooled tile (half the positions)
+    unsigned char* state;   // this thread's pooled position in the pool layer's state, at the CTA's first channel
+};
+template <int NW, int OP>
+__device__ __forceinline__ void deliver(uint32_t (&ow)[NW], const StageSink& sink, uint32_t col_byte, const PoolCtx& pc, bool state_ok)
+{
+    if (!pc.on) {
+#pragma unroll
+        for (int j4 = 0; j4 < NW / 4; ++j4)
+            stage_store16(sink, col_byte + 16u * j4, make_int4((int)ow[4 * j4], (int)ow[4 * j4 + 1], (int)ow[4 * j4 + 2], (int)ow[4 * j4 + 3]));
+        return;
+    }
+#pragma unroll
+    for (int j = 0; j < NW; ++j) ow[j] = word_max<OP>(ow[j], __shfl_xor_sync(0xffffffffu, ow[j], 1));
+    if (!pc.writer || pc.drop) return;
+#pragma unroll
+    for (int j4 = 0; j4 < NW / 4; ++j4) {
+        int4 v = make_int4((int)ow[4 * j4], (int)ow[4 * j4 + 1], (int)ow[4 * j4 + 2], (int)ow[4 * j4 + 3]);
+        if (pc.second) {
+            int4 h = make_int4(0, 0, 0, 0);
+            if (!pc.from_state) h = stage_load16(pc.sink, col_byte + 16u * j4);
+            else if (state_ok) h = *(const int4*)(pc.state + col_byte + 16u * j4);
+            v.x = (int)word_max<OP>((uint32_t)v.x, (uint32_t)h.x); v.y = (int)word_max<OP>((uint32_t)v.y, (uint32_t)h.y);
+            v.z = (int)word_max<OP>((uint32_t)v.z, (uint32_t)h.z); v.w = (int)word_max<OP>((uint32_t)v.w, (uint32_t)h.w);
+        }
+        if (pc.to_state) { if (state_ok) *(int4*)(pc.state + col_byte + 16u * j4) = v; }
+        else stage_store16(pc.sink, col_byte + 16u * j4, v);
+    }
 }
 __device__ __forceinline__ void tma_store_4d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2, int c3)
 {
@@ -295,7 +352,7 @@ __device__ __forceinline__ bool named_bar_and(int id, int count, bool pred)
 template <int DT, int W, typename TS>
 __device__ __forceinline__ void finalise_chunk(const uint32_t (&v)[W], bool carried_in, bool emit, TS* rp,
                                                const TS* bias_c, const StageSink& sink, uint32_t col_byte, int out_elem,
-                                               int relu, int shift)
+                                               int relu, int shift, const PoolCtx& pc, bool state_ok)
 {
     TS acc[W];
 #pragma unroll
@@ -353,36 +410,31 @@ __device__ __forceinline__ void finalise_chunk(const uint32_t (&v)[W], bool carr
                 for (int j = 0; j < W / 2; ++j)
                     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk[j]) : "f"(f[2 * j + 1]), "f"(f[2 * j]));
             }
-#pragma unroll
-            for (int j8 = 0; j8 < W / 8; ++j8)
-                stage_store16(sink, col_byte + 16u * j8,
-                              make_int4((int)pk[4 * j8], (int)pk[4 * j8 + 1], (int)pk[4 * j8 + 2], (int)pk[4 * j8 + 3]));
+            deliver<W / 2, 0>(pk, sink, col_byte, pc, state_ok);
         } else {
             if (relu) {
 #pragma unroll
                 for (int j = 0; j < W; ++j) f[j] = fmaxf(f[j], 0.f);
             }
+            uint32_t fw[W];
 #pragma unroll
-            for (int j4 = 0; j4 < W / 4; ++j4)
-                stage_store16(sink, col_byte + 16u * j4,
-                              make_int4(__float_as_int(f[4 * j4]), __float_as_int(f[4 * j4 + 1]), __float_as_int(f[4 * j4 + 2]),
-                                        __float_as_int(f[4 * j4 + 3])));
+            for (int j = 0; j < W; ++j) fw[j] = __float_as_uint(f[j]);
+            deliver<W, 1>(fw, sink, col_byte, pc, state_ok);
         }
     } else {
         const int lo = relu ? 0 : -127;
+        uint32_t pk[W / 4];
 #pragma unroll
-        for (int j16 = 0; j16 < W / 16; ++j16) {
-            uint32_t pk[4] = {0, 0, 0, 0};
+        for (int j = 0; j < W / 4; ++j) pk[j] = 0;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                int t = (int)acc[16 * j16 + j] + (bias_c ? (int)bias_c[16 * j16 + j] : 0);
-                if (relu && t < 0) t = 0;
-                if (shift > 0) t = (t + (1 << (shift - 1))) >> shift;
-                t = t < lo ? lo : (t > 127 ? 127 : t);
-                pk[j >> 2] |= ((uint32_t)t & 0xffu) << (8 * (j & 3));
-            }
-            stage_store16(sink, col_byte + 16u * j16, make_int4((int)pk[0], (int)pk[1], (int)pk[2], (int)pk[3]));
+        for (int j = 0; j < W; ++j) {
+            int t = (int)acc[j] + (bias_c ? (int)bias_c[j] : 0);
+            if (relu && t < 0) t = 0;
+            if (shift > 0) t = (t + (1 << (shift - 1))) >> shift;
+            t = t < lo ? lo : (t > 127 ? 127 : t);
+            pk[j >> 2] |= ((uint32_t)t & 0xffu) << (8 * (j & 3));
         }
+        deliver<W / 4, 2>(pk, sink, col_byte, pc, state_ok);
     }
 }
 
@@ -406,9 +458,15 @@ struct TcArgs {
     int shift_mode;              // 1: one box per (row, K block) holds the kx halo, taps address it at row offsets
     int a_stage_bytes;
     int out_esize, out_pwb, out_panels, out_stage_bytes;   // emitted rows: staging panels of out_pwb-byte rows
+    int out_stage_rows;          // rows of one staging panel: 128, or 64 when only pooled rows are staged
     int out_groups;              // epilogue groups at work (1 or 2), each with its own staging tile
     int out_row_dim;             // position of the row coordinate in the output tensor map (2 or 3)
     int out_row_first;           // tensor-map row index of relative output row 0
+    // 2x2 max-pooling folded into the emission (the output tensor map then describes the pooled rows)
+    int pool;                    // 1: emit pooled rows
+    int pool_keep;               // 1: a trailing first row of a pair waits in pool_state for a later launch; 0: end of input, it is dropped
+    void* pool_state;            // [S][Wout/2][Cout] in the output type: x-pooled first row of an open pair
+    long long pool_row_base;     // pooled row p goes to tensor-map row p - pool_row_base
 };
 
 template <int DT> struct Acc;
@@ -679,12 +737,23 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int md = bs * a.BX + bx;                   // row of the dense output tile
         StageSink sink;
         sink.pwb_log2 = 31u - (uint32_t)__clz(a.out_pwb);
-        sink.panel_bytes = 128u * (uint32_t)a.out_pwb;
+        sink.panel_bytes = (uint32_t)a.out_stage_rows * (uint32_t)a.out_pwb;
         sink.row_base = sOut + (uint32_t)grp * a.out_stage_bytes + (uint32_t)md * a.out_pwb;
         sink.phase = a.out_pwb == 128 ? (uint32_t)(md & 7) : (a.out_pwb == 64 ? (uint32_t)((md >> 1) & 3)
                    : (a.out_pwb == 32 ? (uint32_t)((md >> 2) & 1) : 0u));
         const uint32_t stg = sOut + (uint32_t)grp * a.out_stage_bytes;
         const int panel_cols = a.out_pwb / a.out_esize;
+        PoolCtx pc;
+        pc.on = a.pool; pc.second = 0; pc.from_state = 0; pc.to_state = 0; pc.drop = 0;
+        pc.writer = in_tile && !(bx & 1);
+        const int mdp = bs * (a.BX >> 1) + (bx >> 1);   // row of the pooled tile
+        pc.sink = sink;
+        pc.sink.row_base = stg + (uint32_t)mdp * a.out_pwb;
+        pc.sink.phase = a.out_pwb == 128 ? (uint32_t)(mdp & 7) : (a.out_pwb == 64 ? (uint32_t)((mdp >> 1) & 3)
+                      : (a.out_pwb == 32 ? (uint32_t)((mdp >> 2) & 1) : 0u));
+        const int wp = a.Wout >> 1;
+        const bool state_ok = valid && (x >> 1) < wp;
+        pc.state = (unsigned char*)a.pool_state + (((long long)s * wp + (x >> 1)) * a.Cout + n0) * a.out_esize;
         bool ok = true;
         // every ring slot in tensor memory starts at zero (all MMAs accumulate)
         if (grp == 0)
@@ -700,7 +769,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // slot is read before it is rewritten.  The other rows go round the groups.
         const int n_cin = a.r0_positive ? (a.base_ty + a.stride - 1) / a.stride : 0;
         for (int orel = 0; orel < a.n_orows && ok && grp < a.out_groups; ++orel) {
-            const int owner = (orel < n_cin || orel >= a.done_rel) ? 0 : orel % a.out_groups;
+            int owner;
+            if (!a.pool) {
+                owner = (orel < n_cin || orel >= a.done_rel) ? 0 : orel % a.out_groups;
+            } else {
+                // both rows of a pooling pair go to one group; pairs touching the global ring go to group 0
+                const int first = orel - (int)((a.o_begin + orel) & 1);
+                owner = (first < n_cin || first + 1 >= a.done_rel) ? 0 : (int)(((a.o_begin + orel) >> 1) % a.out_groups);
+            }
             if (owner != grp) continue;
             const int slot = orel % a.nslot;
             const uint32_t par = (uint32_t)((orel / a.nslot) & 1);
@@ -714,6 +790,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (!named_bar_and(1 + grp, 128, got != 0)) { ok = false; break; }
             tc_fence_after();
             const bool carried_in = a.r0_positive && (orel * a.stride - a.base_ty < 0);
+            const bool pool_emit = a.pool && emit;
+            if (pool_emit) {
+                pc.second = (int)((a.o_begin + orel) & 1);
+                pc.from_state = pc.second && orel == 0;
+                const bool trailing = !pc.second && orel == a.done_rel - 1;
+                pc.to_state = trailing && a.pool_keep;
+                pc.drop = trailing && !a.pool_keep;
+            }
             TS* rp = ring_pos + (long long)((a.o_begin + orel) % a.ring_rows) * ring_slot_stride;
             const uint32_t trow = tlane + (uint32_t)(slot * a.Ntile);
             if (a.Ntile == 64 || a.Ntile == 32) {
@@ -727,11 +811,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_free + 8u * slot);   // one arrival per warp
-                if (emit ? in_tile : valid) {
-                    finalise_chunk<DT, 32, TS>(v0, carried_in && valid, emit, rp, bias, sink, 0u, a.out_elem, a.relu, a.shift);
+                if (pool_emit || (emit ? in_tile : valid)) {
+                    finalise_chunk<DT, 32, TS>(v0, carried_in && valid, emit, rp, bias, sink, 0u, a.out_elem, a.relu, a.shift, pc, state_ok);
                     if (a.Ntile == 64)
                         finalise_chunk<DT, 32, TS>(v1, carried_in && valid, emit, rp + 32, bias ? bias + 32 : nullptr, sink,
-                                                   (uint32_t)(32 * a.out_esize), a.out_elem, a.relu, a.shift);
+                                                   (uint32_t)(32 * a.out_esize), a.out_elem, a.relu, a.shift, pc, state_ok);
                 }
             } else {
                 if (wide) {
@@ -739,18 +823,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         uint32_t v[32];
                         tmem_ld<32>(trow + c, v);
                         tmem_st_zero<32>(trow + c);           // the slot's next row starts from zero
-                        if (emit ? in_tile : valid)
+                        if (pool_emit || (emit ? in_tile : valid))
                             finalise_chunk<DT, 32, TS>(v, carried_in && valid, emit, rp + c, bias ? bias + c : nullptr, sink,
-                                                       (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift);
+                                                       (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift, pc, state_ok);
                     }
                 } else {
                     for (int c = 0; c < a.Ntile; c += 16) {
                         uint32_t v[16];
                         tmem_ld<16>(trow + c, v);
                         tmem_st_zero<16>(trow + c);
-                        if (emit ? in_tile : valid)
+                        if (pool_emit || (emit ? in_tile : valid))
                             finalise_chunk<DT, 16, TS>(v, carried_in && valid, emit, rp + c, bias ? bias + c : nullptr, sink,
-                                                       (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift);
+                                                       (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift, pc, state_ok);
                     }
                 }
                 tmem_st_wait();
@@ -758,16 +842,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_free + 8u * slot);   // one arrival per warp
             }
-            if (emit) {
+            if (emit && (!a.pool || pc.second)) {      // with pooling only the second row of a pair sends a (pooled) row out
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 named_bar_sync(1 + grp, 128);
                 if (leader) {
-                    const int orow = a.out_row_first + orel;
+                    const int orow = a.pool ? (int)(((a.o_begin + orel) >> 1) - a.pool_row_base) : a.out_row_first + orel;
+                    const int xc = a.pool ? (x0 >> 1) : x0;
                     for (int pnl = 0; pnl < a.out_panels; ++pnl) {
                         if (a.out_row_dim == 3)
-                            tma_store_4d(&tmO, stg + (uint32_t)pnl * sink.panel_bytes, n0 + pnl * panel_cols, x0, s0, orow);
+                            tma_store_4d(&tmO, stg + (uint32_t)pnl * sink.panel_bytes, n0 + pnl * panel_cols, xc, s0, orow);
                         else
-                            tma_store_4d(&tmO, stg + (uint32_t)pnl * sink.panel_bytes, n0 + pnl * panel_cols, x0, orow, s0);
+                            tma_store_4d(&tmO, stg + (uint32_t)pnl * sink.panel_bytes, n0 + pnl * panel_cols, xc, orow, s0);
                     }
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
@@ -828,7 +913,7 @@ CUtensorMapSwizzle swizzle_of(int swb)
 }  // namespace
 
 bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh, int Kw, int stride_x, int ring_rows,
-                  int out_esize, TcPlan* p)
+                  int out_esize, int pooled, TcPlan* p)
 {
     *p = TcPlan{};
     if (dtype != 1 && dtype != 2) return false;
@@ -860,13 +945,15 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     p->a_stage_bytes = (int)a_stage;
     p->n_mt = p->n_xt * ((S + p->BS - 1) / p->BS);
     const int taps = Kh * Kw;
+    // a launch that emits pooled rows stages half a tile of positions
+    const int stage_rows = pooled ? 64 : 128;
     int best = 0, best_units = -1;
     for (int nt = 256; nt >= 16; nt >>= 1) {
         if (Cout % nt) continue;
         if ((ring_rows + 1) * nt > 512) continue;
         if ((ring_rows + 256 / nt - 1) / (256 / nt) + 1 > 4) continue;   // at most 4 MMA segments per input row
         const size_t wb = (size_t)taps * p->n_kb * nt * p->swb;
-        if (wb + 3 * a_stage + 128 * (size_t)nt * out_esize + 10240 > SMEM_LIMIT) continue;   // one staging tile at least
+        if (wb + 3 * a_stage + (size_t)stage_rows * nt * out_esize + 10240 > SMEM_LIMIT) continue;   // one staging tile at least
         const int units = p->n_mt * (Cout / nt);
         if (units >= 120) { best = nt; break; }          // enough CTAs for the 148 SMs: take the widest such tile
         if (units > best_units) { best_units = units; best = nt; }
@@ -885,7 +972,8 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     p->out_esize = out_esize;
     p->out_pwb = best * out_esize >= 128 ? 128 : best * out_esize;
     p->out_panels = best * out_esize / p->out_pwb;
-    p->out_stage_bytes = p->out_panels * 128 * p->out_pwb;
+    p->out_stage_rows = stage_rows;
+    p->out_stage_bytes = p->out_panels * stage_rows * p->out_pwb;
     // as many epilogue groups (one staging tile each) as still leave three Δ-row stages
     p->out_groups = 1;
     for (int g = MAX_GROUPS; g > 1; --g)
@@ -941,9 +1029,13 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     const int row_dim = a.out_row_stride > a.out_stream_stride ? 3 : 2;
     {
         const int oes = p.out_esize;
-        cuuint64_t od[4] = {(cuuint64_t)a.Cout, (cuuint64_t)a.Wout, 0, 0};
+        const int ow = a.pool_fused ? a.Wout / 2 : a.Wout;            // width of the rows that leave the kernel
+        const int obx = a.pool_fused ? p.BX / 2 : p.BX;
+        if (a.pool_fused && ((p.BX & 1) || ow < 1 || !a.pool_state)) return cudaErrorNotSupported;
+        if ((a.pool_fused != 0) != (p.out_stage_rows == 64)) return cudaErrorNotSupported;   // the plan's staging tile must fit the rows that leave
+        cuuint64_t od[4] = {(cuuint64_t)a.Cout, (cuuint64_t)ow, 0, 0};
         cuuint64_t os[3] = {(cuuint64_t)a.Cout * oes, 0, 0};
-        cuuint32_t ob[4] = {(cuuint32_t)(p.out_pwb / oes), (cuuint32_t)p.BX, 1, 1};
+        cuuint32_t ob[4] = {(cuuint32_t)(p.out_pwb / oes), (cuuint32_t)obx, 1, 1};
         od[row_dim] = (cuuint64_t)a.out_rows_extent; od[5 - row_dim] = (cuuint64_t)a.S;
         os[row_dim - 1] = (cuuint64_t)a.out_row_stride * oes; os[4 - row_dim] = (cuuint64_t)a.out_stream_stride * oes;
         ob[5 - row_dim] = (cuuint32_t)p.BS;
@@ -977,8 +1069,9 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     t.BX = p.BX; t.BS = p.BS; t.n_xt = p.n_xt; t.Ntile = p.Ntile; t.n_nt = p.n_nt; t.KB = p.KB; t.n_kb = p.n_kb;
     t.swb = p.swb; t.nslot = p.nslot; t.nstage = p.nstage; t.tmem_cols = p.tmem_cols;
     t.BXP = p.BXP; t.shift_mode = p.shift_mode; t.a_stage_bytes = p.a_stage_bytes;
-    t.out_esize = p.out_esize; t.out_pwb = p.out_pwb; t.out_panels = p.out_panels; t.out_stage_bytes = p.out_stage_bytes; t.out_groups = p.out_groups;
+    t.out_esize = p.out_esize; t.out_pwb = p.out_pwb; t.out_panels = p.out_panels; t.out_stage_bytes = p.out_stage_bytes; t.out_stage_rows = p.out_stage_rows; t.out_groups = p.out_groups;
     t.out_row_dim = row_dim; t.out_row_first = (int)(a.o_begin - a.out_row_base);
+    t.pool = a.pool_fused; t.pool_keep = a.pool_keep; t.pool_state = a.pool_state; t.pool_row_base = a.out_row_base;
     const unsigned grid = (unsigned)(p.n_mt * p.n_nt);
     typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const TcArgs);
     static const KernelFn kernels[2][3] = {

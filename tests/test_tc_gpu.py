@@ -93,3 +93,58 @@ def test_tensor_core_and_cuda_core_paths_agree_bitwise_on_int8(orc, monkeypatch)
     got_cc, tc2 = _run("i8", layers, x, ws, bs)
     assert not any(tc2)
     assert np.array_equal(got_tc, got_cc)
+
+
+# ---- 2x2 max-pooling folded into the emission of the conv layer in front of it ----------------------
+POOL_CASES = [
+    # (name, mode, layers, H, W, S)
+    ("i8_conv_pool", "i8", (conv(32, 32, 3, pad=1), POOL), 18, 24, 7),
+    ("i8_conv_pool_conv", "i8", (conv(32, 64, 3, pad=1), POOL, conv(64, 32, 3, pad=1), POOL), 22, 40, 5),
+    ("i8_pool_odd_rows_valid", "i8", (conv(64, 32, 3), POOL, conv(32, 32, 3)), 21, 30, 6),
+    ("i8_pool_wide_two_x_tiles", "i8", (conv(32, 16, 3, pad=1), POOL), 9, 224, 2),
+    ("i8_pool_odd_width", "i8", (conv(32, 32, 3), POOL), 12, 29, 4),            # Wout = 27: the last column is dropped
+    ("bf16_last_conv_pool_fp32", "bf16", (conv(64, 32, 3, pad=1), POOL), 14, 56, 5),   # fp32 rows pooled
+    ("bf16_pool_then_conv", "bf16", (conv(64, 64, 3, pad=1), POOL, conv(64, 16, 3, pad=1)), 16, 24, 5),
+    ("i8_unfold_pool", "i8", (conv(16, 32, 3, pad=1), POOL), 15, 26, 7),
+]
+
+
+@pytest.mark.parametrize("name,mode,layers,H,W,S", POOL_CASES, ids=[c[0] for c in POOL_CASES])
+def test_pool_folded_into_the_conv_launch_matches_oracle(orc, monkeypatch, name, mode, layers, H, W, S):
+    if mode == "i8":
+        layers = with_shifts(layers, 9)
+    x, ws, bs = rand_net(mode, layers, H, W, layers[0].cin, S=S, seed=3 + len(name))
+    want = orc.forward(mode, layers, x, ws, bs)
+    n_conv = sum(l.kind == "conv" for l in layers)
+
+    def run(chunks, rb, last):
+        net = idf.Net(mode, layers, W, layers[0].cin, S, ws, bs, row_block=rb)
+        got = idf.infer(net, x, chunks=chunks, last=last)
+        return got, net.launches
+
+    def check(got, what):
+        if mode == "i8":
+            assert_equal(got, want, what)
+        elif n_conv == 1:
+            assert_close(got, want, what)
+        else:
+            err = np.abs(got - want)
+            ok = err <= 1e-4 + 1e-3 * np.abs(want)
+            assert ok.mean() > 0.97 and err.max() < 0.05, (what, ok.mean(), err.max())
+
+    # pairs of rows split across launches in every way: one row at a time, odd groups, everything at once
+    fused_launches = None
+    for chunks, rb, last in ((None, 0, True), (None, 0, False), ([1] * H, 0, False), ([3, 2, 5, 1], 3, True),
+                             ([H - 1], 0, True), (None, 5, True)):
+        got, n = run(chunks, rb, last)
+        check(got, f"{name}/chunks={chunks}/rb={rb}/last={last}")
+        if chunks is None and rb == 0 and last:
+            fused_launches = n
+    # the same net with the folding switched off runs the pool layers as launches of their own
+    monkeypatch.setenv("IDF_NO_POOL_FUSION", "1")
+    got, n = run(None, 0, True)
+    check(got, f"{name}/unfused")
+    if name == "i8_pool_odd_width":          # an odd tile width cannot pair lanes: this net never folds
+        assert n == fused_launches
+    else:
+        assert n > fused_launches, (n, fused_launches)
