@@ -941,7 +941,10 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     }
     p->BXP = p->BX + halo;
     if (p->BXP > 256) return false;
-    const size_t a_stage = ((size_t)((128 + halo + 7) / 8 * 8) * p->swb + 1023) / 1024 * 1024;
+    // A stage holds exactly the TMA box (BS streams x BXP positions).  The MMAs read 128 rows from row kx on,
+    // so for the last positions they run past the box into whatever follows in shared memory: those are
+    // lanes outside the tile, whose accumulators nobody reads.
+    const size_t a_stage = ((size_t)p->BS * p->BXP * p->swb + 1023) / 1024 * 1024;
     p->a_stage_bytes = (int)a_stage;
     p->n_mt = p->n_xt * ((S + p->BS - 1) / p->BS);
     const int taps = Kh * Kw;
@@ -976,14 +979,23 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     p->out_stage_bytes = p->out_panels * stage_rows * p->out_pwb;
     // as many epilogue groups (one staging tile each) as still leave three Δ-row stages
     p->out_groups = 1;
+    // layers with many short K blocks per row (little MMA work per tile) need a deeper pipeline to cover the
+    // copy latency more than they need a second epilogue group
+    const size_t want_stages = p->n_kb >= 4 ? 4 : 3;
     for (int g = MAX_GROUPS; g > 1; --g)
-        if (wb + 3 * a_stage + (size_t)g * p->out_stage_bytes + 10240 <= SMEM_LIMIT) { p->out_groups = g; break; }
-    const size_t room = SMEM_LIMIT - 8192 - wb - 1024 - (size_t)p->out_groups * p->out_stage_bytes;   // static shared memory and alignment slack stay free
+        if (wb + want_stages * a_stage + (size_t)g * p->out_stage_bytes + 10240 <= SMEM_LIMIT) { p->out_groups = g; break; }
+    // the MMAs' run past a small box (see a_stage) must end inside this CTA's shared memory: what follows the
+    // last stage (the staging tiles) covers it, or padding is added behind them
+    const size_t overrun = (size_t)(128 + halo) * p->swb > a_stage ? (size_t)(128 + halo) * p->swb - a_stage : 0;
+    const size_t tail_have = (size_t)p->out_groups * p->out_stage_bytes;
+    const size_t tail_pad = overrun > tail_have ? (overrun - tail_have + 1023) / 1024 * 1024 : 0;
+    if (SMEM_LIMIT < 8192 + wb + 1024 + tail_have + tail_pad + 2 * a_stage) return false;
+    const size_t room = SMEM_LIMIT - 8192 - wb - 1024 - tail_have - tail_pad;   // static shared memory and alignment slack stay free
     int nstage = (int)(room / a_stage);
     if (nstage > 8) nstage = 8;
     if (nstage < 2) return false;
     p->nstage = nstage;
-    p->smem_bytes = 1024 + wb + (size_t)nstage * a_stage + (size_t)p->out_groups * p->out_stage_bytes + 8 * (2 * nstage + taps + 2 * p->nslot) + 64;
+    p->smem_bytes = 1024 + wb + (size_t)nstage * a_stage + (size_t)p->out_groups * p->out_stage_bytes + tail_pad + 8 * (2 * nstage + taps + 2 * p->nslot) + 64;
     p->w_bytes = (size_t)taps * Cout * Cin * esize;
     p->ok = 1;
     return true;
