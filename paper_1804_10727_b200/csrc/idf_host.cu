@@ -533,8 +533,13 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
                 }
             }
             if (biases && biases[i]) {
-                P.b_packed.resize((size_t)l.cout * 4);
-                memcpy(P.b_packed.data(), biases[i], (size_t)l.cout * 4);
+                // an all-zero bias is no bias: the kernels then skip the add (state words: +0.0f and 0 are all-zero bits)
+                bool any = false;
+                for (size_t k = 0; k < (size_t)l.cout * 4 && !any; ++k) any = ((const unsigned char*)biases[i])[k] != 0;
+                if (any) {
+                    P.b_packed.resize((size_t)l.cout * 4);
+                    memcpy(P.b_packed.data(), biases[i], (size_t)l.cout * 4);
+                }
             }
         } else if (l.kind == IDF_MAXPOOL2) {
             P.out_w = (w == 1) ? 1 : w / 2;
