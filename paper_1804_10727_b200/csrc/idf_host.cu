@@ -71,6 +71,7 @@ struct idf_net {
     int dtype = 0, in_w = 0, in_c = 0, n_streams = 0, row_block = 0;
     std::vector<LayerPlan> L;
     size_t workspace_bytes = 0, state_region_off = 0, state_region_bytes = 0, counters_off = 0, status_off = 0;
+    size_t ring_scratch_off = 0;           // room for a copy of the largest tensor-core layer's ring (row-chunked launches)
     size_t state_bytes_stream = 0;
     unsigned char* ws = nullptr;
     cudaStream_t stream = nullptr;
@@ -179,6 +180,7 @@ int launch_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, boo
         a.w = net->ws + P.w_off;
         a.bias = P.b_packed.empty() ? nullptr : net->ws + P.b_off;
         a.ring = net->ws + P.state_off;
+    a.ring_scratch = net->ring_scratch_off ? net->ws + net->ring_scratch_off : nullptr;
         a.out = out_ptr;
         a.out_row_stride = row_stride; a.out_stream_stride = stream_stride; a.out_row_base = row_base;
         a.out_rows_extent = last ? out_cap : P.out_cap_rows;
@@ -256,6 +258,7 @@ int launch_conv_pool(idf_net* net, size_t i, const void* in_ptr, long long n_in,
     a.w = net->ws + P.w_off;
     a.bias = P.b_packed.empty() ? nullptr : net->ws + P.b_off;
     a.ring = net->ws + P.state_off;
+    a.ring_scratch = net->ring_scratch_off ? net->ws + net->ring_scratch_off : nullptr;
     if (last) {
         a.out = final_out;
         a.out_row_stride = (long long)Q.out_w * Q.out_c;
@@ -589,6 +592,12 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
             P.unf_off = off;
             off = align_up(off + (size_t)P.in_cap_rows * net->n_streams * P.out_w * P.kpad * elem_size(P.in_elem), 1024);
         }
+    {
+        size_t biggest = 0;
+        for (auto& P : net->L)
+            if (P.l.kind == IDF_CONV && P.tc.ok) biggest = std::max(biggest, P.state_bytes_all);
+        if (biggest) { net->ring_scratch_off = off; off = align_up(off + biggest); }
+    }
     net->counters_off = off;
     off = align_up(off + net->L.size() * sizeof(unsigned long long));
     net->status_off = off;

@@ -24,6 +24,7 @@ struct ConvArgs {
     const void* w;         // packed weights (layout depends on the kernel)
     const void* bias;      // [Cout] in the state type, or nullptr
     void* ring;            // [ring_rows][S][Wout][Cout] state words
+    void* ring_scratch;    // tensor-core kernel: room for a copy of the ring (same size), or nullptr
     void* out;             // emitted rows
     long long out_row_stride, out_stream_stride, out_row_base;  // element strides; row o goes to (o - out_row_base)
     long long out_rows_extent;   // rows the output buffer holds per stream

@@ -352,13 +352,13 @@ __device__ __forceinline__ bool named_bar_and(int id, int count, bool pred)
 template <int DT, int W, typename TS>
 __device__ __forceinline__ void finalise_chunk(const uint32_t (&v)[W], bool carried_in, bool emit, TS* rp,
                                                const TS* bias_c, const StageSink& sink, uint32_t col_byte, int out_elem,
-                                               int relu, int shift, const PoolCtx& pc, bool state_ok)
+                                               int relu, int shift, const PoolCtx& pc, bool state_ok, long long carry_off)
 {
     TS acc[W];
 #pragma unroll
     for (int j = 0; j < W; ++j) acc[j] = DT == 1 ? (TS)__uint_as_float(v[j]) : (TS)(int)v[j];
     if (carried_in) {
-        const int4* p4 = (const int4*)rp;
+        const int4* p4 = (const int4*)(rp + carry_off);      // what earlier blocks left: the ring itself, or the launch's copy of it
 #pragma unroll
         for (int j4 = 0; j4 < W / 4; ++j4) {
             const int4 t4 = p4[j4];
@@ -441,6 +441,8 @@ __device__ __forceinline__ void finalise_chunk(const uint32_t (&v)[W], bool carr
 struct TcArgs {
     const void* bias;
     void* ring;
+    const void* ring_in;         // where the rows begun by earlier blocks are read: the ring, or a copy of it made before a
+                                 // launch whose row chunks run in CTAs of their own (one parks rows while another still reads)
     void* out;
     unsigned int* status;
     long long out_row_stride, out_stream_stride, out_row_base;
@@ -456,6 +458,8 @@ struct TcArgs {
     int S, Wout, Cout, Kh, Kw, stride, pad_x, relu, shift, ring_rows, out_elem;
     int BX, BXP, BS, n_xt, Ntile, n_nt, KB, n_kb, swb, nslot, nstage, tmem_cols;
     int shift_mode;              // 1: one box per (row, K block) holds the kx halo, taps address it at row offsets
+    int n_chunks, chunk_rows, chunk_shift;   // the block's output rows are cut into n_chunks runs of chunk_rows rows (the first one
+                                 // chunk_shift shorter), one CTA each: see the kernel's prologue
     int a_stage_bytes;
     int out_esize, out_pwb, out_panels, out_stage_bytes;   // emitted rows: staging panels of out_pwb-byte rows
     int out_stage_rows;          // rows of one staging panel: 128, or 64 when only pooled rows are staged
@@ -505,7 +509,27 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t bar_free = bar_ready + 8u * a.nslot;
 
     const int nt = blockIdx.x % a.n_nt;
-    const int mt = blockIdx.x / a.n_nt;
+    const int mt_all = blockIdx.x / a.n_nt;
+    const int n_mt_all = a.n_xt * ((a.S + a.BS - 1) / a.BS);
+    const int mt = mt_all % n_mt_all;
+    // Row chunks.  When a layer has few (position, channel) tiles, the block's output rows are cut into runs and
+    // every run gets CTAs of its own: a run needs only the input rows its output rows reach, which it reads again
+    // at its edges instead of taking partial sums from its neighbour.  Inside a chunk everything is as in a block
+    // that starts at the chunk's first output row: taps into rows of other chunks drop out, only the first chunk
+    // takes up the ring, only the last one parks rows in it.
+    const int chunk = mt_all / n_mt_all;
+    const int c_oa = chunk == 0 ? 0 : chunk * a.chunk_rows - a.chunk_shift;                       // first relative output row
+    const int c_ob = chunk == a.n_chunks - 1 ? a.n_orows : (chunk + 1) * a.chunk_rows - a.chunk_shift;
+    int c_ra = c_oa * a.stride - a.base_ty;                                                        // first input row that reaches it
+    if (c_ra < 0) c_ra = 0;
+    int c_rb = (c_ob - 1) * a.stride - a.base_ty + a.Kh;                                           // one past the last
+    if (c_rb > a.n_rows || chunk == a.n_chunks - 1) c_rb = a.n_rows;
+    const long long c_o_begin = a.o_begin + c_oa;
+    const int c_base_ty = a.base_ty + c_ra - c_oa * a.stride;
+    const int c_n_orows = c_ob - c_oa;
+    const int c_done_rel = min(max(a.done_rel - c_oa, 0), c_n_orows);
+    const int c_sched_rel = min(max(a.sched_rel - c_oa, 0), c_n_orows);
+    const bool c_r0_positive = a.r0_positive && chunk == 0;
     const int xt = mt % a.n_xt, stile = mt / a.n_xt;
     const int x0 = xt * a.BX, s0 = stile * a.BS, n0 = nt * a.Ntile;
 
@@ -538,7 +562,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t tmem_base = s_tmem_base;
     volatile int* abort_flag = &s_abort;
-    const int n_rows = a.n_rows;
+    const int n_rows = c_rb - c_ra;
 
     if (warp == 0) {
         // ------------------------------ TMA producer + row scheduler ---------------------------
@@ -562,26 +586,28 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int ri = r_chunk + lane;
                 if (ri < n_rows) {
                     uint32_t* q = s_rowq[ri & (ROWQ - 1)];
-                    const int t0 = a.base_ty + ri;
+                    const int t0 = c_base_ty + ri;
                     const int hi = t0 / s, ph = t0 - hi * s;
                     const int slot_hi = hi % nslot, u_hi = hi / nslot;
                     // a new output row starts when ph == 0: its slot's previous row must have been read out
-                    const bool fresh = (ri > 0 && ph == 0 && hi >= nslot);
+                    const bool fresh = (ri > 0 && ph == 0 && hi >= nslot && hi < c_n_orows);
                     q[0] = fresh ? bar_free + 8u * (uint32_t)slot_hi : 0u;
                     q[1] = (uint32_t)(u_hi & 1);
                     // the row completed by input row ri is (t0 - (Kh-1)) / s when that is a whole number >= 0
                     const int tf = t0 - (a.Kh - 1);
                     const int of = tf >= 0 ? tf / s : -1;
-                    q[3] = (tf >= 0 && of * s == tf && of < a.sched_rel) ? bar_ready + 8u * (uint32_t)(of % nslot) : 0u;
+                    q[3] = (tf >= 0 && of * s == tf && of < c_sched_rel) ? bar_ready + 8u * (uint32_t)(of % nslot) : 0u;
                     // taps ky = ph, ph+s, ... < Kh; those that would reach rows above the map drop out
                     const int cnt = (a.Kh - ph + s - 1) / s;
                     int n_t = cnt;
                     if (n_t > hi + 1) n_t = hi + 1;
-                    int sl = slot_hi - (n_t - 1);
+                    int sl = (slot_hi - (n_t - 1)) % nslot;
                     if (sl < 0) sl += nslot;
                     int poff = 0;
                     for (int p = 0; p < ph; ++p) poff += (a.Kh - p + s - 1) / s;
                     uint32_t blk = (uint32_t)(poff + cnt - n_t);
+                    // ... and so do those that reach rows beyond this chunk (the highest rows = the first taps)
+                    if (hi > c_n_orows - 1) n_t -= hi - (c_n_orows - 1);
                     // segments: runs of rows whose slots are consecutive TMEM column blocks (N <= 256 each)
                     int n_seg = 0;
                     for (int rem = n_t; rem > 0 && n_seg < 4; ++n_seg) {
@@ -611,7 +637,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                             mbar_expect_tx(bar_full + 8u * stage, a_box_bytes);
                             tma_load_4d(sA + (uint32_t)stage * a_stage_bytes, &tmA, bar_full + 8u * stage,
-                                        kb * a.KB, x0 - a.pad_x + xl, s0, ri);
+                                        kb * a.KB, x0 - a.pad_x + xl, s0, c_ra + ri);
                             ++t;
                             if (++stage == a.nstage) { stage = 0; phase ^= 1u; }
                         }
@@ -679,7 +705,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         uint64_t bdesc = bdesc_base + (uint64_t)((a.shift_mode ? 0u : (uint32_t)xl) * wtile_kx + (uint32_t)kb * wtile_kb);
                         uint32_t next_ok = 1u;
                         for (int kxi = 0; kxi < n_kx; ++kxi, adesc += kx_bytes, bdesc += wtile_kx) {
-                            if (issuer) {
+                            if (issuer && hdr.z > 0) {
                                 umma_tile<DT, KSTEPS>(sa.x, adesc, bdesc + (uint64_t)sa.y, sa.z);
                                 if (hdr.z > 1) {
                                     umma_tile<DT, KSTEPS>(sa.w, adesc, bdesc + (uint64_t)sb.x, sb.y);
@@ -701,7 +727,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                 // (to be parked in the ring, or emitted if only bottom padding was missing)
                                 if (hdr.w) umma_commit(hdr.w);
                                 if (last_row)
-                                    for (int orel = a.sched_rel; orel < a.n_orows; ++orel) umma_commit(bar_ready + 8u * (uint32_t)(orel % nslot));
+                                    for (int orel = c_sched_rel; orel < c_n_orows; ++orel) umma_commit(bar_ready + 8u * (uint32_t)(orel % nslot));
                             }
                         }
                         if (!next_ok && !mbar_wait(bar_full + 8u * nstage_i, nphase, abort_flag)) { ok = false; break; }
@@ -733,6 +759,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const long long row_elems = (long long)a.Wout * a.Cout;
         TS* ring_pos = (TS*)a.ring + (long long)s * row_elems + (long long)x * a.Cout + n0;   // + ring slot * S * row_elems
         const long long ring_slot_stride = (long long)a.S * row_elems;
+        const long long carry_off = (const TS*)a.ring_in - (const TS*)a.ring;
         const uint32_t tlane = tmem_base + ((uint32_t)(q * 32) << 16);
         const int md = bs * a.BX + bx;                   // row of the dense output tile
         StageSink sink;
@@ -767,20 +794,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // Rows that exchange state with the ring in global memory (those begun by an earlier block and
         // those left open by this one) may share a ring slot; group 0 takes them all, in order, so a
         // slot is read before it is rewritten.  The other rows go round the groups.
-        const int n_cin = a.r0_positive ? (a.base_ty + a.stride - 1) / a.stride : 0;
-        for (int orel = 0; orel < a.n_orows && ok && grp < a.out_groups; ++orel) {
+        const int n_cin = c_r0_positive ? (c_base_ty + a.stride - 1) / a.stride : 0;
+        for (int orel = 0; orel < c_n_orows && ok && grp < a.out_groups; ++orel) {
             int owner;
             if (!a.pool) {
-                owner = (orel < n_cin || orel >= a.done_rel) ? 0 : orel % a.out_groups;
+                owner = (orel < n_cin || orel >= c_done_rel) ? 0 : orel % a.out_groups;
             } else {
                 // both rows of a pooling pair go to one group; pairs touching the global ring go to group 0
-                const int first = orel - (int)((a.o_begin + orel) & 1);
-                owner = (first < n_cin || first + 1 >= a.done_rel) ? 0 : (int)(((a.o_begin + orel) >> 1) % a.out_groups);
+                const int first = orel - (int)((c_o_begin + orel) & 1);
+                owner = (first < n_cin || first + 1 >= c_done_rel) ? 0 : (int)(((c_o_begin + orel) >> 1) % a.out_groups);
             }
             if (owner != grp) continue;
             const int slot = orel % a.nslot;
             const uint32_t par = (uint32_t)((orel / a.nslot) & 1);
-            const bool emit = orel < a.done_rel;
+            const bool emit = orel < c_done_rel;
             // one thread of the group polls the barrier; the named barrier below releases the other warps
             int got = 1;
             if (leader) got = mbar_wait_relaxed(bar_ready + 8u * slot, par, abort_flag) ? 1 : 0;
@@ -789,16 +816,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (emit && leader) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             if (!named_bar_and(1 + grp, 128, got != 0)) { ok = false; break; }
             tc_fence_after();
-            const bool carried_in = a.r0_positive && (orel * a.stride - a.base_ty < 0);
+            const bool carried_in = c_r0_positive && (orel * a.stride - c_base_ty < 0);
             const bool pool_emit = a.pool && emit;
             if (pool_emit) {
-                pc.second = (int)((a.o_begin + orel) & 1);
+                pc.second = (int)((c_o_begin + orel) & 1);
                 pc.from_state = pc.second && orel == 0;
-                const bool trailing = !pc.second && orel == a.done_rel - 1;
+                const bool trailing = !pc.second && orel == c_done_rel - 1 && c_oa + c_done_rel == a.done_rel;   // the block's last emitted row
                 pc.to_state = trailing && a.pool_keep;
                 pc.drop = trailing && !a.pool_keep;
             }
-            TS* rp = ring_pos + (long long)((a.o_begin + orel) % a.ring_rows) * ring_slot_stride;
+            TS* rp = ring_pos + (long long)((c_o_begin + orel) % a.ring_rows) * ring_slot_stride;
             const uint32_t trow = tlane + (uint32_t)(slot * a.Ntile);
             if (a.Ntile == 64 || a.Ntile == 32) {
                 // the whole row fits in registers: take it, clear and release the slot at once, then finalise
@@ -812,10 +839,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_free + 8u * slot);   // one arrival per warp
                 if (pool_emit || (emit ? in_tile : valid)) {
-                    finalise_chunk<DT, 32, TS>(v0, carried_in && valid, emit, rp, bias, sink, 0u, a.out_elem, a.relu, a.shift, pc, state_ok);
+                    finalise_chunk<DT, 32, TS>(v0, carried_in && valid, emit, rp, bias, sink, 0u, a.out_elem, a.relu, a.shift, pc, state_ok, carry_off);
                     if (a.Ntile == 64)
                         finalise_chunk<DT, 32, TS>(v1, carried_in && valid, emit, rp + 32, bias ? bias + 32 : nullptr, sink,
-                                                   (uint32_t)(32 * a.out_esize), a.out_elem, a.relu, a.shift, pc, state_ok);
+                                                   (uint32_t)(32 * a.out_esize), a.out_elem, a.relu, a.shift, pc, state_ok, carry_off);
                 }
             } else {
                 if (wide) {
@@ -825,7 +852,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         tmem_st_zero<32>(trow + c);           // the slot's next row starts from zero
                         if (pool_emit || (emit ? in_tile : valid))
                             finalise_chunk<DT, 32, TS>(v, carried_in && valid, emit, rp + c, bias ? bias + c : nullptr, sink,
-                                                       (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift, pc, state_ok);
+                                                       (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift, pc, state_ok, carry_off);
                     }
                 } else {
                     for (int c = 0; c < a.Ntile; c += 16) {
@@ -834,7 +861,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         tmem_st_zero<16>(trow + c);
                         if (pool_emit || (emit ? in_tile : valid))
                             finalise_chunk<DT, 16, TS>(v, carried_in && valid, emit, rp + c, bias ? bias + c : nullptr, sink,
-                                                       (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift, pc, state_ok);
+                                                       (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift, pc, state_ok, carry_off);
                     }
                 }
                 tmem_st_wait();
@@ -846,7 +873,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 named_bar_sync(1 + grp, 128);
                 if (leader) {
-                    const int orow = a.pool ? (int)(((a.o_begin + orel) >> 1) - a.pool_row_base) : a.out_row_first + orel;
+                    const int orow = a.pool ? (int)(((c_o_begin + orel) >> 1) - a.pool_row_base) : a.out_row_first + c_oa + orel;
                     const int xc = a.pool ? (x0 >> 1) : x0;
                     for (int pnl = 0; pnl < a.out_panels; ++pnl) {
                         if (a.out_row_dim == 3)
@@ -1084,7 +1111,34 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     t.out_esize = p.out_esize; t.out_pwb = p.out_pwb; t.out_panels = p.out_panels; t.out_stage_bytes = p.out_stage_bytes; t.out_stage_rows = p.out_stage_rows; t.out_groups = p.out_groups;
     t.out_row_dim = row_dim; t.out_row_first = (int)(a.o_begin - a.out_row_base);
     t.pool = a.pool_fused; t.pool_keep = a.pool_keep; t.pool_state = a.pool_state; t.pool_row_base = a.out_row_base;
-    const unsigned grid = (unsigned)(p.n_mt * p.n_nt);
+    // row chunks: a layer with few tiles (few streams, narrow rows) spreads the block's rows over more CTAs
+    t.n_chunks = 1; t.chunk_rows = t.n_orows; t.chunk_shift = 0;
+    {
+        const int units = p.n_mt * p.n_nt;
+        int min_rows = 2 * a.ring_rows + 2;
+        if (min_rows < 16) min_rows = 16;
+        static const bool no_chunks = getenv("IDF_NO_ROW_CHUNKS") != nullptr;
+        // (a block that continues rows of an earlier one needs room for the copy of the ring, see ring_in)
+        if (!no_chunks && units < 120 && t.n_orows >= 2 * min_rows && (a.r0 == 0 || a.ring_scratch)) {
+            int want = (296 + units - 1) / units;
+            if (want > t.n_orows / min_rows) want = t.n_orows / min_rows;
+            if (want > 1) {
+                int rows = (t.n_orows + want - 1) / want;
+                rows += rows & 1;                                   // even: a pooling pair stays in one chunk
+                t.chunk_shift = a.pool_fused ? (int)(a.o_begin & 1) : 0;
+                t.chunk_rows = rows;
+                t.n_chunks = (t.n_orows + t.chunk_shift + rows - 1) / rows;
+            }
+        }
+    }
+    t.ring_in = a.ring;
+    if (t.n_chunks > 1 && a.r0 > 0) {
+        const size_t ring_bytes = (size_t)a.ring_rows * a.S * a.Wout * a.Cout * 4;
+        cudaError_t ce = cudaMemcpyAsync(a.ring_scratch, a.ring, ring_bytes, cudaMemcpyDeviceToDevice, st);
+        if (ce != cudaSuccess) return ce;
+        t.ring_in = a.ring_scratch;
+    }
+    const unsigned grid = (unsigned)(p.n_mt * p.n_nt * t.n_chunks);
     typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const TcArgs);
     static const KernelFn kernels[2][3] = {
         {conv_tc_kernel<1, 1>, conv_tc_kernel<1, 2>, conv_tc_kernel<1, 4>},

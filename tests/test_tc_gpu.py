@@ -148,3 +148,36 @@ def test_pool_folded_into_the_conv_launch_matches_oracle(orc, monkeypatch, name,
         assert n == fused_launches
     else:
         assert n > fused_launches, (n, fused_launches)
+
+
+# ---- few streams, many rows: the block's output rows are spread over CTAs in chunks ------------------
+CHUNK_CASES = [
+    ("i8_same_pad", "i8", (conv(32, 32, 3, pad=1),), 150, 20, 3),
+    ("i8_valid_pool", "i8", (conv(32, 32, 3), POOL, conv(32, 16, 3, pad=1)), 131, 24, 2),
+    ("i8_stride2_1d", "i8", (conv(32, 64, 9, stride=2, one_d=True), conv(64, 64, 9, one_d=True)), 700, 1, 40),
+    ("i8_k5_pool_pool", "i8", (conv(64, 32, 5, pad=2), POOL, conv(32, 32, 3, pad=1), POOL), 97, 16, 4),
+    ("bf16_1d_single", "bf16", (conv(64, 64, 9, stride=2, one_d=True),), 900, 1, 100),
+]
+
+
+@pytest.mark.parametrize("name,mode,layers,H,W,S", CHUNK_CASES, ids=[c[0] for c in CHUNK_CASES])
+def test_row_chunks_match_oracle(orc, monkeypatch, name, mode, layers, H, W, S):
+    if mode == "i8":
+        layers = with_shifts(layers, 9)
+    x, ws, bs = rand_net(mode, layers, H, W, layers[0].cin, S=S, seed=11 + len(name))
+    want = orc.forward(mode, layers, x, ws, bs)
+    # blocks that begin, continue and end streams, with rows carried over launch boundaries in both directions
+    for chunks, rb, last in ((None, 0, True), (None, 0, False), ([H // 2 + 1], 0, True), ([H // 2, H // 4], 0, False),
+                             ([37, 50], 64, False), (None, 1024, True)):
+        net = idf.Net(mode, layers, W, layers[0].cin, S, ws, bs, row_block=rb)
+        got = idf.infer(net, x, chunks=chunks, last=last)
+        what = f"{name}/chunks={chunks}/rb={rb}/last={last}"
+        if mode == "i8":
+            assert_equal(got, want, what)
+        else:
+            assert_close(got, want, what)
+    if mode == "i8":
+        # the same with the rows of a block kept in one CTA per tile: bit-identical
+        monkeypatch.setenv("IDF_NO_ROW_CHUNKS", "1")
+        net = idf.Net(mode, layers, W, layers[0].cin, S, ws, bs)
+        assert_equal(idf.infer(net, x, last=True), want, name + "/unchunked")
