@@ -281,6 +281,13 @@ def run_ours(args, w):
         flops = 2.0 * sum(macs[i] for i in dense) * w.n_streams
         achieved = flops / (dom_ms * 1e-3) / 1e12 if dom_ms > 0 else 0.0
         ratio = {"bf16": 1.0, "i8": 2.0, "f32": 0.5}[w.dtype]      # nominal ratio to the bf16 dense peak
+        # DRAM bytes of the conv launches of one step, from the ncu capture summarised in
+        # profiles/conv_tc_kernel_vgg2d_rows64.md (dram__bytes_read.sum + dram__bytes_write.sum of the seven launches
+        # of a 64-row case = 408.3 MB; the traffic is rows in + rows out, so it grows with the number of rows)
+        traffic, traffic_note = None, "no ncu capture for this workload"
+        if w.name == "vgg2d" and w.n_streams == 64:
+            traffic = 408.3e6 * w.H / 64.0
+            traffic_note = "bytes per step over all conv launches, scaled by rows from a 64-row ncu capture (cold caches)"
         peak = peaks["bf16_tflops"] * ratio
         line = {
             "metric": METRIC, "value": whole_job_value(w, world, args.steps, ms), "unit": UNIT, "n_gpus": world,
@@ -301,7 +308,8 @@ def run_ours(args, w):
                           "note": "segments pushed as they arrive for all streams, the last push carries the end of input"},
             "roofline": {"bound": "tensor", "kernel": "dense conv update (all conv layers)", "achieved": achieved,
                          "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak if peak else None,
-                         "peak_source": f"{peaks['source']} bf16 sustained x{ratio}", "traffic": None,
+                         "peak_source": f"{peaks['source']} bf16 sustained x{ratio}", "traffic": traffic,
+                         "traffic_note": traffic_note,
                          "launches_per_step": dom_launches, "ms_per_step": dom_ms,
                          "layer_ms": [round(v, 4) for v in lms]},
         }
