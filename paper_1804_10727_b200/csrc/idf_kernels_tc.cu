@@ -1117,7 +1117,7 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
         const int units = p.n_mt * p.n_nt;
         int min_rows = 2 * a.ring_rows + 2;
         if (min_rows < 16) min_rows = 16;
-        static const bool no_chunks = getenv("IDF_NO_ROW_CHUNKS") != nullptr;
+        const bool no_chunks = getenv("IDF_NO_ROW_CHUNKS") != nullptr;     // (read per launch: tests switch it)
         // (a block that continues rows of an earlier one needs room for the copy of the ring, see ring_in)
         if (!no_chunks && units < 120 && t.n_orows >= 2 * min_rows && (a.r0 == 0 || a.ring_scratch)) {
             int want = (296 + units - 1) / units;
