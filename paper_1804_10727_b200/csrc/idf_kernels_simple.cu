@@ -174,23 +174,24 @@ cudaError_t launch_conv_simple(const ConvArgs& a, int dtype, cudaStream_t st)
 //   3. finalisation of the ring rows that this input row completed: emit f(c + b), zero the slot.
 // Rows still open at the end of the block go back to the ring in global memory.
 // ------------------------------------------------------------------------------------------------
-constexpr int SPARSE_THREADS = 256;
+constexpr int SPARSE_MAX_THREADS = 512;
 constexpr int SPARSE_MAX_EVENTS = 2048;   // list capacity per pass; longer rows take several passes
 
 template <typename TS> __device__ __forceinline__ void atomic_add(TS* p, TS v) { atomicAdd(p, v); }
 
 template <typename TI, typename TW, typename TS, typename TO, bool RING_IN_SMEM>
-__global__ void __launch_bounds__(SPARSE_THREADS) conv_sparse_kernel(ConvArgs a)
+__global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArgs a)
 {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ int ev_pos[SPARSE_MAX_EVENTS];      // x * Cin + ci
+    __shared__ short ev_x[SPARSE_MAX_EVENTS], ev_ci[SPARSE_MAX_EVENTS];   // position and channel of the event
     __shared__ TS ev_val[SPARSE_MAX_EVENTS];
     __shared__ int ev_count;
     __shared__ unsigned long long ev_total;
 
     const int s = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31;
+    const int SPARSE_THREADS = blockDim.x;      // 256, or 512 for wide rows (more warps to hide the finalisation's latency)
     const TI* __restrict__ in = (const TI*)a.in;
     const TW* __restrict__ w = (const TW*)a.w;
     const TS* __restrict__ bias = (const TS*)a.bias;
@@ -232,7 +233,9 @@ __global__ void __launch_bounds__(SPARSE_THREADS) conv_sparse_kernel(ConvArgs a)
                         off = __shfl_sync(0xffffffffu, off, 0);
                         if (v != (TS)0) {
                             const int k = off + __popc(m & ((1u << lane) - 1u));
-                            ev_pos[k] = i;
+                            const int x = i / a.Cin;
+                            ev_x[k] = (short)x;
+                            ev_ci[k] = (short)(i - x * a.Cin);
                             ev_val[k] = v;
                         }
                     }
@@ -240,25 +243,32 @@ __global__ void __launch_bounds__(SPARSE_THREADS) conv_sparse_kernel(ConvArgs a)
                 __syncthreads();
                 const int n_ev = ev_count;
                 if (tid == 0) ev_total += (unsigned long long)n_ev;
-                // scatter: item = (event, tap, co); consecutive threads differ in co.  All index
-                // arithmetic in 32 bits: for every tap row ky the target ring slot is worked out once.
-                const int items = n_ev * taps * a.Cout;
-                // relative target row of tap ky: (r + pad - ky) / stride when whole and not below o_begin
-                for (int it = tid; it < items; it += SPARSE_THREADS) {
-                    const int co = it % a.Cout;
-                    const int t2 = it / a.Cout;
-                    const int tap = t2 % taps, e = t2 / taps;
-                    const int ky = tap / a.Kw, kx = tap - ky * a.Kw;
-                    const int pos = ev_pos[e];
-                    const int x = pos / a.Cin, ci = pos - x * a.Cin;
-                    const int ty = (int)(r - a.o_begin * a.stride) + a.pad - ky;    // relative to row o_begin
-                    const int tx = x + a.pad_x - kx;
-                    if (ty < 0 || tx < 0) continue;
-                    const int orel = ty / a.stride, ox = tx / a.stride_x;
-                    if (orel * a.stride != ty || ox * a.stride_x != tx || ox >= a.Wout) continue;
-                    const int slot = (slot0 + orel) % a.ring_rows;
-                    const TS wv = (TS)to_acc(w[((ky * a.Kw + kx) * a.Cin + ci) * a.Cout + co]);
-                    atomic_add(&ring[ring_base + slot * slot_stride + ox * a.Cout + co], ev_val[e] * wv);
+                // scatter: a warp takes one event at a time and walks its kernel taps, the lanes take the output
+                // channels; target row, ring slot and target x are worked out once per tap row / tap (no
+                // per-channel index arithmetic, no division when the stride is 1)
+                const int ty0 = (int)(r - a.o_begin * a.stride) + a.pad;          // tap ky reaches relative row (ty0 - ky) / stride
+                for (int e = tid >> 5; e < n_ev; e += SPARSE_THREADS / 32) {
+                    const int x = ev_x[e], ci = ev_ci[e];
+                    const TS val = ev_val[e];
+                    for (int ky = 0; ky < a.Kh; ++ky) {
+                        const int ty = ty0 - ky;
+                        if (ty < 0) break;
+                        int orel = ty;
+                        if (a.stride != 1) { orel = ty / a.stride; if (orel * a.stride != ty) continue; }
+                        const int slot = (slot0 + orel) % a.ring_rows;
+                        TS* drow = &ring[ring_base + slot * slot_stride];
+                        const TW* wrow = w + ((long long)ky * a.Kw * a.Cin + ci) * a.Cout;
+                        for (int kx = 0; kx < a.Kw; ++kx) {
+                            const int tx = x + a.pad_x - kx;
+                            if (tx < 0) break;
+                            int ox = tx;
+                            if (a.stride_x != 1) { ox = tx / a.stride_x; if (ox * a.stride_x != tx) continue; }
+                            if (ox >= a.Wout) continue;
+                            const TW* wp = wrow + (long long)kx * a.Cin * a.Cout;
+                            TS* dst = drow + ox * a.Cout;
+                            for (int co = lane; co < a.Cout; co += 32) atomic_add(dst + co, val * (TS)to_acc(wp[co]));
+                        }
+                    }
                 }
                 __syncthreads();
             }
@@ -277,15 +287,18 @@ __global__ void __launch_bounds__(SPARSE_THREADS) conv_sparse_kernel(ConvArgs a)
             TO* orow = out + (done - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride;
             if (sizeof(TO) == 1 && (a.Cout & 3) == 0 && (((uintptr_t)orow) & 3) == 0) {
                 // int8 rows: four channels per thread, one 4-byte store
+                const bool pow2 = (a.Cout & (a.Cout - 1)) == 0;
                 for (int i = tid * 4; i < row_elems; i += SPARSE_THREADS * 4) {
                     TS* p = &ring[ring_base + slot * slot_stride + i];
-                    const int co = i % a.Cout;
+                    const int co = pow2 ? (i & (a.Cout - 1)) : i % a.Cout;
+                    // (16-byte accesses: the ring row starts on a 16-byte boundary and i is a multiple of 4)
+                    __align__(16) TS c[4];
+                    *(int4*)c = *(const int4*)p;
+                    *(int4*)p = make_int4(0, 0, 0, 0);
                     uint32_t pk = 0;
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const TS c = p[j];
-                        p[j] = 0;
-                        const TO v = Emit<TO, TS>::run(c, bias ? bias[co + j] : (TS)0, a.relu, a.shift);
+                        const TO v = Emit<TO, TS>::run(c[j], bias ? bias[co + j] : (TS)0, a.relu, a.shift);
                         pk |= ((uint32_t)(*(const unsigned char*)&v)) << (8 * j);
                     }
                     *(uint32_t*)(orow + i) = pk;
@@ -318,19 +331,22 @@ static cudaError_t launch_sparse_t(const ConvArgs& a, cudaStream_t st)
 {
     if (a.S == 0) return cudaSuccess;
     const size_t ring_bytes = (size_t)a.ring_rows * a.Wout * a.Cout * sizeof(TS);
+    const int nthr = (long long)a.Wout * a.Cout >= 4096 ? SPARSE_MAX_THREADS : 256;
     if (ring_bytes <= conv_sparse_max_smem()) {
         auto k = conv_sparse_kernel<TI, TW, TS, TO, true>;
         cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring_bytes);
         if (e != cudaSuccess) return e;
-        k<<<a.S, SPARSE_THREADS, ring_bytes, st>>>(a);
+        k<<<a.S, nthr, ring_bytes, st>>>(a);
     } else {
-        conv_sparse_kernel<TI, TW, TS, TO, false><<<a.S, SPARSE_THREADS, 0, st>>>(a);
+        conv_sparse_kernel<TI, TW, TS, TO, false><<<a.S, nthr, 0, st>>>(a);
     }
     return cudaGetLastError();
 }
 
 cudaError_t launch_conv_sparse(const ConvArgs& a, int dtype, cudaStream_t st)
 {
+    // (the event list keeps positions and channels in 16 bits; beyond that the dense kernel gives the same result)
+    if (a.Win > 32767 || a.Cin > 32767) return launch_conv_simple(a, dtype, st);
     if (dtype == 0) return launch_sparse_t<float, float, float, float>(a, st);
     if (dtype == 1) {
         if (a.in_elem != E_BF16) return cudaErrorInvalidValue;
