@@ -369,6 +369,7 @@ __global__ void __launch_bounds__(256) unfold_rows_kernel(const T* __restrict__ 
     constexpr int V = 16 / (int)sizeof(T);
     const int vecs = kpad / V;
     const long long total = n_pos * vecs;
+    const bool vec_ok = (Cin % V) == 0 && (((uintptr_t)in) & 15) == 0;     // channels of a position in whole 16-byte groups
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (long long)gridDim.x * blockDim.x) {
         const int v = (int)(idx % vecs);
@@ -377,6 +378,16 @@ __global__ void __launch_bounds__(256) unfold_rows_kernel(const T* __restrict__ 
         const long long rs = p / Wout;               // (row, stream)
         const T* row = in + rs * (long long)Win * Cin;
         __align__(16) T vals[V];
+        if (vec_ok) {
+            // a 16-byte group never straddles two taps: it is one aligned 16-byte piece of an input position
+            const int k0 = v * V;
+            const int kx = k0 / Cin, ci = k0 - kx * Cin;
+            const int ix = xo * stride_x - pad_x + kx;
+            int4 q = make_int4(0, 0, 0, 0);
+            if (kx < Kw && ix >= 0 && ix < Win) q = *(const int4*)(row + (long long)ix * Cin + ci);
+            *(int4*)(out + p * kpad + (long long)v * V) = q;
+            continue;
+        }
 #pragma unroll
         for (int j = 0; j < V; ++j) {
             const int k = v * V + j;
