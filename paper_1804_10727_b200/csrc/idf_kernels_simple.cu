@@ -388,12 +388,14 @@ __global__ void __launch_bounds__(256) unfold_rows_kernel(const T* __restrict__ 
             *(int4*)(out + p * kpad + (long long)v * V) = q;
             continue;
         }
+        // the Kw*Cin values of an output position are one contiguous run of the input row, starting at position
+        // xo*stride - pad: element k of the run lies outside the row exactly when its position does
+        const int e0 = (xo * stride_x - pad_x) * Cin + v * V;
+        const int k_end = Kw * Cin - v * V, e_end = Win * Cin;
 #pragma unroll
         for (int j = 0; j < V; ++j) {
-            const int k = v * V + j;
-            const int kx = k / Cin, ci = k - kx * Cin;
-            const int ix = xo * stride_x - pad_x + kx;
-            vals[j] = (kx < Kw && ix >= 0 && ix < Win) ? row[(long long)ix * Cin + ci] : (T)0;
+            const int e = e0 + j;
+            vals[j] = (j < k_end && e >= 0 && e < e_end) ? row[e] : (T)0;
         }
         *(int4*)(out + p * kpad + (long long)v * V) = *(const int4*)vals;
     }
