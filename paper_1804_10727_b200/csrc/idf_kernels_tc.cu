@@ -1120,7 +1120,7 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
         const bool no_chunks = getenv("IDF_NO_ROW_CHUNKS") != nullptr;     // (read per launch: tests switch it)
         // (a block that continues rows of an earlier one needs room for the copy of the ring, see ring_in)
         if (!no_chunks && units < 120 && t.n_orows >= 2 * min_rows && (a.r0 == 0 || a.ring_scratch)) {
-            int want = (296 + units - 1) / units;
+            int want = 296 / units;                                 // at most two full waves of CTAs on the 148 SMs
             if (want > t.n_orows / min_rows) want = t.n_orows / min_rows;
             if (want > 1) {
                 int rows = (t.n_orows + want - 1) / want;
