@@ -178,6 +178,32 @@ int idf_stream_status(idf_net* net, long long* tensor_core_launches);
 int idf_set_timing(idf_net* net, int on);
 int idf_layer_times(idf_net* net, double* ms, long long* launches);
 
+/* Checkpoint of running streams.  The paper's Discussion reads the method as a recurrent model whose
+ * hidden state is the set of partially computed activations; that state (all streams' ring rows and
+ * pooling rows) together with the per-layer row counters is everything a stream needs to go on, so
+ * it can be taken off the device between two pushes and put back later, on this handle or on
+ * another handle created from the same spec and parameters (another workspace, another GPU).
+ *
+ *   idf_state_snapshot_bytes  size of a snapshot of this net in bytes (0 if net is NULL): a small
+ *                             header plus the state of all streams (n_streams * idf_net_state_bytes,
+ *                             each layer rounded up to 256 bytes).
+ *   idf_state_save     h_snapshot: host, at least idf_state_snapshot_bytes, owned by the caller.
+ *                      Valid while streams are open (after open/reset/push, before finish), else
+ *                      IDF_ERR_STATE; IDF_ERR_CAPACITY if bytes is too small.  Copies on the handle's
+ *                      stream and waits for it.  The streams go on unchanged.
+ *   idf_state_restore  h_snapshot: host.  The handle must have a workspace bound (idf_stream_open);
+ *                      whatever streams it was running are abandoned and replaced by the saved ones,
+ *                      which are then open.  IDF_ERR_ARG if the buffer is not a snapshot or is
+ *                      truncated or inconsistent, IDF_ERR_SPEC if it was taken from a net of another
+ *                      shape (layers, types, widths, stream count).  Parameters are not part of a
+ *                      snapshot: the restoring handle uses its own.  Waits for the stream.
+ * Output rows completed before the snapshot are not written again: later pushes write the rows that
+ * follow, at their absolute row index, into whatever d_out the caller passes then.  Continuing from
+ * a snapshot gives bit-identical results to continuing without the interruption. */
+size_t idf_state_snapshot_bytes(const idf_net* net);
+int idf_state_save(idf_net* net, void* h_snapshot, size_t bytes);
+int idf_state_restore(idf_net* net, const void* h_snapshot, size_t bytes);
+
 /* One fp32 conv layer over whole streams, for callers that cannot allocate device memory.
  * (The paper has no counterpart to this call; it exists for deployment reasons only.)
  *

@@ -772,6 +772,111 @@ int idf_stream_status(idf_net* net, long long* tensor_core_launches)
     return IDF_OK;
 }
 
+// Snapshot of the streams' progress: a fixed header (what net it belongs to, how far every layer has
+// come) followed by the rolling state of all streams and the sparse-path event counters.
+namespace {
+struct SnapshotHeader {
+    unsigned long long magic;
+    unsigned long long fingerprint;        // of the net's shape: a snapshot only fits a net built from the same spec
+    unsigned long long state_region_bytes;
+    unsigned long long n_layers;
+    long long out_rows_total;
+};
+constexpr unsigned long long SNAPSHOT_MAGIC = 0x3154504e53464449ULL;      // "IDFSNPT1"
+
+unsigned long long mix(unsigned long long h, unsigned long long v)
+{
+    h ^= v + 0x9e3779b97f4a7c15ULL + (h << 6) + (h >> 2);
+    return h;
+}
+unsigned long long net_fingerprint(const idf_net* net)
+{
+    unsigned long long h = 0x1234;
+    for (long long v : {(long long)net->dtype, (long long)net->in_w, (long long)net->in_c, (long long)net->n_streams, (long long)net->L.size()})
+        h = mix(h, (unsigned long long)v);
+    for (const auto& P : net->L) {
+        const idf_layer& l = P.l;
+        for (long long v : {(long long)l.kind, (long long)l.cin, (long long)l.cout, (long long)l.kh, (long long)l.kw, (long long)l.stride,
+                            (long long)l.pad, (long long)l.relu, (long long)l.shift, (long long)P.use_sparse, (long long)P.state_bytes_all})
+            h = mix(h, (unsigned long long)v);
+    }
+    return h;
+}
+size_t snapshot_bytes(const idf_net* net)
+{
+    return sizeof(SnapshotHeader) + net->L.size() * 3 * sizeof(long long) + net->state_region_bytes;
+}
+}  // namespace
+
+size_t idf_state_snapshot_bytes(const idf_net* net) { return net ? snapshot_bytes(net) : 0; }
+
+int idf_state_save(idf_net* net, void* h_snapshot, size_t bytes)
+{
+    if (!net || !h_snapshot) return fail(IDF_ERR_ARG, "net and h_snapshot must not be NULL");
+    if (net->phase != OPEN) return fail(IDF_ERR_STATE, "state_save needs open streams (after open/reset/push, before finish)");
+    if (bytes < snapshot_bytes(net)) return fail(IDF_ERR_CAPACITY, "snapshot needs %zu bytes, %zu given", snapshot_bytes(net), bytes);
+    for (const auto& P : net->L)
+        if (P.pending != 0) return fail(IDF_ERR_STATE, "internal: rows in flight between layers");   // (a push leaves none behind)
+    unsigned char* p = (unsigned char*)h_snapshot;
+    SnapshotHeader h{SNAPSHOT_MAGIC, net_fingerprint(net), net->state_region_bytes, net->L.size(), net->out_rows_total};
+    memcpy(p, &h, sizeof h);
+    p += sizeof h;
+    long long* prog = (long long*)p;                     // per layer: rows received, rows emitted, events applied
+    for (size_t i = 0; i < net->L.size(); ++i) { prog[3 * i] = net->L[i].rows_in; prog[3 * i + 1] = net->L[i].rows_done; }
+    std::vector<unsigned long long> ev(net->L.size());
+    cudaError_t e = cudaMemcpyAsync(ev.data(), net->ws + net->counters_off, ev.size() * sizeof(unsigned long long),
+                                    cudaMemcpyDeviceToHost, net->stream);
+    p += net->L.size() * 3 * sizeof(long long);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(p, net->ws + net->state_region_off, net->state_region_bytes, cudaMemcpyDeviceToHost, net->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(net->stream);
+    if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "state_save: %s", cudaGetErrorString(e));
+    for (size_t i = 0; i < net->L.size(); ++i) prog[3 * i + 2] = (long long)ev[i];
+    return IDF_OK;
+}
+
+int idf_state_restore(idf_net* net, const void* h_snapshot, size_t bytes)
+{
+    if (!net || !h_snapshot) return fail(IDF_ERR_ARG, "net and h_snapshot must not be NULL");
+    if (net->phase == CREATED) return fail(IDF_ERR_STATE, "state_restore before stream_open");
+    if (bytes < sizeof(SnapshotHeader)) return fail(IDF_ERR_ARG, "not a snapshot (too short)");
+    SnapshotHeader h;
+    memcpy(&h, h_snapshot, sizeof h);
+    if (h.magic != SNAPSHOT_MAGIC) return fail(IDF_ERR_ARG, "not a snapshot (bad magic)");
+    if (h.fingerprint != net_fingerprint(net) || h.n_layers != net->L.size() || h.state_region_bytes != net->state_region_bytes)
+        return fail(IDF_ERR_SPEC, "the snapshot was taken from a net with a different spec or stream count");
+    if (bytes < snapshot_bytes(net)) return fail(IDF_ERR_ARG, "snapshot truncated: %zu of %zu bytes", bytes, snapshot_bytes(net));
+    const unsigned char* p = (const unsigned char*)h_snapshot + sizeof h;
+    const long long* prog = (const long long*)p;
+    // the progress record must be one the schedule can produce: every layer has emitted exactly the rows
+    // complete after its input rows, and its successor has received them all
+    long long r = prog[0];
+    if (r < 0) return fail(IDF_ERR_ARG, "snapshot corrupt (negative row count)");
+    for (size_t i = 0; i < net->L.size(); ++i) {
+        if (prog[3 * i] != r) return fail(IDF_ERR_ARG, "snapshot corrupt (layer %zu row count)", i);
+        r = layer_done_after(net->L[i], r);
+        if (prog[3 * i + 1] != r) return fail(IDF_ERR_ARG, "snapshot corrupt (layer %zu rows emitted)", i);
+    }
+    if (h.out_rows_total != r) return fail(IDF_ERR_ARG, "snapshot corrupt (output row count)");
+    p += net->L.size() * 3 * sizeof(long long);
+    std::vector<unsigned long long> ev(net->L.size());
+    for (size_t i = 0; i < net->L.size(); ++i) ev[i] = (unsigned long long)prog[3 * i + 2];
+    cudaError_t e = cudaMemsetAsync(net->ws + net->status_off, 0, sizeof(unsigned int), net->stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(net->ws + net->state_region_off, p, net->state_region_bytes, cudaMemcpyHostToDevice, net->stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(net->ws + net->counters_off, ev.data(), ev.size() * sizeof(unsigned long long), cudaMemcpyHostToDevice, net->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(net->stream);      // (ev and possibly the caller's buffer are pageable)
+    if (e != cudaSuccess) { net->phase = CREATED; return fail(IDF_ERR_CUDA, "state_restore: %s", cudaGetErrorString(e)); }
+    for (size_t i = 0; i < net->L.size(); ++i) {
+        LayerPlan& P = net->L[i];
+        P.rows_in = prog[3 * i]; P.rows_done = prog[3 * i + 1]; P.pending = 0;
+    }
+    net->out_rows_total = h.out_rows_total;
+    net->phase = OPEN;
+    return IDF_OK;
+}
+
 int idf_set_timing(idf_net* net, int on)
 {
     if (!net) return fail(IDF_ERR_ARG, "net must not be NULL");

@@ -28,6 +28,7 @@ EXPORTS = (
     "idf_net_create", "idf_net_destroy", "idf_net_state_bytes", "idf_net_workspace_bytes", "idf_out_shape",
     "idf_stream_open", "idf_stream_reset", "idf_stream_push", "idf_stream_push_last", "idf_stream_finish", "idf_run_host", "idf_event_counts",
     "idf_launch_count", "idf_stream_status", "idf_set_timing", "idf_layer_times", "idf_conv_rows_noalloc", "idf_last_error",
+    "idf_state_snapshot_bytes", "idf_state_save", "idf_state_restore",
 )
 
 
@@ -76,6 +77,9 @@ def lib():
         L.idf_conv_rows_noalloc.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp,
                                             ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                             ctypes.c_int, vp, ll, ctypes.POINTER(ll), vp]
+        L.idf_state_snapshot_bytes.argtypes = [vp]; L.idf_state_snapshot_bytes.restype = sz
+        L.idf_state_save.argtypes = [vp, vp, sz]
+        L.idf_state_restore.argtypes = [vp, vp, sz]
         L.idf_last_error.restype = ctypes.c_char_p
         _lib = L
     return _lib
@@ -237,6 +241,17 @@ class Net:
         _check(lib().idf_run_host(self._h, h_segments.data_ptr(), h_segments.shape[0], d_segments.data_ptr(),
                                   h_out.data_ptr(), d_out.data_ptr(), d_out.shape[1], ctypes.byref(tot)))
         return int(tot.value)
+
+    def save_state(self) -> torch.Tensor:
+        """Snapshot of the open streams (host uint8 tensor); see idf_state_save."""
+        buf = torch.empty(int(lib().idf_state_snapshot_bytes(self._h)), dtype=torch.uint8)
+        _check(lib().idf_state_save(self._h, buf.data_ptr(), buf.numel()))
+        return buf
+
+    def restore_state(self, snapshot: torch.Tensor):
+        """Replace this handle's streams by the saved ones; see idf_state_restore."""
+        assert not snapshot.is_cuda and snapshot.dtype == torch.uint8 and snapshot.is_contiguous()
+        _check(lib().idf_state_restore(self._h, snapshot.data_ptr(), snapshot.numel()))
 
     def close(self):
         if self._h:

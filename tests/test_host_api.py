@@ -113,6 +113,22 @@ def test_bad_arguments_and_call_order():
     assert L.idf_stream_open(net._h, 257, 1 << 30, None) == idf.ERR_ARG    # misaligned workspace
 
 
+def test_snapshot_size_and_call_order():
+    L = idf.lib()
+    assert L.idf_state_snapshot_bytes(None) == 0
+    w = workloads.get("mnist2d", n_streams=3)
+    net = idf.net_from_workload(w, *workloads.make_params(w))
+    n = L.idf_state_snapshot_bytes(net._h)
+    # header + three words per layer + every layer's state of all streams, each rounded up to 256 bytes
+    assert 3 * net.state_bytes <= n <= 3 * net.state_bytes + 256 * len(w.layers) + 64 + 24 * len(w.layers)
+    buf = (ctypes.c_ubyte * n)()
+    assert L.idf_state_save(None, buf, n) == idf.ERR_ARG
+    assert L.idf_state_save(net._h, None, n) == idf.ERR_ARG
+    assert L.idf_state_save(net._h, buf, n) == idf.ERR_STATE            # no open streams
+    assert L.idf_state_restore(net._h, buf, n) == idf.ERR_STATE          # no workspace bound
+    assert L.idf_state_restore(net._h, None, n) == idf.ERR_ARG
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(idf, "_lib", None)
     monkeypatch.setattr(idf, "LIB_PATH", tmp_path / "libidf.so")
