@@ -50,7 +50,21 @@ typedef enum {
                        /* q = clamp((c + 2^(shift-1)) >> shift, relu ? 0 : -127, 127); output int8   */
 } idf_dtype;
 
-typedef enum { IDF_CONV = 0, IDF_MAXPOOL2 = 1 } idf_kind;   /* 2x2 max pool, stride 2, floor; rows only when width is 1 */
+typedef enum {
+    IDF_CONV = 0,
+    IDF_MAXPOOL2 = 1,    /* 2x2 max pool, stride 2, floor; rows only when width is 1 */
+    IDF_GLOBAL_AVG = 2   /* output sink, last layer only: the averaging output unit of the paper's Fig. 1.  Every value
+                            arriving from the layer below is added to one running sum per stream and channel
+                            (c_out += dh, Eq. 4 with weight 1; 4 bytes of state per channel).  The net's output is then
+                            ONE row [n_streams][out_capacity_rows >= 1][1][C] of fp32 (for every idf_dtype; for int
+                            nets the exact int32 sum divided in double precision and rounded once): the mean over all
+                            positions received so far.  It is rewritten by every push that brings it new rows, so it
+                            can be read between pushes (the paper's output that converges while the input arrives,
+                            Section "Experimental verification"), and is final after idf_stream_finish. */
+} idf_kind;
+/* A fully connected output layer over a map of known size H x W x C (the paper's 10 output units) is an IDF_CONV layer
+ * with kh = H, kw = W, stride = H, pad = 0 and weights [n_out][H][W][C]: one output row of width 1, one ring row of
+ * state, and every arriving row adds its share w * dh at once. */
 typedef enum { IDF_PATH_AUTO = 0, IDF_PATH_DENSE = 1, IDF_PATH_SPARSE = 2 } idf_path;
 
 typedef enum {

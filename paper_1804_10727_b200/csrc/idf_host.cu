@@ -110,13 +110,14 @@ long long conv_rows_at_flush(const idf_layer& l, long long rows_in)
     return q < 0 ? 0 : q / l.stride + 1;
 }
 
+// (a global-average sink has one output row, rewritten with the running mean whenever rows arrive)
 long long layer_done_after(const LayerPlan& P, long long rows_in)
 {
-    return P.l.kind == IDF_CONV ? conv_done_after(P.l, rows_in) : rows_in / 2;
+    return P.l.kind == IDF_CONV ? conv_done_after(P.l, rows_in) : P.l.kind == IDF_MAXPOOL2 ? rows_in / 2 : (rows_in > 0 ? 1 : 0);
 }
 long long layer_rows_at_flush(const LayerPlan& P, long long rows_in)
 {
-    return P.l.kind == IDF_CONV ? conv_rows_at_flush(P.l, rows_in) : rows_in / 2;
+    return P.l.kind == IDF_CONV ? conv_rows_at_flush(P.l, rows_in) : P.l.kind == IDF_MAXPOOL2 ? rows_in / 2 : (rows_in > 0 ? 1 : 0);
 }
 
 // Enqueue one layer on n_in input rows found at in_ptr (slots 0..n_in-1).  With `flush` (n_in == 0)
@@ -134,9 +135,11 @@ int launch_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, boo
         done_end = flush ? conv_rows_at_flush(P.l, r1) : conv_done_after(P.l, r1);
         const long long started = r1 > 0 ? (r1 - 1 + P.l.pad) / P.l.stride + 1 : 0;   // rows reached so far
         o_end = std::max(started, done_end);
-    } else {
+    } else if (P.l.kind == IDF_MAXPOOL2) {
         done_end = r1 / 2;
         o_end = (r1 + 1) / 2;
+    } else {
+        done_end = o_end = r1 > 0 ? 1 : 0;
     }
     const long long o_begin = P.rows_done;
     if (done_end < o_begin) done_end = o_begin;
@@ -208,6 +211,15 @@ int launch_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, boo
         }
         if (ce == cudaErrorNotSupported)
             ce = P.use_sparse ? launch_conv_sparse(a, net->dtype, net->stream) : launch_conv_simple(a, net->dtype, net->stream);
+    } else if (P.l.kind == IDF_GLOBAL_AVG) {
+        AvgArgs a{};
+        a.in = in_ptr;
+        a.sum = net->ws + P.state_off;
+        a.out = (float*)out_ptr;
+        a.out_stream_stride = stream_stride;
+        a.S = (int)S; a.W = P.in_w; a.C = P.in_c; a.elem = P.in_elem;
+        a.n_rows = n_in; a.rows_total = r1;
+        ce = launch_avg(a, net->stream);
     } else {
         PoolArgs a{};
         a.in = in_ptr;
@@ -553,6 +565,14 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
             P.use_sparse = 0;
             P.state_bytes_stream = (size_t)P.out_w * P.out_c * elem_size(elem);
             cap = std::max(2 * net->row_block + 8, cap / 2 + 1);
+        } else if (l.kind == IDF_GLOBAL_AVG) {
+            if (i + 1 != spec->n_layers) { delete net; return fail(IDF_ERR_SPEC, "layer %d: a global-average sink must be the last layer", i); }
+            P.out_w = 1;
+            P.out_c = c;
+            P.ring_rows = 1;
+            P.out_elem = E_F32;
+            P.use_sparse = 0;
+            P.state_bytes_stream = (size_t)c * state_word;      // one running sum per channel
         } else {
             delete net;
             return fail(IDF_ERR_SPEC, "layer %d: unknown kind %d", i, l.kind);
@@ -626,7 +646,7 @@ int idf_out_shape(const idf_net* net, long long in_rows, long long* out_rows, in
     if (!net) return fail(IDF_ERR_ARG, "net must not be NULL");
     if (in_rows < 0) return fail(IDF_ERR_ARG, "in_rows must not be negative");
     long long h = in_rows;
-    for (const auto& P : net->L) h = P.l.kind == IDF_CONV ? conv_rows_at_flush(P.l, h) : h / 2;
+    for (const auto& P : net->L) h = layer_rows_at_flush(P, h);
     if (out_rows) *out_rows = h;
     if (out_w) *out_w = net->L.back().out_w;
     if (out_c) *out_c = net->L.back().out_c;

@@ -51,6 +51,18 @@ struct PoolArgs {
     long long r0, r1, o_begin, o_end, done_end;
 };
 
+// Global-average sink: every arriving row is added into one running sum per (stream, channel); the
+// output row holds the mean over all positions received so far.
+struct AvgArgs {
+    const void* in;        // [n_rows][S][W][C] in the element type `elem`
+    void* sum;             // [S][C] state words (fp32, or int32 for E_I8 rows)
+    float* out;            // mean of stream s at out + s * out_stream_stride, C floats
+    long long out_stream_stride;
+    int S, W, C, elem;
+    long long n_rows;      // rows arriving in this launch
+    long long rows_total;  // rows received since open, these included
+};
+
 // Static plan of the tensor-core path for one conv layer (tile shapes, shared-memory budget).
 struct TcPlan {
     int ok = 0;
@@ -85,6 +97,7 @@ cudaError_t launch_unfold(const ConvArgs& a, int n_rows, int kpad, void* out, cu
 cudaError_t launch_conv_simple(const ConvArgs& a, int dtype, cudaStream_t st);
 cudaError_t launch_conv_sparse(const ConvArgs& a, int dtype, cudaStream_t st);
 cudaError_t launch_pool(const PoolArgs& a, cudaStream_t st);
+cudaError_t launch_avg(const AvgArgs& a, cudaStream_t st);
 size_t conv_sparse_max_smem();
 
 }  // namespace idf

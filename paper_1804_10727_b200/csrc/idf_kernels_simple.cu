@@ -547,4 +547,50 @@ cudaError_t launch_pool(const PoolArgs& a, cudaStream_t st)
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Global-average sink (the averaging output unit of the paper's Fig. 1): c_out += dh for every
+// arriving value, one running sum per (stream, channel); the mean over the positions received so
+// far is written after every launch, so the output can be read at any time.
+// One thread per (stream, channel); channels are innermost, so a warp reads consecutive addresses.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float avg_term(float v) { return v; }
+__device__ __forceinline__ float avg_term(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ int avg_term(int8_t v) { return (int)v; }
+
+template <typename TI, typename TS>
+__global__ void __launch_bounds__(256) avg_rows_kernel(AvgArgs a)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const TI* __restrict__ in = (const TI*)a.in;
+    TS* sum = (TS*)a.sum;
+    const long long total = (long long)a.S * a.C;
+    const double count = (double)a.rows_total * (double)a.W;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(idx % a.C);
+        const long long s = idx / a.C;
+        TS acc = sum[idx];
+        for (long long r = 0; r < a.n_rows; ++r) {
+            const TI* row = in + (r * a.S + s) * (long long)a.W * a.C + c;
+            for (int x = 0; x < a.W; ++x) acc += avg_term(row[(long long)x * a.C]);
+        }
+        sum[idx] = acc;
+        a.out[s * a.out_stream_stride + c] = (float)((double)acc / count);
+    }
+}
+cudaError_t launch_avg(const AvgArgs& a, cudaStream_t st)
+{
+    const long long total = (long long)a.S * a.C;
+    if (total == 0 || a.n_rows <= 0) return cudaSuccess;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148LL * 32) blocks = 148LL * 32;
+    switch (a.elem) {
+        case E_F32: avg_rows_kernel<float, float><<<(unsigned)blocks, 256, 0, st>>>(a); break;
+        case E_BF16: avg_rows_kernel<__nv_bfloat16, float><<<(unsigned)blocks, 256, 0, st>>>(a); break;
+        case E_I8: avg_rows_kernel<int8_t, int><<<(unsigned)blocks, 256, 0, st>>>(a); break;
+        default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
 }  // namespace idf

@@ -18,7 +18,7 @@ LIB_PATH = _HERE / "libidf.so"
 _lib = None
 
 F32, BF16_F32, I8_I32 = 0, 1, 2
-CONV, MAXPOOL2 = 0, 1
+CONV, MAXPOOL2, GLOBAL_AVG = 0, 1, 2
 PATH_AUTO, PATH_DENSE, PATH_SPARSE = 0, 1, 2
 DTYPES = {"f32": F32, "bf16": BF16_F32, "i8": I8_I32}
 
@@ -91,7 +91,7 @@ def _check(rc: int):
 
 
 def _layer_struct(l) -> IdfLayer:
-    kind = l.kind if isinstance(l.kind, int) else {"conv": CONV, "pool": MAXPOOL2}[l.kind]
+    kind = l.kind if isinstance(l.kind, int) else {"conv": CONV, "pool": MAXPOOL2, "avg": GLOBAL_AVG}[l.kind]
     return IdfLayer(kind, l.cin, l.cout, l.kh, l.kw, l.stride, l.pad, l.relu, l.shift, l.path)
 
 
@@ -137,6 +137,7 @@ class Net:
         self._h = h
         self._ws = None
         self.n_layers = n
+        self._avg_sink = int(self._layers[n - 1].kind) == GLOBAL_AVG
 
     # -- queries ---------------------------------------------------------------------------------
     @property
@@ -154,7 +155,7 @@ class Net:
 
     @property
     def out_torch_dtype(self):
-        return torch.int8 if self.dtype == I8_I32 else torch.float32
+        return torch.int8 if self.dtype == I8_I32 and not self._avg_sink else torch.float32
 
     @property
     def act_torch_dtype(self):

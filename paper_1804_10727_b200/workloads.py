@@ -38,7 +38,7 @@ BLOCK = 32  # streams per generator block
 
 @dataclass(frozen=True)
 class Layer:
-    kind: str = "conv"          # 'conv' | 'pool'
+    kind: str = "conv"          # 'conv' | 'pool' | 'avg' (global-average output sink, last layer only)
     cin: int = 0
     cout: int = 0
     kh: int = 1

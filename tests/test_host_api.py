@@ -64,6 +64,24 @@ def test_fig1_ring_count_is_seven():
     seven = int([l for l in open(os.path.join(ROOT, "tests", "golden", "fig1_state_count.txt")) if l[0] != "#"][0])
     net = _mk((conv(1, 1, 3, one_d=True), conv(1, 1, 3, one_d=True)), in_w=1)
     assert net.state_bytes // 4 + 1 == seven
+    # ... and with the averaging unit as the library's global-average sink the count is the library's own
+    net = _mk((conv(1, 1, 3, one_d=True), conv(1, 1, 3, one_d=True), Layer("avg")), in_w=1)
+    assert net.state_bytes == 4 * seven
+
+
+def test_sink_layers_shapes_and_state():
+    # global average: one output row of width 1, one state word per channel, only as the last layer
+    net = _mk((conv(2, 6, 3), POOL, Layer("avg")), in_w=12, in_c=2)
+    assert net.out_shape(0) == (0, 1, 6) and net.out_shape(5) == (1, 1, 6) and net.out_shape(500) == (1, 1, 6)
+    assert net.state_bytes == 3 * 10 * 6 * 4 + 5 * 6 * 4 + 6 * 4
+    with pytest.raises(idf.IdfError) as e:
+        _mk((conv(2, 6, 3), Layer("avg"), conv(6, 2, 3)), in_w=12, in_c=2)
+    assert e.value.code == idf.ERR_SPEC
+    # a fully connected layer over a 7 x 9 x 6 map is a conv layer with kh = 7, kw = 9, stride = 7: one ring row
+    fc = Layer("conv", 6, 10, 7, 9, 7, 0, 0, 0, 0)
+    net = _mk((conv(2, 6, 3), fc), in_w=11, in_c=2)
+    assert net.out_shape(9) == (1, 1, 10) and net.out_shape(8) == (0, 1, 10)
+    assert net.state_bytes == 3 * 9 * 6 * 4 + 10 * 4
 
 
 def test_out_shape_follows_the_floor_formula():

@@ -294,3 +294,37 @@ def test_causality_rows_do_not_depend_on_later_input(orc):
     safe = [o for o in range(full.shape[0]) if 4 * o + 6 <= 9]
     assert safe and np.array_equal(full[safe], alt[safe])
     assert not np.array_equal(full, alt)
+
+
+@pytest.mark.parametrize("mode", ["f32", "i8"])
+def test_output_sinks_reduce_to_matrix_product_and_mean(orc, mode):
+    """A fully connected output layer is the conv layer whose kernel covers the whole map (one output position):
+    it must equal a matrix-vector product over the flattened map; the global-average sink must equal the exact
+    rational mean; and the event-by-event checker must reach both."""
+    H, W, C, n_out = 5, 4, 3, 6
+    fc = Layer("conv", C, n_out, H, W, H, 0, 0, 9 if mode == "i8" else 0, 0)
+    x, ws, bs = _rand_net(mode, (fc,), H, W, C, S=3, seed=8)
+    got = orc.forward(mode, (fc,), x, ws, bs)
+    assert got.shape == (3, 1, 1, n_out)
+    flat = torch.tensor(np.asarray(x, dtype=np.float64).reshape(3, -1))
+    wmat = torch.tensor(np.asarray(ws[0], dtype=np.float64).reshape(n_out, -1))
+    lin = torch.nn.functional.linear(flat, wmat, torch.tensor(np.asarray(bs[0], dtype=np.float64))).numpy()
+    if mode == "i8":
+        lin = np.clip(np.floor((lin + 2 ** 8) / 2 ** 9), -127, 127)
+        assert np.array_equal(got.reshape(3, n_out), lin.astype(np.int64))
+    else:
+        np.testing.assert_allclose(got.reshape(3, n_out), lin, rtol=1e-12, atol=1e-12)
+    ev = orc.event_run(mode, (fc,), x[0], ws, bs, eager=True)
+    np.testing.assert_allclose(ev["out"].reshape(-1), got[0].reshape(-1), rtol=1e-10, atol=1e-10)
+    # global average behind a conv layer: exact fractions
+    from fractions import Fraction
+    layers = (conv(C, 2, 3, shift=7 if mode == "i8" else 0), Layer("avg"))
+    x, ws, bs = _rand_net(mode, layers, 6, 5, C, S=2, seed=9)
+    maps = orc.forward(mode, layers, x, ws, bs, return_all=True)
+    pre, avg = maps[-2], maps[-1]
+    assert avg.shape == (2, 1, 1, 2)
+    for s in range(2):
+        for c in range(2):
+            vals = pre[s, :, :, c].reshape(-1)
+            exact = sum(Fraction(float(v)) for v in vals) / len(vals)
+            assert abs(Fraction(float(avg[s, 0, 0, c])) - exact) <= abs(exact) * Fraction(1, 10 ** 12)
