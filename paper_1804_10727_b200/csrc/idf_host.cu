@@ -83,6 +83,9 @@ struct idf_net {
     struct Timed { int layer; cudaEvent_t a, b; };
     std::vector<Timed> timed;
     std::vector<cudaEvent_t> event_pool;
+    // idf_run_host: copy streams and ordering events, made at the first call (no device memory involved)
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    std::vector<cudaEvent_t> order_events;
 };
 
 namespace {
@@ -632,6 +635,9 @@ int idf_net_destroy(idf_net* net)
     if (net) {
         for (auto& t : net->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
         for (auto e : net->event_pool) cudaEventDestroy(e);
+        for (auto e : net->order_events) cudaEventDestroy(e);
+        if (net->copy_in) cudaStreamDestroy(net->copy_in);
+        if (net->copy_out) cudaStreamDestroy(net->copy_out);
     }
     delete net;
     return IDF_OK;
@@ -750,17 +756,66 @@ int idf_run_host(idf_net* net, const void* h_segments, int n_seg, void* d_segmen
     if (!net || !h_segments || !d_segments || !h_out || !d_out) return fail(IDF_ERR_ARG, "NULL argument");
     if (net->phase != OPEN || net->L[0].rows_in != 0) return fail(IDF_ERR_STATE, "run_host needs a freshly opened handle");
     if (n_seg < 0) return fail(IDF_ERR_ARG, "negative count");
-    const size_t in_bytes = (size_t)n_seg * net->n_streams * net->in_w * net->in_c * elem_size(net->L[0].in_elem);
-    cudaError_t e = cudaMemcpyAsync(d_segments, h_segments, in_bytes, cudaMemcpyHostToDevice, net->stream);
-    if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "run_host h2d: %s", cudaGetErrorString(e));
-    long long tot = 0;
-    int rc = idf_stream_push_last(net, d_segments, n_seg, d_out, out_capacity_rows, &tot);
-    if (rc != IDF_OK) return rc;
+    // Pipeline over row blocks: while block b is computed on the handle's stream, block b + 1 travels to the
+    // device on a second stream and the output rows block b - 1 completed travel back on a third.
+    const long long nb = n_seg > 0 ? (n_seg + net->row_block - 1) / net->row_block : 1;
+    if (!net->copy_in) {
+        if (cudaStreamCreateWithFlags(&net->copy_in, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&net->copy_out, cudaStreamNonBlocking) != cudaSuccess)
+            return fail(IDF_ERR_CUDA, "run_host: cannot create the copy streams");
+    }
+    while ((long long)net->order_events.size() < 2 * nb + 1) {
+        cudaEvent_t e;
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return fail(IDF_ERR_CUDA, "cudaEventCreate failed");
+        net->order_events.push_back(e);
+    }
     const LayerPlan& P = net->L.back();
-    const size_t out_bytes = (size_t)net->n_streams * out_capacity_rows * P.out_w * P.out_c * elem_size(P.out_elem);
-    e = cudaMemcpyAsync(h_out, d_out, out_bytes, cudaMemcpyDeviceToHost, net->stream);
+    const size_t seg_bytes = (size_t)net->n_streams * net->in_w * net->in_c * elem_size(net->L[0].in_elem);
+    const size_t orow_bytes = (size_t)P.out_w * P.out_c * elem_size(P.out_elem);
+    const size_t opitch = (size_t)out_capacity_rows * orow_bytes;
+    cudaError_t e = cudaEventRecord(net->order_events[0], net->stream);      // earlier work on the caller's stream comes first
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(net->copy_in, net->order_events[0], 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(net->copy_out, net->order_events[0], 0);
+    if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "run_host: %s", cudaGetErrorString(e));
+    long long tot = 0, copied = 0;
+    for (long long b = 0; b < nb; ++b) {
+        const long long s0 = b * net->row_block, n = std::min<long long>(net->row_block, n_seg - s0);
+        const bool last_block = b + 1 == nb;
+        cudaEvent_t ev_in = net->order_events[1 + 2 * b], ev_done = net->order_events[2 + 2 * b];
+        if (n > 0) {
+            e = cudaMemcpyAsync((unsigned char*)d_segments + (size_t)s0 * seg_bytes, (const unsigned char*)h_segments + (size_t)s0 * seg_bytes,
+                                (size_t)n * seg_bytes, cudaMemcpyHostToDevice, net->copy_in);
+            if (e == cudaSuccess) e = cudaEventRecord(ev_in, net->copy_in);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(net->stream, ev_in, 0);
+            if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "run_host h2d: %s", cudaGetErrorString(e));
+        }
+        const void* blk = (const unsigned char*)d_segments + (size_t)s0 * seg_bytes;
+        int rc;
+        if (last_block) {
+            rc = idf_stream_push_last(net, blk, (int)std::max<long long>(n, 0), d_out, out_capacity_rows, &tot);
+        } else {
+            int em = 0;
+            rc = idf_stream_push(net, blk, (int)n, d_out, out_capacity_rows, &em);
+            tot = net->out_rows_total;
+        }
+        if (rc != IDF_OK) { cudaStreamSynchronize(net->copy_in); cudaStreamSynchronize(net->copy_out); return rc; }
+        // (a global-average sink rewrites its one row with every push: it travels once, at the end)
+        if (tot > copied && (P.l.kind != IDF_GLOBAL_AVG || last_block)) {
+            // output rows [copied, tot) of every stream: a strided copy (one run of rows per stream)
+            e = cudaEventRecord(ev_done, net->stream);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(net->copy_out, ev_done, 0);
+            if (e == cudaSuccess)
+                e = cudaMemcpy2DAsync((unsigned char*)h_out + (size_t)copied * orow_bytes, opitch,
+                                      (const unsigned char*)d_out + (size_t)copied * orow_bytes, opitch,
+                                      (size_t)(tot - copied) * orow_bytes, (size_t)net->n_streams, cudaMemcpyDeviceToHost, net->copy_out);
+            if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "run_host d2h: %s", cudaGetErrorString(e));
+            copied = tot;
+        }
+    }
+    e = cudaStreamSynchronize(net->copy_out);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(net->copy_in);
     if (e == cudaSuccess) e = cudaStreamSynchronize(net->stream);
-    if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "run_host d2h: %s", cudaGetErrorString(e));
+    if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "run_host: %s", cudaGetErrorString(e));
     if (total_rows) *total_rows = tot;
     return IDF_OK;
 }

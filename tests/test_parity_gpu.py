@@ -269,3 +269,29 @@ def test_bf16_workloads_layer_by_layer_strict(orc, name, S, H):
         got = idf.infer(net, a)
         assert_close(got, want, f"{name} layer {i}")
         net.close()
+
+
+# ---- idf_run_host: host buffers in and out, copies pipelined with the compute ---------------------
+@pytest.mark.parametrize("name,mode,rb", [("same_pool", "f32", 4), ("stride2", "i8", 3), ("oned_k9", "f32", 16), ("valid3", "bf16", 0)])
+def test_run_host_equals_device_path(orc, name, mode, rb):
+    layers = SMALL_NETS[name]
+    if mode == "i8":
+        layers = with_shifts(layers, 8)
+    H, W = small_dims(name)
+    C0 = next(l.cin for l in layers if l.kind == "conv")
+    x, ws, bs = rand_net(mode, layers, H, W, C0, S=5, seed=21)
+    ref, _ = _run(mode, layers, x, ws, bs, row_block=rb, chunks=[rb] * H if rb else None, last=True)
+    net = idf.Net(mode, layers, W, C0, 5, ws, bs, row_block=rb)
+    h_seg = idf.segments_from_maps(x, net.dtype).pin_memory()
+    d_seg = torch.empty_like(h_seg, device="cuda")
+    d_out = net.alloc_out(H)
+    h_out = torch.full(d_out.shape, 77, dtype=d_out.dtype).pin_memory()
+    net.open()
+    for _ in range(2):                                  # twice: the second call reuses streams, events and buffers
+        net.reset()
+        h_out.fill_(77)
+        rows = net.run_host(h_seg, d_seg, h_out, d_out)
+        net.status()
+        assert rows == ref.shape[1]
+        assert np.array_equal(h_out[:, :rows].numpy().view(np.uint8), ref.view(np.uint8)), (name, mode)
+    net.close()
