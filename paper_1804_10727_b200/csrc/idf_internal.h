@@ -69,6 +69,7 @@ struct TcPlan {
     int BX = 0, BS = 0;      // a 128-row M tile = BS streams x BX consecutive x positions
     int BXP = 0;             // positions per stream held in the shared-memory tile (BX + kx halo)
     int shift_mode = 0;      // kx taps read one haloed tile at row offsets instead of one box per kx
+    int sx = 1;              // x stride (> 1 only without shift_mode: the tensor map walks the input row in steps of sx)
     int a_stage_bytes = 0;
     int n_xt = 0, n_mt = 0;  // x tiles per row, M tiles in all
     int Ntile = 0, n_nt = 0; // output channels per CTA, N tiles

@@ -458,6 +458,8 @@ struct TcArgs {
     int S, Wout, Cout, Kh, Kw, stride, pad_x, relu, shift, ring_rows, out_elem;
     int BX, BXP, BS, n_xt, Ntile, n_nt, KB, n_kb, swb, nslot, nstage, tmem_cols;
     int shift_mode;              // 1: one box per (row, K block) holds the kx halo, taps address it at row offsets
+    int sx;                      // x stride of the conv (1, or more when every kx tap has a box of its own: the tensor map then
+                                 // walks the input row in steps of sx, so a box still holds BXP consecutive OUTPUT positions)
     int n_chunks, chunk_rows, chunk_shift;   // the block's output rows are cut into n_chunks runs of chunk_rows rows (the first one
                                  // chunk_shift shorter), one CTA each: see the kernel's prologue
     int a_stage_bytes;
@@ -637,7 +639,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                             mbar_expect_tx(bar_full + 8u * stage, a_box_bytes);
                             tma_load_4d(sA + (uint32_t)stage * a_stage_bytes, &tmA, bar_full + 8u * stage,
-                                        kb * a.KB, x0 - a.pad_x + xl, s0, c_ra + ri);
+                                        kb * a.KB, x0 * a.sx - a.pad_x + xl, s0, c_ra + ri);
                             ++t;
                             if (++stage == a.nstage) { stage = 0; phase ^= 1u; }
                         }
@@ -946,7 +948,7 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     if (dtype != 1 && dtype != 2) return false;
     const int esize = dtype == 1 ? 2 : 1;
     const int row_bytes = Cin * esize;
-    if (stride_x != 1) return false;
+    if (stride_x < 1 || stride_x > 8) return false;     // (a tensor map's traversal stride is at most 8)
     if (!(row_bytes == 32 || row_bytes == 64 || (row_bytes >= 128 && row_bytes % 128 == 0))) return false;
     if (Kh * Kw > 32 || Cout % 16 != 0) return false;
     p->swb = row_bytes >= 128 ? 128 : row_bytes;
@@ -967,7 +969,12 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
         if (p->BS > S) p->BS = S;
     }
     p->BXP = p->BX + halo;
-    if (p->BXP > 256) return false;
+    // An x-strided layer needs one box per kx tap (the tap's positions x' * stride + kx - pad are then one strided
+    // walk of the input row, which the tensor map does); the haloed tile of the row-shift mode has no such form.
+    if (stride_x != 1 && (p->shift_mode || Kw == 1)) return false;
+    if (stride_x != 1 && getenv("IDF_UNFOLD_X_STRIDE") != nullptr) return false;    // (switch for comparisons: x-unfold pre-pass instead)
+    p->sx = stride_x;
+    if (p->BXP * stride_x > 256) return false;          // the box is given in input positions
     // A stage holds exactly the TMA box (BS streams x BXP positions).  The MMAs read 128 rows from row kx on,
     // so for the last positions they run past the box into whatever follows in shared memory: those are
     // lanes outside the tile, whose accumulators nobody reads.
@@ -1056,10 +1063,12 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     cuuint64_t dims[4] = {(cuuint64_t)a.Cin, (cuuint64_t)a.Win, (cuuint64_t)a.S, (cuuint64_t)n_in_rows};
     cuuint64_t strides[3] = {(cuuint64_t)a.Cin * esize, (cuuint64_t)a.Win * a.Cin * esize,
                              (cuuint64_t)a.S * a.Win * a.Cin * esize};
-    cuuint32_t box[4] = {(cuuint32_t)p.KB, (cuuint32_t)p.BXP, (cuuint32_t)p.BS, 1};
-    cuuint32_t es[4] = {1, 1, 1, 1};
+    // (with a traversal stride the box is counted in input positions and delivers every sx-th of them)
+    cuuint32_t box[4] = {(cuuint32_t)p.KB, (cuuint32_t)(p.BXP * p.sx), (cuuint32_t)p.BS, 1};
+    cuuint32_t es[4] = {1, 1, 1, 1}, es_in[4] = {1, (cuuint32_t)p.sx, 1, 1};
+    if (a.stride_x != p.sx) return cudaErrorNotSupported;
     CUresult r = enc(&tmA, dtype == 1 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 4,
-                     const_cast<void*>(a.in), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(p.swb),
+                     const_cast<void*>(a.in), dims, strides, box, es_in, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(p.swb),
                      CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorNotSupported;
 
@@ -1107,7 +1116,7 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     t.pad_x = a.pad_x; t.relu = a.relu; t.shift = a.shift; t.ring_rows = a.ring_rows; t.out_elem = a.out_elem;
     t.BX = p.BX; t.BS = p.BS; t.n_xt = p.n_xt; t.Ntile = p.Ntile; t.n_nt = p.n_nt; t.KB = p.KB; t.n_kb = p.n_kb;
     t.swb = p.swb; t.nslot = p.nslot; t.nstage = p.nstage; t.tmem_cols = p.tmem_cols;
-    t.BXP = p.BXP; t.shift_mode = p.shift_mode; t.a_stage_bytes = p.a_stage_bytes;
+    t.BXP = p.BXP; t.shift_mode = p.shift_mode; t.sx = p.sx; t.a_stage_bytes = p.a_stage_bytes;
     t.out_esize = p.out_esize; t.out_pwb = p.out_pwb; t.out_panels = p.out_panels; t.out_stage_bytes = p.out_stage_bytes; t.out_stage_rows = p.out_stage_rows; t.out_groups = p.out_groups;
     t.out_row_dim = row_dim; t.out_row_first = (int)(a.o_begin - a.out_row_base);
     t.pool = a.pool_fused; t.pool_keep = a.pool_keep; t.pool_state = a.pool_state; t.pool_row_base = a.out_row_base;

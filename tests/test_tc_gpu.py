@@ -52,7 +52,14 @@ CASES = [
     ("bf16_stride2_unfold", "bf16", (conv(64, 64, 3, stride=2, pad=1),), 15, 31, 4),
     ("bf16_5ch_k5_unfold", "bf16", (conv(5, 16, 5, stride=2, pad=2),), 17, 29, 3),
     ("i8_16ch_unfold", "i8", (conv(16, 32, 3),), 12, 26, 7),
-    ("i8_stride2_unfold", "i8", (conv(32, 64, 3, stride=2),), 21, 33, 5),
+    # x-strided layers with 32- or 64-byte rows: the tensor map walks the input row in steps of the stride
+    ("i8_stride2_x", "i8", (conv(32, 64, 3, stride=2),), 21, 33, 5),
+    ("i8_stride2_x_pad", "i8", (conv(64, 32, 3, stride=2, pad=1),), 22, 37, 4),
+    ("i8_stride2_x_wide", "i8", (conv(32, 32, 3, stride=2, pad=1),), 9, 300, 2),
+    ("i8_stride3_x_k5", "i8", (conv(32, 16, 5, stride=3, pad=2),), 23, 41, 3),
+    ("bf16_stride2_x_16ch", "bf16", (conv(16, 32, 3, stride=2),), 19, 30, 6),
+    ("bf16_stride2_x_32ch_pad", "bf16", (conv(32, 64, 3, stride=2, pad=1),), 18, 53, 3),
+    ("i8_stride2_x_pool", "i8", (conv(32, 32, 3, stride=2), POOL), 27, 45, 5),
     ("i8_2ch_unfold", "i8", (conv(2, 32, 3, path=1),), 12, 30, 6),     # forced dense: AUTO would scatter events
     ("i8_64", "i8", (conv(64, 64, 3),), 12, 30, 6),
     ("i8_32", "i8", (conv(32, 64, 3),), 12, 30, 6),
