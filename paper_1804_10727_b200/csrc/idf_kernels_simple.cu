@@ -175,9 +175,21 @@ cudaError_t launch_conv_simple(const ConvArgs& a, int dtype, cudaStream_t st)
 // Rows still open at the end of the block go back to the ring in global memory.
 // ------------------------------------------------------------------------------------------------
 constexpr int SPARSE_MAX_THREADS = 512;
-constexpr int SPARSE_MAX_EVENTS = 2048;   // list capacity per pass; longer rows take several passes
+constexpr int SPARSE_MAX_EVENTS = 1024;   // list capacity per pass; longer rows take several passes
 
 template <typename TS> __device__ __forceinline__ void atomic_add(TS* p, TS v) { atomicAdd(p, v); }
+// The same on an address known to lie in shared memory: a reduction in the shared state space (the generic
+// form has to find out at run time which space the pointer belongs to).  No memory clobber: the statements are
+// volatile, so they keep their order, and whoever reads the sums does so behind a __syncthreads().
+__device__ __forceinline__ void atomic_add_shared(int* p, int v)
+{
+    asm volatile("red.shared.add.s32 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(p)), "r"(v));
+}
+__device__ __forceinline__ void atomic_add_shared(float* p, float v)
+{
+    asm volatile("red.shared.add.f32 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(p)), "f"(v));
+}
+constexpr int SPARSE_W_SMEM = 1024;       // weights of a thin layer (Kh*Kw*Cin*Cout values at most this many) are kept in shared memory
 
 template <typename TI, typename TW, typename TS, typename TO, bool RING_IN_SMEM>
 __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArgs a)
@@ -188,6 +200,7 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
     __shared__ TS ev_val[SPARSE_MAX_EVENTS];
     __shared__ int ev_count;
     __shared__ unsigned long long ev_total;
+    __shared__ TS w_s[SPARSE_W_SMEM];
 
     const int s = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31;
@@ -203,6 +216,10 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
     const long long ring_base = RING_IN_SMEM ? 0 : (long long)s * row_elems;
 
     if (tid == 0) ev_total = 0;
+    const int n_w = a.Kh * a.Kw * a.Cin * a.Cout;
+    const bool w_in_smem = n_w <= SPARSE_W_SMEM;
+    if (w_in_smem)
+        for (int i = tid; i < n_w; i += SPARSE_THREADS) w_s[i] = (TS)to_acc(w[i]);
     if (RING_IN_SMEM) {
         for (int i = tid; i < a.ring_rows * row_elems; i += SPARSE_THREADS) {
             const int slot = i / row_elems, e = i - slot * row_elems;
@@ -247,6 +264,32 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
                 // channels; target row, ring slot and target x are worked out once per tap row / tap (no
                 // per-channel index arithmetic, no division when the stride is 1)
                 const int ty0 = (int)(r - a.o_begin * a.stride) + a.pad;          // tap ky reaches relative row (ty0 - ky) / stride
+                if (RING_IN_SMEM && w_in_smem && a.stride == 1 && a.stride_x == 1 && a.Kh == 3 && a.Kw == 3) {
+                    // the common 3x3, stride-1 case with everything in shared memory, unrolled: the three target rows'
+                    // slot offsets are worked out once per input row, a tap costs an address, a weight, a reduction
+                    int soff[3];
+#pragma unroll
+                    for (int ky = 0; ky < 3; ++ky) soff[ky] = ty0 - ky >= 0 ? ((slot0 + ty0 - ky) % a.ring_rows) * row_elems : -1;
+                    const int tap_w = a.Cin * a.Cout;
+                    TS* ring_s = (TS*)smem_raw;
+                    for (int e = tid >> 5; e < n_ev; e += SPARSE_THREADS / 32) {
+                        const int x = ev_x[e] + a.pad_x;
+                        const TS val = ev_val[e];
+                        const TS* wp = w_s + ev_ci[e] * a.Cout;
+                        for (int co = lane; co < a.Cout; co += 32) {
+#pragma unroll
+                            for (int ky = 0; ky < 3; ++ky) {
+                                if (soff[ky] < 0) continue;
+#pragma unroll
+                                for (int kx = 0; kx < 3; ++kx) {
+                                    const int ox = x - kx;
+                                    if (ox < 0 || ox >= a.Wout) continue;
+                                    atomic_add_shared(ring_s + soff[ky] + ox * a.Cout + co, val * wp[(ky * 3 + kx) * tap_w + co]);
+                                }
+                            }
+                        }
+                    }
+                } else
                 for (int e = tid >> 5; e < n_ev; e += SPARSE_THREADS / 32) {
                     const int x = ev_x[e], ci = ev_ci[e];
                     const TS val = ev_val[e];
@@ -257,16 +300,21 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
                         if (a.stride != 1) { orel = ty / a.stride; if (orel * a.stride != ty) continue; }
                         const int slot = (slot0 + orel) % a.ring_rows;
                         TS* drow = &ring[ring_base + slot * slot_stride];
-                        const TW* wrow = w + ((long long)ky * a.Kw * a.Cin + ci) * a.Cout;
+                        const int wrow_i = (ky * a.Kw * a.Cin + ci) * a.Cout;
+                        const TW* wrow = w + wrow_i;
                         for (int kx = 0; kx < a.Kw; ++kx) {
                             const int tx = x + a.pad_x - kx;
                             if (tx < 0) break;
                             int ox = tx;
                             if (a.stride_x != 1) { ox = tx / a.stride_x; if (ox * a.stride_x != tx) continue; }
                             if (ox >= a.Wout) continue;
-                            const TW* wp = wrow + (long long)kx * a.Cin * a.Cout;
+                            const int wofs = kx * a.Cin * a.Cout;
                             TS* dst = drow + ox * a.Cout;
-                            for (int co = lane; co < a.Cout; co += 32) atomic_add(dst + co, val * (TS)to_acc(wp[co]));
+                            for (int co = lane; co < a.Cout; co += 32) {
+                                const TS wv = w_in_smem ? w_s[wrow_i + wofs + co] : (TS)to_acc(wrow[wofs + co]);
+                                if (RING_IN_SMEM) atomic_add_shared(dst + co, val * wv);
+                                else atomic_add(dst + co, val * wv);
+                            }
                         }
                     }
                 }
