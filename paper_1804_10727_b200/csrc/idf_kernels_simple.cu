@@ -198,7 +198,7 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ short ev_x[SPARSE_MAX_EVENTS], ev_ci[SPARSE_MAX_EVENTS];   // position and channel of the event
     __shared__ TS ev_val[SPARSE_MAX_EVENTS];
-    __shared__ int ev_count;
+    __shared__ int ev_count[2];
     __shared__ unsigned long long ev_total;
     __shared__ TS w_s[SPARSE_W_SMEM];
 
@@ -215,7 +215,7 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
     const long long slot_stride = RING_IN_SMEM ? row_elems : (long long)a.S * row_elems;
     const long long ring_base = RING_IN_SMEM ? 0 : (long long)s * row_elems;
 
-    if (tid == 0) ev_total = 0;
+    if (tid == 0) { ev_total = 0; ev_count[0] = 0; ev_count[1] = 0; }
     const int n_w = a.Kh * a.Kw * a.Cin * a.Cout;
     const bool w_in_smem = n_w <= SPARSE_W_SMEM;
     if (w_in_smem)
@@ -232,104 +232,8 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
     const int taps = a.Kh * a.Kw;
     const int slot0 = (int)(a.o_begin % a.ring_rows);     // ring slot of the first visited row
     long long done = a.o_begin;                      // rows below `done` have been emitted
-    for (long long r = a.r0; r <= a.r1; ++r) {
-        // r == r1 is the flush pass: no input, only rows up to done_end are finalised
-        if (r < a.r1) {
-            const TI* row = in + ((r - a.r0) * a.S + s) * (long long)n_comp;
-            for (int base = 0; base < n_comp; base += SPARSE_MAX_EVENTS) {
-                if (tid == 0) ev_count = 0;
-                __syncthreads();
-                const int lim = min(n_comp, base + SPARSE_MAX_EVENTS);
-                for (int i0 = base + (tid - lane); i0 < lim; i0 += SPARSE_THREADS) {
-                    const int i = i0 + lane;
-                    const TS v = (i < lim) ? (TS)to_acc(row[i]) : (TS)0;
-                    const unsigned m = __ballot_sync(0xffffffffu, v != (TS)0);
-                    if (m) {
-                        int off = 0;
-                        if (lane == 0) off = atomicAdd(&ev_count, __popc(m));
-                        off = __shfl_sync(0xffffffffu, off, 0);
-                        if (v != (TS)0) {
-                            const int k = off + __popc(m & ((1u << lane) - 1u));
-                            const int x = i / a.Cin;
-                            ev_x[k] = (short)x;
-                            ev_ci[k] = (short)(i - x * a.Cin);
-                            ev_val[k] = v;
-                        }
-                    }
-                }
-                __syncthreads();
-                const int n_ev = ev_count;
-                if (tid == 0) ev_total += (unsigned long long)n_ev;
-                // scatter: a warp takes one event at a time and walks its kernel taps, the lanes take the output
-                // channels; target row, ring slot and target x are worked out once per tap row / tap (no
-                // per-channel index arithmetic, no division when the stride is 1)
-                const int ty0 = (int)(r - a.o_begin * a.stride) + a.pad;          // tap ky reaches relative row (ty0 - ky) / stride
-                if (RING_IN_SMEM && w_in_smem && a.stride == 1 && a.stride_x == 1 && a.Kh == 3 && a.Kw == 3) {
-                    // the common 3x3, stride-1 case with everything in shared memory, unrolled: the three target rows'
-                    // slot offsets are worked out once per input row, a tap costs an address, a weight, a reduction
-                    int soff[3];
-#pragma unroll
-                    for (int ky = 0; ky < 3; ++ky) soff[ky] = ty0 - ky >= 0 ? ((slot0 + ty0 - ky) % a.ring_rows) * row_elems : -1;
-                    const int tap_w = a.Cin * a.Cout;
-                    TS* ring_s = (TS*)smem_raw;
-                    for (int e = tid >> 5; e < n_ev; e += SPARSE_THREADS / 32) {
-                        const int x = ev_x[e] + a.pad_x;
-                        const TS val = ev_val[e];
-                        const TS* wp = w_s + ev_ci[e] * a.Cout;
-                        for (int co = lane; co < a.Cout; co += 32) {
-#pragma unroll
-                            for (int ky = 0; ky < 3; ++ky) {
-                                if (soff[ky] < 0) continue;
-#pragma unroll
-                                for (int kx = 0; kx < 3; ++kx) {
-                                    const int ox = x - kx;
-                                    if (ox < 0 || ox >= a.Wout) continue;
-                                    atomic_add_shared(ring_s + soff[ky] + ox * a.Cout + co, val * wp[(ky * 3 + kx) * tap_w + co]);
-                                }
-                            }
-                        }
-                    }
-                } else
-                for (int e = tid >> 5; e < n_ev; e += SPARSE_THREADS / 32) {
-                    const int x = ev_x[e], ci = ev_ci[e];
-                    const TS val = ev_val[e];
-                    for (int ky = 0; ky < a.Kh; ++ky) {
-                        const int ty = ty0 - ky;
-                        if (ty < 0) break;
-                        int orel = ty;
-                        if (a.stride != 1) { orel = ty / a.stride; if (orel * a.stride != ty) continue; }
-                        const int slot = (slot0 + orel) % a.ring_rows;
-                        TS* drow = &ring[ring_base + slot * slot_stride];
-                        const int wrow_i = (ky * a.Kw * a.Cin + ci) * a.Cout;
-                        const TW* wrow = w + wrow_i;
-                        for (int kx = 0; kx < a.Kw; ++kx) {
-                            const int tx = x + a.pad_x - kx;
-                            if (tx < 0) break;
-                            int ox = tx;
-                            if (a.stride_x != 1) { ox = tx / a.stride_x; if (ox * a.stride_x != tx) continue; }
-                            if (ox >= a.Wout) continue;
-                            const int wofs = kx * a.Cin * a.Cout;
-                            TS* dst = drow + ox * a.Cout;
-                            for (int co = lane; co < a.Cout; co += 32) {
-                                const TS wv = w_in_smem ? w_s[wrow_i + wofs + co] : (TS)to_acc(wrow[wofs + co]);
-                                if (RING_IN_SMEM) atomic_add_shared(dst + co, val * wv);
-                                else atomic_add(dst + co, val * wv);
-                            }
-                        }
-                    }
-                }
-                __syncthreads();
-            }
-        }
-        // rows completed by input row r (or, in the flush pass, everything below done_end)
-        long long upto;
-        if (r < a.r1) {
-            const long long q = r + a.pad - a.Kh + 1;    // row o completes at r = o*stride - pad + Kh - 1
-            upto = q < 0 ? 0 : q / a.stride + 1;
-            if (upto > a.done_end) upto = a.done_end;
-        } else {
-            upto = a.done_end;
-        }
+    // finalisation of the ring rows below `upto`: emit f(c + b), zero the slot
+    auto finalise_upto = [&](long long upto) {
         for (; done < upto; ++done) {
             const long long slot = done % a.ring_rows;
             TO* orow = out + (done - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride;
@@ -361,7 +265,114 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
                 }
             }
         }
-        __syncthreads();
+    };
+    // Per input row two block-wide phases: (A) the row's non-zero components are compacted into the event list
+    // while the rows that the PREVIOUS input row completed are finalised (independent work: the loads of one
+    // hide behind the arithmetic of the other); (B) the events are scattered into the ring.  The event
+    // counter is double-buffered so that it can be cleared for the next pass while this one's is still read.
+    int cb = 0;
+    for (long long r = a.r0; r <= a.r1; ++r) {
+        // r == r1 is the closing pass: no input, everything below done_end is finalised
+        const bool have = r < a.r1;
+        long long upto = a.done_end;
+        if (have) {
+            const long long q = r + a.pad - a.Kh;        // row o completes at input row o*stride - pad + Kh - 1, here: <= r - 1
+            upto = q < 0 ? 0 : q / a.stride + 1;
+            if (upto > a.done_end) upto = a.done_end;
+        }
+        const TI* row = in + ((r - a.r0) * a.S + s) * (long long)n_comp;
+        const int n_pass = have ? (n_comp + SPARSE_MAX_EVENTS - 1) / SPARSE_MAX_EVENTS : 1;
+        for (int pass = 0; pass < n_pass; ++pass) {
+            const int base = pass * SPARSE_MAX_EVENTS;
+            const int lim = min(n_comp, base + SPARSE_MAX_EVENTS);
+            TS v_first = (TS)0;
+            if (have && base + tid < lim) v_first = (TS)to_acc(row[base + tid]);      // in flight during the finalisation
+            if (pass == 0) finalise_upto(upto);
+            if (have) {
+                for (int i0 = base + (tid - lane); i0 < lim; i0 += SPARSE_THREADS) {
+                    const int i = i0 + lane;
+                    const TS v = (i0 == base + (tid - lane)) ? v_first : ((i < lim) ? (TS)to_acc(row[i]) : (TS)0);
+                    const unsigned m = __ballot_sync(0xffffffffu, v != (TS)0);
+                    if (m) {
+                        int off = 0;
+                        if (lane == 0) off = atomicAdd(&ev_count[cb], __popc(m));
+                        off = __shfl_sync(0xffffffffu, off, 0);
+                        if (v != (TS)0) {
+                            const int k = off + __popc(m & ((1u << lane) - 1u));
+                            const int x = i / a.Cin;
+                            ev_x[k] = (short)x;
+                            ev_ci[k] = (short)(i - x * a.Cin);
+                            ev_val[k] = v;
+                        }
+                    }
+                }
+            }
+            __syncthreads();
+            if (have) {
+                const int n_ev = ev_count[cb];
+                if (tid == 0) { ev_total += (unsigned long long)n_ev; ev_count[cb ^ 1] = 0; }
+            // scatter: a warp takes one event at a time and walks its kernel taps, the lanes take the output
+            // channels; target row, ring slot and target x are worked out once per tap row / tap (no
+            // per-channel index arithmetic, no division when the stride is 1)
+            const int ty0 = (int)(r - a.o_begin * a.stride) + a.pad;          // tap ky reaches relative row (ty0 - ky) / stride
+            if (RING_IN_SMEM && w_in_smem && a.stride == 1 && a.stride_x == 1 && a.Kh == 3 && a.Kw == 3) {
+                // the common 3x3, stride-1 case with everything in shared memory, unrolled: the three target rows'
+                // slot offsets are worked out once per input row, a tap costs an address, a weight, a reduction
+                int soff[3];
+#pragma unroll
+                for (int ky = 0; ky < 3; ++ky) soff[ky] = ty0 - ky >= 0 ? ((slot0 + ty0 - ky) % a.ring_rows) * row_elems : -1;
+                const int tap_w = a.Cin * a.Cout;
+                TS* ring_s = (TS*)smem_raw;
+                for (int e = tid >> 5; e < n_ev; e += SPARSE_THREADS / 32) {
+                    const int x = ev_x[e] + a.pad_x;
+                    const TS val = ev_val[e];
+                    const TS* wp = w_s + ev_ci[e] * a.Cout;
+                    for (int co = lane; co < a.Cout; co += 32) {
+#pragma unroll
+                        for (int ky = 0; ky < 3; ++ky) {
+                            if (soff[ky] < 0) continue;
+#pragma unroll
+                            for (int kx = 0; kx < 3; ++kx) {
+                                const int ox = x - kx;
+                                if (ox < 0 || ox >= a.Wout) continue;
+                                atomic_add_shared(ring_s + soff[ky] + ox * a.Cout + co, val * wp[(ky * 3 + kx) * tap_w + co]);
+                            }
+                        }
+                    }
+                }
+            } else
+            for (int e = tid >> 5; e < n_ev; e += SPARSE_THREADS / 32) {
+                const int x = ev_x[e], ci = ev_ci[e];
+                const TS val = ev_val[e];
+                for (int ky = 0; ky < a.Kh; ++ky) {
+                    const int ty = ty0 - ky;
+                    if (ty < 0) break;
+                    int orel = ty;
+                    if (a.stride != 1) { orel = ty / a.stride; if (orel * a.stride != ty) continue; }
+                    const int slot = (slot0 + orel) % a.ring_rows;
+                    TS* drow = &ring[ring_base + slot * slot_stride];
+                    const int wrow_i = (ky * a.Kw * a.Cin + ci) * a.Cout;
+                    const TW* wrow = w + wrow_i;
+                    for (int kx = 0; kx < a.Kw; ++kx) {
+                        const int tx = x + a.pad_x - kx;
+                        if (tx < 0) break;
+                        int ox = tx;
+                        if (a.stride_x != 1) { ox = tx / a.stride_x; if (ox * a.stride_x != tx) continue; }
+                        if (ox >= a.Wout) continue;
+                        const int wofs = kx * a.Cin * a.Cout;
+                        TS* dst = drow + ox * a.Cout;
+                        for (int co = lane; co < a.Cout; co += 32) {
+                            const TS wv = w_in_smem ? w_s[wrow_i + wofs + co] : (TS)to_acc(wrow[wofs + co]);
+                            if (RING_IN_SMEM) atomic_add_shared(dst + co, val * wv);
+                            else atomic_add(dst + co, val * wv);
+                        }
+                    }
+                }
+            }
+                __syncthreads();
+                cb ^= 1;
+            }
+        }
     }
     if (RING_IN_SMEM) {
         for (int i = tid; i < a.ring_rows * row_elems; i += SPARSE_THREADS) {
