@@ -240,6 +240,19 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
             if (sizeof(TO) == 1 && (a.Cout & 3) == 0 && (((uintptr_t)orow) & 3) == 0) {
                 // int8 rows: four channels per thread, one 4-byte store
                 const bool pow2 = (a.Cout & (a.Cout - 1)) == 0;
+                if (RING_IN_SMEM && !bias && a.relu) {
+                    // the usual case (ReLU, no bias): max, rounding shift, min on four words, three byte permutes to pack
+                    const int rnd = a.shift > 0 ? 1 << (a.shift - 1) : 0;
+                    const int4* src = (const int4*)(smem_raw) + (int)slot * (row_elems >> 2);
+                    uint32_t* dst = (uint32_t*)orow;
+                    for (int i = tid; i < (row_elems >> 2); i += SPARSE_THREADS) {
+                        const int4 c = src[i];
+                        ((int4*)src)[i] = make_int4(0, 0, 0, 0);
+                        const int v0 = min((max(c.x, 0) + rnd) >> a.shift, 127), v1 = min((max(c.y, 0) + rnd) >> a.shift, 127);
+                        const int v2 = min((max(c.z, 0) + rnd) >> a.shift, 127), v3 = min((max(c.w, 0) + rnd) >> a.shift, 127);
+                        dst[i] = __byte_perm(__byte_perm(v0, v1, 0x4040), __byte_perm(v2, v3, 0x4040), 0x5410);
+                    }
+                } else
                 for (int i = tid * 4; i < row_elems; i += SPARSE_THREADS * 4) {
                     TS* p = &ring[ring_base + slot * slot_stride + i];
                     const int co = pow2 ? (i & (a.Cout - 1)) : i % a.Cout;
