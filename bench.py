@@ -283,10 +283,10 @@ def run_ours(args, w):
         ratio = {"bf16": 1.0, "i8": 2.0, "f32": 0.5}[w.dtype]      # nominal ratio to the bf16 dense peak
         # DRAM bytes of the conv launches of one step, from the ncu capture summarised in
         # profiles/conv_tc_kernel_vgg2d_rows64.md (dram__bytes_read.sum + dram__bytes_write.sum of the seven launches
-        # of a 64-row case = 408.3 MB; the traffic is rows in + rows out, so it grows with the number of rows)
+        # of a 64-row case = 408.9 MB; the traffic is rows in + rows out, so it grows with the number of rows)
         traffic, traffic_note = None, "no ncu capture for this workload"
         if w.name == "vgg2d" and w.n_streams == 64:
-            traffic = 408.3e6 * w.H / 64.0
+            traffic = 408.9e6 * w.H / 64.0
             traffic_note = "bytes per step over all conv launches, scaled by rows from a 64-row ncu capture (cold caches)"
         peak = peaks["bf16_tflops"] * ratio
         line = {
