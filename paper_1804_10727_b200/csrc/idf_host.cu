@@ -186,7 +186,7 @@ int launch_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, boo
         a.w = net->ws + P.w_off;
         a.bias = P.b_packed.empty() ? nullptr : net->ws + P.b_off;
         a.ring = net->ws + P.state_off;
-    a.ring_scratch = net->ring_scratch_off ? net->ws + net->ring_scratch_off : nullptr;
+        a.ring_scratch = net->ring_scratch_off ? net->ws + net->ring_scratch_off : nullptr;
         a.out = out_ptr;
         a.out_row_stride = row_stride; a.out_stream_stride = stream_stride; a.out_row_base = row_base;
         a.out_rows_extent = last ? out_cap : P.out_cap_rows;
@@ -273,7 +273,7 @@ int launch_conv_pool(idf_net* net, size_t i, const void* in_ptr, long long n_in,
     a.w = net->ws + P.w_off;
     a.bias = P.b_packed.empty() ? nullptr : net->ws + P.b_off;
     a.ring = net->ws + P.state_off;
-    a.ring_scratch = net->ring_scratch_off ? net->ws + net->ring_scratch_off : nullptr;
+        a.ring_scratch = net->ring_scratch_off ? net->ws + net->ring_scratch_off : nullptr;
     if (last) {
         a.out = final_out;
         a.out_row_stride = (long long)Q.out_w * Q.out_c;
