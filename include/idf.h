@@ -149,6 +149,15 @@ int idf_stream_reset(idf_net* net);
 int idf_stream_push(idf_net* net, const void* d_segments, int n_seg,
                     void* d_out, long long out_capacity_rows, int* rows_emitted);
 
+/* Output window for streams of unbounded length (the paper's 1D case: state constant in the input length, so the
+ * output buffer should be too).  By default output row o of a stream is written at row index o of d_out.  After
+ * this call rows are written at index o - first_row instead: the caller has consumed the rows below first_row and
+ * reuses the buffer from its start.  first_row must not exceed the number of rows emitted so far (IDF_ERR_ARG), so
+ * that no row still to come would land below index 0; IDF_ERR_STATE unless streams are open.  The capacity check of
+ * the push calls counts from first_row.  idf_stream_open, idf_stream_reset and idf_state_restore set it back to 0.
+ * A global-average sink always writes its single row at index 0. */
+int idf_stream_set_out_base(idf_net* net, long long first_row);
+
 /* End of input: complete the rows that wait only for bottom zero padding, in depth order, and
  * drop rows that can never complete.  total_rows (host, may be NULL) receives the number of output
  * rows per stream since open.  After this call only idf_stream_open or idf_net_destroy are valid. */

@@ -78,6 +78,7 @@ struct idf_net {
     int phase = CREATED;
     long long launches = 0;
     long long out_rows_total = 0;
+    long long out_base = 0;                // output row written at index 0 of the caller's buffer (idf_stream_set_out_base)
     // optional per-launch timing (CUDA events on the handle's stream)
     bool timing = false;
     struct Timed { int layer; cudaEvent_t a, b; };
@@ -148,7 +149,7 @@ int launch_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, boo
     if (done_end < o_begin) done_end = o_begin;
     const long long n_out = done_end - o_begin;
     *n_out_p = n_out;
-    if (last && done_end > out_cap)
+    if (last && done_end - net->out_base > out_cap)
         return fail(IDF_ERR_CAPACITY, "output row %lld does not fit out_capacity_rows=%lld", done_end - 1, out_cap);
     if (!last && n_out + out_slot > P.out_cap_rows)
         return fail(IDF_ERR_CAPACITY, "internal: layer %zu emits %lld rows at slot %lld of a %d-row buffer", i, n_out,
@@ -164,7 +165,7 @@ int launch_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, boo
         out_ptr = final_out;
         row_stride = (long long)P.out_w * P.out_c;
         stream_stride = out_cap * row_stride;
-        row_base = 0;
+        row_base = net->out_base;
     } else {
         out_ptr = net->ws + P.out_off;
         stream_stride = (long long)P.out_w * P.out_c;
@@ -262,7 +263,7 @@ int launch_conv_pool(idf_net* net, size_t i, const void* in_ptr, long long n_in,
     const long long o_end = std::max(started, done_end);
     const long long q_begin = Q.rows_done, q_done = done_end / 2;
     const long long n_out = q_done - q_begin;
-    if (last && q_done > out_cap)
+    if (last && q_done - net->out_base > out_cap)
         return fail(IDF_ERR_CAPACITY, "output row %lld does not fit out_capacity_rows=%lld", q_done - 1, out_cap);
     if (!last && n_out + out_slot > Q.out_cap_rows)
         return fail(IDF_ERR_CAPACITY, "internal: layer %zu emits %lld rows at slot %lld of a %d-row buffer", i + 1, n_out,
@@ -278,7 +279,7 @@ int launch_conv_pool(idf_net* net, size_t i, const void* in_ptr, long long n_in,
         a.out = final_out;
         a.out_row_stride = (long long)Q.out_w * Q.out_c;
         a.out_stream_stride = out_cap * a.out_row_stride;
-        a.out_row_base = 0;
+        a.out_row_base = net->out_base;
         a.out_rows_extent = out_cap;
     } else {
         a.out = net->ws + Q.out_off;
@@ -400,7 +401,7 @@ int run_segments(idf_net* net, const void* d_segments, long long n_seg, bool flu
     {
         long long r = net->L[0].rows_in + n_seg;
         for (size_t i = 0; i < nl; ++i) r = flush ? layer_rows_at_flush(net->L[i], r) : layer_done_after(net->L[i], r);
-        if (r > out_cap)
+        if (r - net->out_base > out_cap)
             return fail(IDF_ERR_CAPACITY, "output row %lld does not fit out_capacity_rows=%lld", r - 1, out_cap);
     }
     const size_t seg_bytes = (size_t)net->n_streams * net->in_w * net->in_c * elem_size(net->L[0].in_elem);
@@ -700,6 +701,7 @@ int idf_stream_reset(idf_net* net)
     net->phase = OPEN;
     net->launches = 0;
     net->out_rows_total = 0;
+    net->out_base = 0;
     return IDF_OK;
 }
 
@@ -717,6 +719,16 @@ int idf_stream_push(idf_net* net, const void* d_segments, int n_seg, void* d_out
     if (rc != IDF_OK) return rc;
     net->out_rows_total += em;
     if (rows_emitted) *rows_emitted = (int)em;
+    return IDF_OK;
+}
+
+int idf_stream_set_out_base(idf_net* net, long long first_row)
+{
+    if (!net) return fail(IDF_ERR_ARG, "net must not be NULL");
+    if (net->phase != OPEN) return fail(IDF_ERR_STATE, "set_out_base needs open streams");
+    if (first_row < 0 || first_row > net->out_rows_total)
+        return fail(IDF_ERR_ARG, "first_row=%lld: only rows emitted so far (%lld) can be left behind", first_row, net->out_rows_total);
+    net->out_base = first_row;
     return IDF_OK;
 }
 
@@ -948,6 +960,7 @@ int idf_state_restore(idf_net* net, const void* h_snapshot, size_t bytes)
         P.rows_in = prog[3 * i]; P.rows_done = prog[3 * i + 1]; P.pending = 0;
     }
     net->out_rows_total = h.out_rows_total;
+    net->out_base = 0;
     net->phase = OPEN;
     return IDF_OK;
 }

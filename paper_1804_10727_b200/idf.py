@@ -28,7 +28,7 @@ EXPORTS = (
     "idf_net_create", "idf_net_destroy", "idf_net_state_bytes", "idf_net_workspace_bytes", "idf_out_shape",
     "idf_stream_open", "idf_stream_reset", "idf_stream_push", "idf_stream_push_last", "idf_stream_finish", "idf_run_host", "idf_event_counts",
     "idf_launch_count", "idf_stream_status", "idf_set_timing", "idf_layer_times", "idf_conv_rows_noalloc", "idf_last_error",
-    "idf_state_snapshot_bytes", "idf_state_save", "idf_state_restore",
+    "idf_state_snapshot_bytes", "idf_state_save", "idf_state_restore", "idf_stream_set_out_base",
 )
 
 
@@ -77,6 +77,7 @@ def lib():
         L.idf_conv_rows_noalloc.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp,
                                             ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                             ctypes.c_int, vp, ll, ctypes.POINTER(ll), vp]
+        L.idf_stream_set_out_base.argtypes = [vp, ll]
         L.idf_state_snapshot_bytes.argtypes = [vp]; L.idf_state_snapshot_bytes.restype = sz
         L.idf_state_save.argtypes = [vp, vp, sz]
         L.idf_state_restore.argtypes = [vp, vp, sz]
@@ -226,6 +227,10 @@ class Net:
         _check(lib().idf_stream_push_last(self._h, segments.data_ptr(), segments.shape[0], out.data_ptr(), out.shape[1],
                                           ctypes.byref(tot)))
         return int(tot.value)
+
+    def set_out_base(self, first_row: int):
+        """Later output rows are written at index (row - first_row) of the output buffer; see idf_stream_set_out_base."""
+        _check(lib().idf_stream_set_out_base(self._h, int(first_row)))
 
     def finish(self, out: torch.Tensor) -> int:
         tot = ctypes.c_longlong()

@@ -126,6 +126,7 @@ def test_bad_arguments_and_call_order():
     assert L.idf_stream_push_last(net._h, 256, 1, 256, 4, None) == idf.ERR_STATE
     assert L.idf_stream_reset(net._h) == idf.ERR_STATE
     assert b"before stream_open" in L.idf_last_error()
+    assert L.idf_stream_set_out_base(net._h, 0) == idf.ERR_STATE and L.idf_stream_set_out_base(None, 0) == idf.ERR_ARG
     assert L.idf_stream_open(net._h, None, 0, None) == idf.ERR_ARG
     assert L.idf_stream_open(net._h, 256, 16, None) == idf.ERR_CAPACITY
     assert L.idf_stream_open(net._h, 257, 1 << 30, None) == idf.ERR_ARG    # misaligned workspace

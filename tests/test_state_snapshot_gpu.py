@@ -140,3 +140,50 @@ def test_snapshot_of_another_net_is_refused():
     a.finish(out)
     for n in (a, b, c):
         n.close()
+
+
+@pytest.mark.parametrize("name,mode", [("oned_k9", "f32"), ("oned_pad", "i8"), ("same_pool", "i8"), ("stride2", "f32")])
+def test_bounded_output_window_on_long_streams(orc, name, mode):
+    """A small output buffer reused from its start (idf_stream_set_out_base) collects the same rows as a full one."""
+    layers = SMALL_NETS[name]
+    if mode == "i8":
+        layers = with_shifts(layers, 8)
+    H, W = small_dims(name)
+    H *= 3
+    C0 = next(l.cin for l in layers if l.kind == "conv")
+    x, ws, bs = rand_net(mode, layers, H, W, C0, S=3, seed=31)
+    want = orc.forward(mode, layers, x, ws, bs)
+    net = idf.Net(mode, layers, W, C0, 3, ws, bs, row_block=4)
+    seg = _segments(net, x)
+    cap = 9                                                  # rows of output buffer; a push of 7 segments never emits more
+    out = torch.zeros((3, cap) + tuple(want.shape[2:]), dtype=net.out_torch_dtype, device="cuda")
+    net.open()
+    got, total, r, k = [], 0, 0, 0
+    while r < H:
+        m = min((7, 1, 5, 2)[k % 4], H - r)
+        k += 1
+        net.set_out_base(total)
+        if r + m == H:
+            new_total = net.push_last(seg[r:r + m].contiguous(), out)
+            em = new_total - total
+        else:
+            em = net.push(seg[r:r + m].contiguous(), out)
+        got.append(out[:, :em].cpu().numpy().copy())
+        total += em
+        r += m
+    net.status()
+    merged = np.concatenate(got, axis=1)
+    assert merged.shape == want.shape
+    if mode == "i8":
+        assert_equal(merged, want, name)
+    else:
+        assert_close(merged, want, name)
+    # rows still to come must not land below index 0, and a full window refuses further rows
+    net.reset()
+    with pytest.raises(idf.IdfError) as e:
+        net.set_out_base(1)
+    assert e.value.code == idf.ERR_ARG
+    with pytest.raises(idf.IdfError) as e:
+        net.push(seg[:H].contiguous(), out)
+    assert e.value.code == idf.ERR_CAPACITY
+    net.close()
