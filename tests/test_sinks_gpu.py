@@ -121,3 +121,23 @@ def test_sink_state_survives_a_snapshot(orc):
     assert b.push_last(seg[9:].contiguous(), out_b) == 1
     assert np.array_equal(out_b.cpu().numpy(), want.astype(np.float32))
     a.close(); b.close()
+
+
+def test_mnist_shaped_classifier_many_streams(orc):
+    """The paper's experiment in shape: 28x28 images fed row by row through the mnist2d conv stack and ten fully
+    connected output units (random weights: accuracy is not the point), 512 streams, int8, bit-exact."""
+    from paper_1804_10727_b200 import workloads
+    w = workloads.get("mnist2d", n_streams=512)
+    x = workloads.make_input(w)
+    ws, bs = workloads.make_params(w)
+    layers = tuple(w.layers) + (_fc(32, 10, 10, 10, shift=11),)
+    r = np.random.default_rng(12)
+    ws = list(ws) + [r.integers(-127, 128, size=(10, 10, 10, 32)).astype(np.int8)]
+    bs = list(bs) + [r.integers(-2000, 2000, size=(10,)).astype(np.int32)]
+    want = orc.forward("i8", layers, x, ws, bs)
+    assert want.shape == (512, 1, 1, 10) and len(np.unique(want)) > 20          # the logits are not saturated
+    net = idf.Net("i8", layers, w.W, w.C, 512, ws, bs)
+    got = idf.infer(net, x, chunks=[1] * w.H, last=True)                        # one image row per push
+    assert_equal(got, want, "classifier")
+    assert net.state_bytes == 18432 + 10 * 4
+    net.close()
