@@ -204,7 +204,7 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
 
     const int s = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31;
-    const int SPARSE_THREADS = blockDim.x;      // 256, or 512 for wide rows (more warps to hide the finalisation's latency)
+    const int SPARSE_THREADS = blockDim.x;      // 64 to 512 by row length: wide rows want many warps for the finalisation, short rows many small CTAs per SM
     const TI* __restrict__ in = (const TI*)a.in;
     const TW* __restrict__ w = (const TW*)a.w;
     const TS* __restrict__ bias = (const TS*)a.bias;
@@ -403,7 +403,8 @@ static cudaError_t launch_sparse_t(const ConvArgs& a, cudaStream_t st)
 {
     if (a.S == 0) return cudaSuccess;
     const size_t ring_bytes = (size_t)a.ring_rows * a.Wout * a.Cout * sizeof(TS);
-    const int nthr = (long long)a.Wout * a.Cout >= 4096 ? SPARSE_MAX_THREADS : 256;
+    const long long row_words = (long long)a.Wout * a.Cout;
+    const int nthr = row_words >= 4096 ? SPARSE_MAX_THREADS : (row_words >= 1024 ? 256 : (row_words >= 512 ? 128 : 64));     // short rows: more, smaller CTAs per SM
     if (ring_bytes <= conv_sparse_max_smem()) {
         auto k = conv_sparse_kernel<TI, TW, TS, TO, true>;
         cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring_bytes);
