@@ -43,12 +43,16 @@ struct Emit<int8_t, int> {
 };
 
 // ------------------------------------------------------------------------------------------------
-// Dense update + finalisation.  One thread owns one element (slot, stream, x, co) of the ring and
-// walks, in order, every output row of this block that lives in that slot, so a slot is never read
-// and written by different threads.  Weights: [Kh][Kw][Cin][Cout] (threads of a warp differ in co).
+// Dense update + finalisation.  The first `edge_blocks` CTAs: one thread owns one element (slot, stream,
+// x, co) of the ring and walks, in order, every output row of this block that lives in that slot and
+// exchanges state with the ring (begun by an earlier block, or left open by this one), so a slot is
+// never read and written by different threads.  The other CTAs take the interior rows [int_begin, int_end):
+// rows begun AND completed by this block's input never touch the ring (Eq. 1 restricted to the block), so
+// each (row, stream, x, co) has a thread of its own - with few streams and narrow rows that is where the
+// parallelism is.  Weights: [Kh][Kw][Cin][Cout] (threads of a warp differ in co).
 // ------------------------------------------------------------------------------------------------
 template <typename TI, typename TW, typename TS, typename TO>
-__global__ void __launch_bounds__(256) conv_rows_kernel(ConvArgs a)
+__global__ void __launch_bounds__(256) conv_rows_kernel(ConvArgs a, long long int_begin, long long int_end, unsigned edge_blocks)
 {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const TI* __restrict__ in = (const TI*)a.in;
@@ -57,9 +61,37 @@ __global__ void __launch_bounds__(256) conv_rows_kernel(ConvArgs a)
     TS* ring = (TS*)a.ring;
     TO* out = (TO*)a.out;
     const long long row_elems = (long long)a.Wout * a.Cout;
+    if (blockIdx.x >= edge_blocks) {
+        const long long n_int = (int_end - int_begin) * a.S * row_elems;
+        for (long long idx = (long long)(blockIdx.x - edge_blocks) * blockDim.x + threadIdx.x; idx < n_int;
+             idx += (long long)(gridDim.x - edge_blocks) * blockDim.x) {
+            const int co = (int)(idx % a.Cout);
+            long long t = idx / a.Cout;
+            const int x = (int)(t % a.Wout);
+            t /= a.Wout;
+            const int s = (int)(t % a.S);
+            const long long o = int_begin + t / a.S;
+            TS acc = 0;
+            for (int ky = 0; ky < a.Kh; ++ky) {
+                const long long r = o * a.stride - a.pad + ky;
+                if (r < a.r0 || r >= a.r1) continue;             // zero padding above the first or below the last row
+                const TI* row = in + ((r - a.r0) * a.S + s) * (long long)a.Win * a.Cin;
+                for (int kx = 0; kx < a.Kw; ++kx) {
+                    const int ix = x * a.stride_x - a.pad_x + kx;
+                    if (ix < 0 || ix >= a.Win) continue;
+                    const TI* ap = row + (long long)ix * a.Cin;
+                    const TW* wp = w + ((long long)(ky * a.Kw + kx) * a.Cin) * a.Cout + co;
+                    for (int ci = 0; ci < a.Cin; ++ci) acc += to_acc(ap[ci]) * to_acc(wp[(long long)ci * a.Cout]);
+                }
+            }
+            out[(o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride + (long long)x * a.Cout + co] =
+                Emit<TO, TS>::run(acc, bias ? bias[co] : (TS)0, a.relu, a.shift);
+        }
+        return;
+    }
     const long long total = (long long)a.ring_rows * a.S * row_elems;
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-         idx += (long long)gridDim.x * blockDim.x) {
+         idx += (long long)edge_blocks * blockDim.x) {
         const int co = (int)(idx % a.Cout);
         long long t = idx / a.Cout;
         const int x = (int)(t % a.Wout);
@@ -73,6 +105,7 @@ __global__ void __launch_bounds__(256) conv_rows_kernel(ConvArgs a)
         TS leave = 0;
         TS* rp = ring + ((long long)slot * a.S + s) * row_elems + (long long)x * a.Cout + co;
         for (; o < a.o_end; o += a.ring_rows) {
+            if (o >= int_begin && o < int_end) continue;         // an interior row: another CTA's
             TS acc = 0;
             for (int ky = 0; ky < a.Kh; ++ky) {
                 const long long r = o * a.stride - a.pad + ky;
@@ -148,7 +181,19 @@ static cudaError_t launch_rows(const ConvArgs& a, cudaStream_t st)
     if (total == 0 || a.o_end <= a.o_begin) return cudaSuccess;
     long long blocks = (total + 255) / 256;
     if (blocks > 148LL * 64) blocks = 148LL * 64;
-    conv_rows_kernel<TI, TW, TS, TO><<<(unsigned)blocks, 256, 0, st>>>(a);
+    // interior rows: not begun by an earlier block (first tap row o*stride - pad >= r0) and completed by this one
+    long long int_begin = a.r0 > 0 ? (a.r0 + a.pad + a.stride - 1) / a.stride : a.o_begin;
+    if (int_begin < a.o_begin) int_begin = a.o_begin;
+    long long int_end = a.done_end;
+    long long int_blocks = 0;
+    if (int_end - int_begin >= 2LL * a.ring_rows) {
+        const long long n_int = (int_end - int_begin) * a.S * a.Wout * a.Cout;
+        int_blocks = (n_int + 255) / 256;
+        if (int_blocks > 148LL * 64) int_blocks = 148LL * 64;
+    } else {
+        int_begin = int_end = 0;
+    }
+    conv_rows_kernel<TI, TW, TS, TO><<<(unsigned)(blocks + int_blocks), 256, 0, st>>>(a, int_begin, int_end, (unsigned)blocks);
     return cudaGetLastError();
 }
 
