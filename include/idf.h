@@ -117,16 +117,27 @@ int idf_net_destroy(idf_net* net);
  * 2D: proportional to the row width), as the paper's abstract claims.  0 if net is NULL. */
 size_t idf_net_state_bytes(const idf_net* net);
 
-/* Device bytes the caller must provide to idf_stream_open: all streams' rolling state, the packed
- * parameters, and the transient row_block-sized buffers between layers. */
+/* Device bytes the caller must provide to idf_stream_open: all streams' rolling state (the "activation
+ * subset buffers" of the paper's Discussion, idf_net_state_bytes per stream), the packed parameters, and
+ * the transient buffers of at most 2 * row_block + 8 rows between layers that carry the events of Eq. 3
+ * from one layer to the next (sentence after Eq. 5).  Independent of the number of segments.  0 if net
+ * is NULL. */
 size_t idf_net_workspace_bytes(const idf_net* net);
 
-/* Shape of the output map after in_rows segments (out_rows may be 0). Any out pointer may be NULL. */
+/* Shape of the output map once in_rows segments and the end of input have been seen: the extent of the
+ * conventional layer-by-layer result (Eq. 1 with the conv connectivity of Section "Asynchronous
+ * incremental updates"), which the incremental result equals ("identical to the original output",
+ * Introduction).  out_rows may be 0.  Any out pointer may be NULL.  IDF_ERR_ARG for a NULL net or
+ * negative in_rows. */
 int idf_out_shape(const idf_net* net, long long in_rows, long long* out_rows, int* out_w, int* out_c);
 
-/* Bind a workspace (device, 256-byte aligned, >= idf_net_workspace_bytes) and a CUDA stream
- * (a cudaStream_t passed as void*, NULL = default stream); upload the parameters, zero all state,
- * reset the segment counters.  May be called again after idf_stream_finish to start new streams. */
+/* Start streams: every unit's state variable c and activation begin at zero (the paper's convention
+ * in the paragraph after Eq. 3: all units start at 0, so the first events are the inputs themselves).
+ * Binds a workspace (device, 256-byte aligned, >= idf_net_workspace_bytes; owned by the caller, who must
+ * keep it alive and unmodified until the streams are finished) and a CUDA stream (a cudaStream_t passed as
+ * void*, NULL = default stream); uploads the parameters, zeroes all state, resets the segment counters.
+ * May be called again after idf_stream_finish to start new streams.  Errors: IDF_ERR_ARG (NULL or
+ * misaligned workspace), IDF_ERR_CAPACITY (workspace too small), IDF_ERR_CUDA. */
 int idf_stream_open(idf_net* net, void* d_workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Start new streams on the workspace and CUDA stream bound by the last idf_stream_open: zero all
@@ -136,7 +147,12 @@ int idf_stream_open(idf_net* net, void* d_workspace, size_t workspace_bytes, voi
  * (also in the middle of streams, which are then abandoned); IDF_ERR_STATE before it. */
 int idf_stream_reset(idf_net* net);
 
-/* Push n_seg consecutive segments of every stream through all layers, depth first.
+/* Push n_seg consecutive segments of every stream through all layers, depth first: the paper's
+ * streaming core "can process small segments of the input as they arrive" (Introduction, last
+ * paragraph); a segment is a sample or an image row (Fig. 2 and its caption), its non-zero components
+ * are the events of Eq. 3, each layer adds them into its state (Eq. 4), and rows of units that no present
+ * or future segment can reach any more are finalised and passed up at once (sentence after Eq. 5; Fig. 2
+ * caption: such units are fully processed and can be forgotten).
  *   d_segments: device, [n_seg][n_streams][in_w][in_c] in the activation type
  *   d_out     : device, [n_streams][out_capacity_rows][out_w][out_c], fp32 (float nets) or int8;
  *               output rows that become complete are written at their absolute row index
@@ -158,8 +174,10 @@ int idf_stream_push(idf_net* net, const void* d_segments, int n_seg,
  * A global-average sink always writes its single row at index 0. */
 int idf_stream_set_out_base(idf_net* net, long long first_row);
 
-/* End of input: complete the rows that wait only for bottom zero padding, in depth order, and
- * drop rows that can never complete.  total_rows (host, may be NULL) receives the number of output
+/* End of input.  The length of a stream is not known while it runs (segments are taken as they
+ * arrive, Introduction and Discussion), yet the result must equal the conventional output (Introduction:
+ * "identical"; Eq. 1), whose last rows see zero padding below the input.  So this call completes the rows
+ * that wait only for bottom zero padding, in depth order, and drops rows that can never complete.  total_rows (host, may be NULL) receives the number of output
  * rows per stream since open.  After this call only idf_stream_open or idf_net_destroy are valid. */
 int idf_stream_finish(idf_net* net, void* d_out, long long out_capacity_rows, long long* total_rows);
 
@@ -263,6 +281,20 @@ int idf_conv_rows_noalloc(const float* d_in, int n_rows, int n_streams, int in_w
                           const float* d_weights, const float* d_bias, int cout, int kh, int kw,
                           int stride, int pad, int relu, float* d_out, long long out_capacity_rows,
                           long long* out_rows, void* cuda_stream);
+
+/* Debug only.  Process-wide switches that route work away from the default kernels so that tests can compare
+ * the paths with one another; results are the same with any combination (bit-exact for int nets), only the
+ * kernels and launch counts differ.  Not for production use; the paper has no counterpart.  flags is a
+ * combination of the bits below (0 = defaults); IDF_DEBUG_NO_TENSOR_CORES and IDF_DEBUG_NO_POOL_FUSION are
+ * read by idf_net_create (they affect nets created afterwards), the other two at every launch.
+ * IDF_ERR_ARG for an unknown bit (nothing changes). */
+typedef enum {
+    IDF_DEBUG_NO_TENSOR_CORES = 1,  /* dense layers stay on the CUDA-core kernel                              */
+    IDF_DEBUG_NO_POOL_FUSION = 2,   /* max-pool layers run as launches of their own                           */
+    IDF_DEBUG_NO_ROW_CHUNKS = 4,    /* a block's rows stay in one CTA per tile                                */
+    IDF_DEBUG_NO_PDL = 8            /* no programmatic dependent launch                                       */
+} idf_debug_flag;
+int idf_set_debug_flags(unsigned int flags);
 
 /* Message for the most recent failure on the calling thread ("" if none). */
 const char* idf_last_error(void);

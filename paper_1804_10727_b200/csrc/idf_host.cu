@@ -4,6 +4,7 @@
 #include "idf_internal.h"
 
 #include <algorithm>
+#include <atomic>
 #include <cstdarg>
 #include <cstdio>
 #include <cstdlib>
@@ -316,8 +317,14 @@ int launch_conv_pool(idf_net* net, size_t i, const void* in_ptr, long long n_in,
     }
     ce = launch_conv_tc(t, P.tc_pool, net->dtype, P.w_map_pool, (int)n_in, (unsigned int*)(net->ws + net->status_off), net->stream);
     if (net->timing) {
-        cudaEventRecord(ev_b, net->stream);
-        net->timed.push_back({(int)i, ev_a, ev_b});
+        if (ce == cudaSuccess) {
+            cudaEventRecord(ev_b, net->stream);
+            net->timed.push_back({(int)i, ev_a, ev_b});
+        } else {
+            // a declined launch is no layer time: the layer runs again through launch_layer, which records its own pair
+            net->event_pool.push_back(ev_a);
+            net->event_pool.push_back(ev_b);
+        }
     }
     if (ce == cudaErrorNotSupported) return 1;
     if (ce != cudaSuccess) return fail(IDF_ERR_CUDA, "kernel launch failed at layer %zu: %s", i, cudaGetErrorString(ce));
@@ -426,13 +433,25 @@ int run_segments(idf_net* net, const void* d_segments, long long n_seg, bool flu
 
 }  // namespace
 
+namespace {
+std::atomic<unsigned> g_debug_flags{0};
+}
 namespace idf {
 int set_last_error(int code, const char* msg) { return fail(code, "%s", msg); }
+unsigned debug_flags() { return g_debug_flags.load(std::memory_order_relaxed); }
 }  // namespace idf
 
 extern "C" {
 
 const char* idf_last_error(void) { return g_err.c_str(); }
+
+int idf_set_debug_flags(unsigned int flags)
+{
+    if (flags & ~(unsigned)(IDF_DEBUG_NO_TENSOR_CORES | IDF_DEBUG_NO_POOL_FUSION | IDF_DEBUG_NO_ROW_CHUNKS | IDF_DEBUG_NO_PDL))
+        return fail(IDF_ERR_ARG, "unknown debug flag in 0x%x", flags);
+    g_debug_flags.store(flags, std::memory_order_relaxed);
+    return IDF_OK;
+}
 
 int idf_net_create(const idf_spec* spec, const void* const* weights, const void* const* biases, idf_net** out)
 {
@@ -513,9 +532,8 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
                         }
             }
             // tensor-core layout [tap][Cout][Cin], activation type, when the layer qualifies
-            const char* no_tc = getenv("IDF_DISABLE_TC");
             const int in_cap = i == 0 ? net->row_block : net->L[i - 1].out_cap_rows;
-            const bool tc_allowed = !P.use_sparse && !(no_tc && no_tc[0] == '1') && spec->dtype != IDF_F32;
+            const bool tc_allowed = !P.use_sparse && !(debug_flags() & IDF_DEBUG_NO_TENSOR_CORES) && spec->dtype != IDF_F32;
             const size_t es = spec->dtype == IDF_I8_I32 ? 1 : 2;
             const int taps = l.kh * l.kw;
             const bool pool_next = i + 1 < spec->n_layers && spec->layers[i + 1].kind == IDF_MAXPOOL2;
@@ -589,11 +607,11 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
     }
     // a dense tensor-core conv layer directly followed by a 2x2 max-pool emits the pooled rows itself
     {
-        const char* no_fuse = getenv("IDF_NO_POOL_FUSION");
+        const bool no_fuse = (debug_flags() & IDF_DEBUG_NO_POOL_FUSION) != 0;
         for (size_t i = 0; i + 1 < net->L.size(); ++i) {
             LayerPlan& P = net->L[i];
             P.fuse_pool = P.l.kind == IDF_CONV && net->L[i + 1].l.kind == IDF_MAXPOOL2 && P.tc.ok && P.tc_pool.ok && !P.use_sparse &&
-                          P.out_w >= 2 && (P.tc_pool.BX % 2) == 0 && !(no_fuse && no_fuse[0] == '1');
+                          P.out_w >= 2 && (P.tc_pool.BX % 2) == 0 && !no_fuse;
         }
     }
     // workspace: [parameters][state of all streams][rows travelling between layers][counters]

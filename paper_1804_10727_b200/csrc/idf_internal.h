@@ -10,6 +10,9 @@ namespace idf {
 // element types of activation rows travelling between layers
 enum Elem : int { E_F32 = 0, E_BF16 = 1, E_I8 = 2, E_I32 = 3 };
 
+// process-wide debug switches (bits of idf_debug_flag), set through idf_set_debug_flags
+unsigned debug_flags();
+
 inline size_t elem_size(int e) { return e == E_F32 || e == E_I32 ? 4 : (e == E_BF16 ? 2 : 1); }
 
 // How one conv layer advances by a block of input rows.  All row indices are absolute

@@ -587,7 +587,11 @@ __global__ void __launch_bounds__(256) pool_rows_kernel(PoolArgs a)
 }
 
 // 16 bytes of channels per thread (the layout is channels-innermost, so a position's channels are
-// contiguous): the same fold, vectorised.  Used when C * sizeof(T) is a multiple of 16.
+// contiguous): the same fold, vectorised, with a thread per output row.  Used when C * sizeof(T) is a
+// multiple of 16.  The one state row can be read (the first visited row, when its first half came with an
+// earlier launch) and written (the last visited row, when its second half is still to come) in the same
+// launch; when both happen the reading thread also handles the writing row, after its own, so the two
+// accesses to a state element are ordered inside one thread whatever the CTAs' order.
 template <typename T>
 __global__ void __launch_bounds__(256) pool_rows_vec_kernel(PoolArgs a)
 {
@@ -598,7 +602,11 @@ __global__ void __launch_bounds__(256) pool_rows_vec_kernel(PoolArgs a)
     T* out = (T*)a.out;
     const int px = (a.Win == 1) ? 1 : 2;
     const int cv = a.C / V;
-    const long long n_o = a.o_end - a.o_begin;
+    long long n_o = a.o_end - a.o_begin;
+    const bool carried_in = 2 * a.o_begin < a.r0;
+    const bool carried_out = a.o_end - 1 >= a.done_end;
+    const bool chained = carried_in && carried_out && n_o >= 2;     // the first row's thread takes the last row too
+    if (chained) n_o -= 1;
     const long long total = n_o * a.S * a.Wout * cv;
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (long long)gridDim.x * blockDim.x) {
@@ -607,28 +615,32 @@ __global__ void __launch_bounds__(256) pool_rows_vec_kernel(PoolArgs a)
         const int ox = (int)(t % a.Wout);
         t /= a.Wout;
         const int s = (int)(t % a.S);
-        const long long o = a.o_begin + t / a.S;
+        long long o = a.o_begin + t / a.S;
         const long long sidx = ((long long)s * a.Wout + ox) * a.C + c;
-        __align__(16) T m[V];
-        bool have = false;
-        if (2 * o < a.r0) { *(int4*)m = *(const int4*)(state + sidx); have = true; }
-        for (int dy = 0; dy < 2; ++dy) {
-            const long long r = 2 * o + dy;
-            if (r < a.r0 || r >= a.r1) continue;
-            const T* row = in + ((r - a.r0) * a.S + s) * (long long)a.Win * a.C;
-            for (int dx = 0; dx < px; ++dx) {
-                __align__(16) T v[V];
-                *(int4*)v = *(const int4*)(row + (long long)(px * ox + dx) * a.C + c);
+        for (int turn = 0; turn < 2; ++turn) {
+            __align__(16) T m[V];
+            bool have = false;
+            if (2 * o < a.r0) { *(int4*)m = *(const int4*)(state + sidx); have = true; }
+            for (int dy = 0; dy < 2; ++dy) {
+                const long long r = 2 * o + dy;
+                if (r < a.r0 || r >= a.r1) continue;
+                const T* row = in + ((r - a.r0) * a.S + s) * (long long)a.Win * a.C;
+                for (int dx = 0; dx < px; ++dx) {
+                    __align__(16) T v[V];
+                    *(int4*)v = *(const int4*)(row + (long long)(px * ox + dx) * a.C + c);
 #pragma unroll
-                for (int j = 0; j < V; ++j) m[j] = have ? max_of(m[j], v[j]) : v[j];
-                have = true;
+                    for (int j = 0; j < V; ++j) m[j] = have ? max_of(m[j], v[j]) : v[j];
+                    have = true;
+                }
             }
+            if (o < a.done_end)
+                *(int4*)(out + (o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride +
+                         (long long)ox * a.C + c) = *(const int4*)m;
+            else
+                *(int4*)(state + sidx) = *(const int4*)m;
+            if (!(chained && o == a.o_begin)) break;
+            o = a.o_end - 1;
         }
-        if (o < a.done_end)
-            *(int4*)(out + (o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride +
-                     (long long)ox * a.C + c) = *(const int4*)m;
-        else
-            *(int4*)(state + sidx) = *(const int4*)m;
     }
 }
 
@@ -640,8 +652,8 @@ static cudaError_t launch_pool_t(const PoolArgs& a, cudaStream_t st)
     constexpr int V = 16 / (int)sizeof(T);
     const bool aligned = (a.C % V == 0) && (((uintptr_t)a.in | (uintptr_t)a.out | (uintptr_t)a.state) & 15) == 0 &&
                          ((a.out_row_stride | a.out_stream_stride) % V == 0);
-    // each output row has its own thread in the vector kernel, so it needs every row pair to be
-    // independent: true as long as at most one visited row is carried in or out (always the case)
+    // (the vector kernel gives each output row a thread; it orders the one read and the one write of the state
+    // row itself, see there)
     if (aligned) {
         const long long tv = (a.o_end - a.o_begin) * a.S * a.Wout * (a.C / V);
         long long blocks = (tv + 255) / 256;

@@ -18,6 +18,7 @@
 // Warp roles: warp 0 = TMA producer and row scheduler, warp 1 = TMEM owner and MMA issuer,
 // warps 2.. = epilogue groups of four warps (one warp per TMEM lane quarter) that take output rows in turn.
 // Every wait is bounded; on expiry the kernel records IDF_ERR_TIMEOUT in the status word and leaves.
+#include "../../include/idf.h"
 #include "idf_internal.h"
 
 #include <cuda.h>
@@ -802,9 +803,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (!a.pool) {
                 owner = (orel < n_cin || orel >= c_done_rel) ? 0 : orel % a.out_groups;
             } else {
-                // both rows of a pooling pair go to one group; pairs touching the global ring go to group 0
+                // both rows of a pooling pair go to one group; pairs touching the global ring or the pool layer's state
+                // (first < 0: the pair's first row came with an earlier launch) go to group 0
                 const int first = orel - (int)((c_o_begin + orel) & 1);
-                owner = (first < n_cin || first + 1 >= c_done_rel) ? 0 : (int)(((c_o_begin + orel) >> 1) % a.out_groups);
+                owner = (first < 0 || first < n_cin || first + 1 >= c_done_rel) ? 0 : (int)(((c_o_begin + orel) >> 1) % a.out_groups);
             }
             if (owner != grp) continue;
             const int slot = orel % a.nslot;
@@ -972,7 +974,6 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     // An x-strided layer needs one box per kx tap (the tap's positions x' * stride + kx - pad are then one strided
     // walk of the input row, which the tensor map does); the haloed tile of the row-shift mode has no such form.
     if (stride_x != 1 && (p->shift_mode || Kw == 1)) return false;
-    if (stride_x != 1 && getenv("IDF_UNFOLD_X_STRIDE") != nullptr) return false;    // (switch for comparisons: x-unfold pre-pass instead)
     p->sx = stride_x;
     if (p->BXP * stride_x > 256) return false;          // the box is given in input positions
     // A stage holds exactly the TMA box (BS streams x BXP positions).  The MMAs read 128 rows from row kx on,
@@ -1126,9 +1127,12 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
         const int units = p.n_mt * p.n_nt;
         int min_rows = 2 * a.ring_rows + 2;
         if (min_rows < 16) min_rows = 16;
-        const bool no_chunks = getenv("IDF_NO_ROW_CHUNKS") != nullptr;     // (read per launch: tests switch it)
+        const bool no_chunks = (debug_flags() & IDF_DEBUG_NO_ROW_CHUNKS) != 0;
         // (a block that continues rows of an earlier one needs room for the copy of the ring, see ring_in)
-        if (!no_chunks && units < 120 && t.n_orows >= 2 * min_rows && (a.r0 == 0 || a.ring_scratch)) {
+        // a launch that takes a first row out of the pool layer's state (its first row is the second of a pair) and
+        // also parks one there (its last emitted row is the first of a pair) keeps both in one CTA: read before write
+        const bool pool_state_rw = a.pool_fused && a.pool_keep && (a.o_begin & 1) && (a.done_end & 1);
+        if (!no_chunks && !pool_state_rw && units < 120 && t.n_orows >= 2 * min_rows && (a.r0 == 0 || a.ring_scratch)) {
             int want = 296 / units;                                 // at most two full waves of CTAs on the 148 SMs
             if (want > t.n_orows / min_rows) want = t.n_orows / min_rows;
             if (want > 1) {
@@ -1169,8 +1173,8 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    // (IDF_NO_PDL=1 turns it off; the griddepcontrol instructions in the kernels are then no-ops)
-    static const bool use_pdl = getenv("IDF_NO_PDL") == nullptr;
+    // (without the attribute the griddepcontrol instructions in the kernels are no-ops)
+    const bool use_pdl = (debug_flags() & IDF_DEBUG_NO_PDL) == 0;
     cfg.attrs = attr; cfg.numAttrs = use_pdl ? 1 : 0;
     cudaError_t le = cudaLaunchKernelEx(&cfg, fn, tmA, *(const CUtensorMap*)w_map, tmO, t);
     if (le != cudaSuccess) return le;

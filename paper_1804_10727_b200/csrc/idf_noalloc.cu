@@ -92,7 +92,8 @@ extern "C" int idf_conv_rows_noalloc(const float* d_in, int n_rows, int n_stream
     if (cudaGetLastError() != cudaSuccess) return set_last_error(IDF_ERR_CUDA, "noalloc: repack launch failed");
 
     // the same row-block walk as idf_stream_push + idf_stream_finish for a single layer
-    const int row_block = 8;
+    // (blocks as long as the regular entry points' default: neither the ring nor the scratch depends on the length)
+    const int row_block = 25088 / in_w < 32 ? 32 : (25088 / in_w > 1024 ? 1024 : 25088 / in_w);
     long long rows_done = 0;
     for (long long r0 = 0; r0 < n_rows; r0 += row_block) {
         const long long r1 = r0 + row_block < n_rows ? r0 + row_block : n_rows;

@@ -28,8 +28,9 @@ EXPORTS = (
     "idf_net_create", "idf_net_destroy", "idf_net_state_bytes", "idf_net_workspace_bytes", "idf_out_shape",
     "idf_stream_open", "idf_stream_reset", "idf_stream_push", "idf_stream_push_last", "idf_stream_finish", "idf_run_host", "idf_event_counts",
     "idf_launch_count", "idf_stream_status", "idf_set_timing", "idf_layer_times", "idf_conv_rows_noalloc", "idf_last_error",
-    "idf_state_snapshot_bytes", "idf_state_save", "idf_state_restore", "idf_stream_set_out_base",
+    "idf_state_snapshot_bytes", "idf_state_save", "idf_state_restore", "idf_stream_set_out_base", "idf_set_debug_flags",
 )
+DEBUG_NO_TENSOR_CORES, DEBUG_NO_POOL_FUSION, DEBUG_NO_ROW_CHUNKS, DEBUG_NO_PDL = 1, 2, 4, 8
 
 
 class IdfLayer(ctypes.Structure):
@@ -81,6 +82,7 @@ def lib():
         L.idf_state_snapshot_bytes.argtypes = [vp]; L.idf_state_snapshot_bytes.restype = sz
         L.idf_state_save.argtypes = [vp, vp, sz]
         L.idf_state_restore.argtypes = [vp, vp, sz]
+        L.idf_set_debug_flags.argtypes = [ctypes.c_uint]
         L.idf_last_error.restype = ctypes.c_char_p
         _lib = L
     return _lib
@@ -89,6 +91,11 @@ def lib():
 def _check(rc: int):
     if rc != 0:
         raise IdfError(rc, lib().idf_last_error().decode())
+
+
+def set_debug_flags(flags: int):
+    """Debug only: route work away from the default kernels (see idf_set_debug_flags); 0 restores the defaults."""
+    _check(lib().idf_set_debug_flags(int(flags)))
 
 
 def _layer_struct(l) -> IdfLayer:
@@ -332,7 +339,12 @@ def conv_rows_noalloc(segments: torch.Tensor, weights: torch.Tensor, bias: Optio
     assert segments.is_contiguous() and weights.is_contiguous() and out.is_contiguous()
     n_rows, S, in_w, cin = segments.shape
     cout, kh, kw, cin2 = weights.shape
-    assert cin == cin2 and out.shape[0] == S and out.shape[3] == cout
+    assert cin == cin2 and out.dim() == 4 and out.shape[0] == S and out.shape[3] == cout
+    # the C call cannot see the width of `out`: a buffer narrower than the layer's rows would be overrun
+    out_w = 1 if in_w == 1 else (in_w + 2 * pad - kw) // stride + 1
+    assert out.shape[2] == out_w, f"out has width {out.shape[2]}, the layer emits rows of width {out_w}"
+    if bias is not None:
+        assert bias.is_cuda and bias.dtype == torch.float32 and bias.is_contiguous() and tuple(bias.shape) == (cout,)
     rows = ctypes.c_longlong()
     st = torch.cuda.current_stream(segments.device).cuda_stream
     _check(lib().idf_conv_rows_noalloc(segments.data_ptr(), n_rows, S, in_w, cin, weights.data_ptr(),

@@ -17,3 +17,11 @@ def orc():
     from oracle import oracle
     oracle.build()
     return oracle
+
+
+@pytest.fixture
+def debug_flags():
+    """Set the library's debug switches for one test; the defaults come back afterwards."""
+    from paper_1804_10727_b200 import idf
+    yield idf.set_debug_flags
+    idf.set_debug_flags(0)

@@ -186,6 +186,31 @@ def test_bf16_rounding_matches_torch_and_ties(orc):
     assert orc.round_bf16(np.array([0.0]))[0] == 0.0
 
 
+def test_bf16_rounding_of_subnormals_matches_torch_and_closed_forms(orc):
+    """The subnormal range of bfloat16 (below 2^-126, spacing 2^-133): fewer significant bits are kept there.
+    torch's fp32 -> bf16 conversion rounds these to nearest even too, so it pins the branch; the hand-made
+    values pin the ties and the underflow to zero."""
+    r = np.random.default_rng(3)
+    # fp32 bit patterns with biased exponents 0..12: fp32 subnormals and the smallest normals, both signs
+    bits = (r.integers(0, 13, size=40000).astype(np.uint32) << 23) | r.integers(0, 1 << 23, size=40000).astype(np.uint32)
+    bits |= (r.integers(0, 2, size=40000).astype(np.uint32) << 31)
+    v = torch.from_numpy(bits.view(np.float32).copy())
+    want = v.bfloat16().double().numpy()
+    got = orc.round_bf16(v.double().numpy())
+    assert np.array_equal(got, want) and np.array_equal(np.signbit(got), np.signbit(want))
+    assert (want != 0).any() and (want == 0).any() and (np.abs(want[want != 0]) < 2.0 ** -126).any()
+    tiny = 2.0 ** -133                                       # the smallest positive bfloat16
+    one = lambda x: orc.round_bf16(np.array([x], dtype=np.float64))[0]
+    assert one(tiny) == tiny and one(-tiny) == -tiny
+    assert one(tiny / 2) == 0.0                              # tie between 0 and tiny: to even (zero)
+    assert one(tiny / 2 * (1 + 2.0 ** -30)) == tiny          # just above the tie
+    assert one(tiny / 4) == 0.0
+    assert one(1.5 * tiny) == 2 * tiny                       # tie between tiny and 2 tiny: to even
+    assert one(2.5 * tiny) == 2 * tiny                       # tie between 2 tiny and 3 tiny: to even
+    assert one(2.0 ** -126 - tiny / 4) == 2.0 ** -126        # rounds up into the normal range
+    assert one(-(2.0 ** -126 - 0.75 * tiny)) == -(2.0 ** -126 - tiny)
+
+
 def test_requant_matches_exact_rationals(orc):
     r = np.random.default_rng(2)
     c = r.integers(-200000, 200000, size=4000).astype(np.int32)

@@ -91,12 +91,12 @@ def test_tensor_core_layers_match_oracle(orc, name, mode, layers, H, W, S):
             assert ok.mean() > 0.97 and err.max() < 0.05, (what, ok.mean(), err.max())
 
 
-def test_tensor_core_and_cuda_core_paths_agree_bitwise_on_int8(orc, monkeypatch):
+def test_tensor_core_and_cuda_core_paths_agree_bitwise_on_int8(orc, debug_flags):
     layers = with_shifts((conv(64, 64, 3, pad=1), conv(64, 32, 3, stride=1)), 9)
     x, ws, bs = rand_net("i8", layers, 18, 37, 64, S=5, seed=77)
     got_tc, tc = _run("i8", layers, x, ws, bs)
     assert all(t > 0 for t in tc)
-    monkeypatch.setenv("IDF_DISABLE_TC", "1")
+    debug_flags(idf.DEBUG_NO_TENSOR_CORES)
     got_cc, tc2 = _run("i8", layers, x, ws, bs)
     assert not any(tc2)
     assert np.array_equal(got_tc, got_cc)
@@ -117,7 +117,7 @@ POOL_CASES = [
 
 
 @pytest.mark.parametrize("name,mode,layers,H,W,S", POOL_CASES, ids=[c[0] for c in POOL_CASES])
-def test_pool_folded_into_the_conv_launch_matches_oracle(orc, monkeypatch, name, mode, layers, H, W, S):
+def test_pool_folded_into_the_conv_launch_matches_oracle(orc, debug_flags, name, mode, layers, H, W, S):
     if mode == "i8":
         layers = with_shifts(layers, 9)
     x, ws, bs = rand_net(mode, layers, H, W, layers[0].cin, S=S, seed=3 + len(name))
@@ -148,7 +148,7 @@ def test_pool_folded_into_the_conv_launch_matches_oracle(orc, monkeypatch, name,
         if chunks is None and rb == 0 and last:
             fused_launches = n
     # the same net with the folding switched off runs the pool layers as launches of their own
-    monkeypatch.setenv("IDF_NO_POOL_FUSION", "1")
+    debug_flags(idf.DEBUG_NO_POOL_FUSION)
     got, n = run(None, 0, True)
     check(got, f"{name}/unfused")
     if name == "i8_pool_odd_width":          # an odd tile width cannot pair lanes: this net never folds
@@ -168,7 +168,7 @@ CHUNK_CASES = [
 
 
 @pytest.mark.parametrize("name,mode,layers,H,W,S", CHUNK_CASES, ids=[c[0] for c in CHUNK_CASES])
-def test_row_chunks_match_oracle(orc, monkeypatch, name, mode, layers, H, W, S):
+def test_row_chunks_match_oracle(orc, debug_flags, name, mode, layers, H, W, S):
     if mode == "i8":
         layers = with_shifts(layers, 9)
     x, ws, bs = rand_net(mode, layers, H, W, layers[0].cin, S=S, seed=11 + len(name))
@@ -185,6 +185,6 @@ def test_row_chunks_match_oracle(orc, monkeypatch, name, mode, layers, H, W, S):
             assert_close(got, want, what)
     if mode == "i8":
         # the same with the rows of a block kept in one CTA per tile: bit-identical
-        monkeypatch.setenv("IDF_NO_ROW_CHUNKS", "1")
+        debug_flags(idf.DEBUG_NO_ROW_CHUNKS)
         net = idf.Net(mode, layers, W, layers[0].cin, S, ws, bs)
         assert_equal(idf.infer(net, x, last=True), want, name + "/unchunked")

@@ -38,7 +38,7 @@ def _noalloc(layer, x, w, b):
     return out.cpu().numpy()
 
 
-def test_two_calls_in_a_row_match_the_regular_entry_point():
+def test_two_calls_in_a_row_match_the_regular_entry_point(orc):
     # first call: 3x3, stride 1, same padding; it leaves partial rows and its weights in the scratch
     l1 = conv(3, 8, 3, pad=1)
     x1, w1, b1 = rand_net("f32", (l1,), 21, 17, 3, S=4, seed=31)
@@ -50,6 +50,8 @@ def test_two_calls_in_a_row_match_the_regular_entry_point():
         want = _regular(layer, x, w, b)
         assert not np.isnan(got).any()
         assert_close(got, want, "noalloc vs regular entry point")
+        # ... and both equal the CPU oracle's conventional result
+        assert_close(got, orc.forward("f32", (layer,), x, [w], [b]), "noalloc vs oracle")
 
 
 def test_sizes_beyond_the_built_in_scratch_are_refused():
@@ -60,3 +62,14 @@ def test_sizes_beyond_the_built_in_scratch_are_refused():
     with pytest.raises(idf.IdfError) as e:
         idf.conv_rows_noalloc(seg, w, None, 1, 0, True, out)
     assert e.value.code == idf.ERR_CAPACITY and "scratch" in str(e.value)
+
+
+def test_an_output_buffer_narrower_than_the_rows_is_refused_before_any_launch():
+    # the C call sees only a pointer: the binding must not let a too-narrow buffer through (it would be overrun)
+    seg = torch.zeros((6, 2, 20, 3), device="cuda")
+    w = torch.zeros((4, 3, 3, 3), device="cuda")
+    narrow = torch.zeros((2, 4, 17, 4), device="cuda")       # the layer emits rows of width 18
+    with pytest.raises(AssertionError):
+        idf.conv_rows_noalloc(seg, w, None, 1, 0, True, narrow)
+    with pytest.raises(AssertionError):
+        idf.conv_rows_noalloc(seg, w, torch.zeros(3, device="cuda"), 1, 0, True, torch.zeros((2, 4, 18, 4), device="cuda"))
