@@ -33,11 +33,52 @@ UNIT = "pixels/s"
 
 
 def measured_peaks():
+    """Roofline denominators: the machine's measured copy bandwidth and cuBLAS bf16 rate, as a burst (a kernel timed
+    alone or in a short region) and sustained (seconds under the power cap); an earlier measurement if the file is absent."""
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         d = json.load(open(p))
-        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops_sustained"], "source": "measured"}
-    return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback"}
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_burst": d["bf16_tflops"], "bf16_sustained": d["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+def kernel_source_hash() -> str:
+    """Fingerprint of the CUDA sources: a counter record only speaks for the kernels it was taken from."""
+    import hashlib
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_1804_10727_b200", "csrc")
+    for n in sorted(os.listdir(d)):
+        if n.endswith((".cu", ".h")):
+            h.update(open(os.path.join(d, n), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(w):
+    """DRAM bytes per step of the conv launches from the last ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
+    kept beside the kernels in dram_traffic.json together with the fingerprint of the sources it was taken from.
+    None once the kernels have changed since, or when the capture was of another workload."""
+    p = os.path.join(ROOT, "paper_1804_10727_b200", "dram_traffic.json")
+    if not os.path.exists(p):
+        return None, "no ncu capture recorded"
+    rec = json.load(open(p)).get(w.name)
+    if not rec:
+        return None, "no ncu capture recorded for this workload"
+    if rec.get("kernel_source_hash") != kernel_source_hash():
+        return None, "the kernels have changed since the ncu capture was taken"
+    if rec.get("n_streams") != w.n_streams:
+        return None, "the ncu capture was taken at another stream count"
+    # (rows in + rows out: proportional to the number of rows when the capture was of fewer rows)
+    return rec["bytes_per_row"] * w.H, rec.get("note", "")
+
+
+def algorithmic_bytes(w, net) -> int:
+    """Bytes the method must move per step: the input segments in, the output map out, the parameters once."""
+    act = {"f32": 4, "bf16": 2, "i8": 1}[w.dtype]
+    r, ow, oc = net.out_shape(w.H)
+    out_b = w.n_streams * r * ow * oc * (1 if w.dtype == "i8" else 4)
+    par = sum(l.cout * l.cin * l.kh * l.kw * act for l in w.layers if l.kind == "conv")
+    return w.n_streams * w.H * w.W * w.C * act + out_b + par
 
 
 def conv_macs(w: workloads.Workload):
@@ -176,6 +217,60 @@ def whole_job_value(w, world: int, steps: int, ms: float) -> float:
     return world * w.n_streams * w.H * w.W * steps / (ms * 1e-3)
 
 
+def time_steps(net, d_seg, d_out, steps, warmup, flush_buf, stream, barrier):
+    """Device time of `steps` steps (reset + push_last of the whole batch), L2 flushed before each; returns (ms, launches)."""
+    def step():
+        net.reset()
+        net.push_last(d_seg, d_out)
+    for _ in range(max(warmup, 3)):
+        step()
+    barrier()
+    evs, n_launch = [], 0
+    for _ in range(steps):
+        flush_buf.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        step()
+        b.record(stream)
+        evs.append((a, b))
+        n_launch += net.launches
+    barrier()
+    return sum(a.elapsed_time(b) for a, b in evs), n_launch
+
+
+def extra_workloads(args, main_name, dev, flush_buf, stream, barrier, peaks):
+    """The other workloads, device-timed the same way (fewer steps), as context beside the headline line."""
+    from paper_1804_10727_b200 import idf
+    out = {}
+    for name in workloads.NAMES:
+        if name == main_name:
+            continue
+        w = workloads.get(name)
+        ws, bs = workloads.make_params(w)
+        net = idf.net_from_workload(w, ws, bs)
+        d_seg = idf.segments_from_maps(workloads.make_input(w), w.dtype).to(dev)
+        d_out = net.alloc_out(w.H, dev)
+        net.open(dev)
+        sampler = ClockSampler(int(dev.split(":")[1]))
+        sampler.start()
+        time.sleep(0.05)
+        steps = 10
+        ms, n_launch = time_steps(net, d_seg, d_out, steps, 3, flush_buf, stream, barrier)
+        clocks = sampler.stop()
+        macs = conv_macs(w)
+        flops = 2.0 * sum(macs) * w.n_streams
+        ratio = {"bf16": 1.0, "i8": 2.0, "f32": 0.5}[w.dtype]
+        tf = flops / (ms / steps * 1e-3) / 1e12
+        out[name] = {"value": w.n_streams * w.H * w.W * steps / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / steps, "steps": steps,
+                     "n_streams": w.n_streams, "dtype": w.dtype, "gpu_launches_per_step": n_launch // steps,
+                     "dense_equiv_tflops": tf, "frac_of_burst_peak_whole_step": tf / (peaks["bf16_burst"] * ratio),
+                     "state_bytes_per_stream": net.state_bytes, "clocks": clocks}
+        net.close()
+        del d_seg, d_out
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args, w):
     import torch.distributed as dist
     from paper_1804_10727_b200 import idf
@@ -281,14 +376,12 @@ def run_ours(args, w):
         flops = 2.0 * sum(macs[i] for i in dense) * w.n_streams
         achieved = flops / (dom_ms * 1e-3) / 1e12 if dom_ms > 0 else 0.0
         ratio = {"bf16": 1.0, "i8": 2.0, "f32": 0.5}[w.dtype]      # nominal ratio to the bf16 dense peak
-        # DRAM bytes of the conv launches of one step, from the ncu capture summarised in
-        # profiles/conv_tc_kernel_vgg2d_rows64.md (dram__bytes_read.sum + dram__bytes_write.sum of the seven launches
-        # of a 64-row case = 408.9 MB; the traffic is rows in + rows out, so it grows with the number of rows)
-        traffic, traffic_note = None, "no ncu capture for this workload"
-        if w.name == "vgg2d" and w.n_streams == 64:
-            traffic = 408.9e6 * w.H / 64.0
-            traffic_note = "bytes per step over all conv launches, scaled by rows from a 64-row ncu capture (cold caches)"
-        peak = peaks["bf16_tflops"] * ratio
+        traffic, traffic_note = recorded_traffic(w)
+        # which peak applies: a timed region of seconds runs under the power cap (sustained), a short one does not (burst)
+        timed_s = ms * 1e-3
+        kind = "sustained" if timed_s >= 2.0 else "burst"
+        peak = peaks["bf16_" + kind] * ratio
+        mhz = clocks.get("sm_mhz") if clocks else None
         line = {
             "metric": METRIC, "value": whole_job_value(w, world, args.steps, ms), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
@@ -298,6 +391,7 @@ def run_ours(args, w):
                        "row_block": args.row_block or "default", "l2": "flushed between iterations (256 MiB write)",
                        "state_bytes_per_stream": net.state_bytes},
             "clocks": clocks,
+            "ms_per_step_x_sm_mhz": (ms / args.steps) * mhz if mhz else None,
             "e2e": {"value": px_step * args.steps / (e2e_ms * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": h_seg.numel() * h_seg.element_size(),
                     "d2h_bytes_per_step": h_out.numel() * h_out.element_size()},
@@ -308,11 +402,17 @@ def run_ours(args, w):
                           "note": "segments pushed as they arrive for all streams, the last push carries the end of input"},
             "roofline": {"bound": "tensor", "kernel": "dense conv update (all conv layers)", "achieved": achieved,
                          "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak if peak else None,
-                         "peak_source": f"{peaks['source']} bf16 sustained x{ratio}", "traffic": traffic,
-                         "traffic_note": traffic_note,
+                         "peak_source": f"{peaks['source']} bf16 {kind} x{ratio} (timed region {timed_s:.3f} s)",
+                         "frac_of_burst": achieved / (peaks["bf16_burst"] * ratio),
+                         "frac_of_sustained": achieved / (peaks["bf16_sustained"] * ratio),
+                         "frac_of_burst_whole_step": flops / (ms / args.steps * 1e-3) / 1e12 / (peaks["bf16_burst"] * ratio),
+                         "traffic": traffic, "traffic_note": traffic_note,
+                         "algorithmic_bytes": algorithmic_bytes(w, net),
                          "launches_per_step": dom_launches, "ms_per_step": dom_ms,
                          "layer_ms": [round(v, 4) for v in lms]},
         }
+        if world == 1 and args.extra:
+            line["extra"] = extra_workloads(args, w.name, dev, flush_buf, stream, barrier, peaks)
         if world == 1 and not args.no_cpu:
             rate, cores, sample, _ = oracle_rate(w, budget_s=25.0)
             line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
@@ -332,6 +432,7 @@ def main():
     ap.add_argument("--rows", type=int, default=None, help="segments per stream (default: the workload's; shorter runs are for profiling)")
     ap.add_argument("--row-block", type=int, default=0)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--extra", action="store_true", help="also time the other workloads (device time only) under an 'extra' key")
     args = ap.parse_args()
     w = workloads.get(args.workload, n_streams=args.streams, H=args.rows)
     if args.impl == "reference":

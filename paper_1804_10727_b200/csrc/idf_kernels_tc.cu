@@ -677,9 +677,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint64_t bdesc_base = desc_hi | (uint64_t)((sW & 0x3FFFFu) >> 4);
             const int n_st = n_xload * n_kb;                     // tiles per input row
             const bool issuer = elect_one();                     // the lane that issues (the warp stays converged)
-            int stage = 0;
-            uint32_t phase = 0;
-            uint64_t adesc_stage = adesc_base;                   // descriptor of the current stage's tile
             ok = ok && mbar_wait(bar_full, 0, abort_flag);       // first tile of the first row
             tc_fence_after();
             uint4 hdr = make_uint4(0, 0, 0, 0), sa = hdr, sb = hdr, sc = hdr;
@@ -687,59 +684,81 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const uint4* q = (const uint4*)s_rowq[0];
                 hdr = q[0]; sa = q[1]; sb = q[2]; sc = q[3];
             }
-            for (int ri = 0; ri < n_rows && ok; ++ri) {
+            // The loop runs over tiles (input row, kx box, K block), software-pipelined by hand: everything the NEXT
+            // tile needs (stage, barrier, descriptors, and on a row's last tile the next row's schedule entry) is worked
+            // out between the first and the last MMA group of the CURRENT tile, while the pipe is busy, so that between
+            // the last MMA of one tile and the first MMA of the next there is only the commit and a handful of moves.
+            // tap kx reads the same tile kxi rows further down: the swizzle is a function of the absolute
+            // shared-memory address, so a start address moved by whole rows still meets the pattern the TMA
+            // wrote (base-offset field stays 0).
+            const uint32_t b_xl_step = a.shift_mode ? 0u : wtile_kx;       // weight blocks of the next kx box (one box per kx)
+            int ri = 0, st = 0, kb = 0, stage = 0;
+            uint32_t phase = 0;
+            uint64_t adesc_cur = adesc_base, bdesc_cur = bdesc_base;       // the tile at hand
+            const long long n_tiles = (long long)n_rows * n_st;
+            for (long long tile = 0; tile < n_tiles && ok; ++tile) {
+                const bool row_end = st == n_st - 1;
                 const bool last_row = ri == n_rows - 1;
-                // schedule entries are published 32 rows at a time, ahead of the first copy of those rows
-                const bool early_info = !last_row && ((ri + 1) & 31) != 0;
-                const uint4* qn = (const uint4*)s_rowq[(ri + 1) & (ROWQ - 1)];
-                uint4 nh = make_uint4(0, 0, 0, 0), na = nh, nb = nh, nc = nh;
-                int st = 0;
-                for (int xl = 0; xl < n_xload && ok; ++xl)
-                    for (int kb = 0; kb < n_kb; ++kb, ++st) {
-                        const bool row_end = st == n_st - 1;
-                        int nstage_i = stage + 1;
-                        uint32_t nphase = phase;
-                        uint64_t adesc_next = adesc_stage + a_stage_units;
-                        if (nstage_i == nstage) { nstage_i = 0; nphase ^= 1u; adesc_next = adesc_base; }
-                        // tap kx reads the same tile kxi rows further down: the swizzle is a function of
-                        // the absolute shared-memory address, so a start address moved by whole rows
-                        // still meets the pattern the TMA wrote (base-offset field stays 0)
-                        uint64_t adesc = adesc_stage;
-                        uint64_t bdesc = bdesc_base + (uint64_t)((a.shift_mode ? 0u : (uint32_t)xl) * wtile_kx + (uint32_t)kb * wtile_kb);
-                        uint32_t next_ok = 1u;
-                        for (int kxi = 0; kxi < n_kx; ++kxi, adesc += kx_bytes, bdesc += wtile_kx) {
-                            if (issuer && hdr.z > 0) {
-                                umma_tile<DT, KSTEPS>(sa.x, adesc, bdesc + (uint64_t)sa.y, sa.z);
-                                if (hdr.z > 1) {
-                                    umma_tile<DT, KSTEPS>(sa.w, adesc, bdesc + (uint64_t)sb.x, sb.y);
-                                    if (hdr.z > 2) umma_tile<DT, KSTEPS>(sb.z, adesc, bdesc + (uint64_t)sb.w, sc.x);
-                                    if (hdr.z > 3) umma_tile<DT, KSTEPS>(sc.y, adesc, bdesc + (uint64_t)sc.z, sc.w);
-                                }
-                            }
-                            if (kxi == 0) {
-                                // with the first MMAs of the tile queued: look at the next tile's barrier and
-                                // fetch the next row's schedule entry
-                                if (!(last_row && row_end)) next_ok = mbar_test(bar_full + 8u * nstage_i, nphase);
-                                if (row_end && early_info) { nh = qn[0]; na = qn[1]; nb = qn[2]; nc = qn[3]; }
-                            }
-                        }
-                        if (issuer) {
-                            umma_commit(bar_empty + 8u * stage);
-                            if (row_end) {
-                                // the accumulator this input row completed; on the block's last row also everything still open
-                                // (to be parked in the ring, or emitted if only bottom padding was missing)
-                                if (hdr.w) umma_commit(hdr.w);
-                                if (last_row)
-                                    for (int orel = c_sched_rel; orel < c_n_orows; ++orel) umma_commit(bar_ready + 8u * (uint32_t)(orel % nslot));
-                            }
-                        }
-                        if (!next_ok && !mbar_wait(bar_full + 8u * nstage_i, nphase, abort_flag)) { ok = false; break; }
-                        stage = nstage_i; phase = nphase; adesc_stage = adesc_next;
+                // ---- first MMA group of the tile
+                if (issuer && hdr.z > 0) {
+                    umma_tile<DT, KSTEPS>(sa.x, adesc_cur, bdesc_cur + (uint64_t)sa.y, sa.z);
+                    if (hdr.z > 1) {
+                        umma_tile<DT, KSTEPS>(sa.w, adesc_cur, bdesc_cur + (uint64_t)sb.x, sb.y);
+                        if (hdr.z > 2) umma_tile<DT, KSTEPS>(sb.z, adesc_cur, bdesc_cur + (uint64_t)sb.w, sc.x);
+                        if (hdr.z > 3) umma_tile<DT, KSTEPS>(sc.y, adesc_cur, bdesc_cur + (uint64_t)sc.z, sc.w);
                     }
-                if (!ok || last_row) break;
-                if (!early_info) { nh = qn[0]; na = qn[1]; nb = qn[2]; nc = qn[3]; }
-                hdr = nh; sa = na; sb = nb; sc = nc;
-                tc_fence_after();                                // the next row may start on a slot the epilogue has just cleared
+                }
+                // ---- the next tile, worked out while those run
+                int n_stage = stage + 1;
+                uint32_t n_phase = phase;
+                uint64_t adesc_nx = adesc_cur + a_stage_units;
+                if (n_stage == nstage) { n_stage = 0; n_phase ^= 1u; adesc_nx = adesc_base; }
+                uint64_t bdesc_nx = bdesc_cur + wtile_kb;
+                int n_kbi = kb + 1;
+                if (n_kbi == n_kb) { n_kbi = 0; bdesc_nx += (uint64_t)b_xl_step - (uint64_t)((uint32_t)n_kb * wtile_kb); }
+                if (row_end) bdesc_nx = bdesc_base;
+                uint32_t next_ok = 1u;
+                if (!(last_row && row_end)) next_ok = mbar_test(bar_full + 8u * n_stage, n_phase);
+                uint4 nh = hdr, na = sa, nb = sb, nc = sc;
+                // schedule entries are published 32 rows at a time, ahead of the first copy of those rows
+                const bool early_info = row_end && !last_row && ((ri + 1) & 31) != 0;
+                const uint4* qn = (const uint4*)s_rowq[(ri + 1) & (ROWQ - 1)];
+                if (early_info) { nh = qn[0]; na = qn[1]; nb = qn[2]; nc = qn[3]; }
+                // ---- the other kx taps of the tile (row-shifted reads of the same box)
+                {
+                    uint64_t adesc = adesc_cur + kx_bytes, bdesc = bdesc_cur + wtile_kx;
+                    for (int kxi = 1; kxi < n_kx; ++kxi, adesc += kx_bytes, bdesc += wtile_kx) {
+                        if (issuer && hdr.z > 0) {
+                            umma_tile<DT, KSTEPS>(sa.x, adesc, bdesc + (uint64_t)sa.y, sa.z);
+                            if (hdr.z > 1) {
+                                umma_tile<DT, KSTEPS>(sa.w, adesc, bdesc + (uint64_t)sb.x, sb.y);
+                                if (hdr.z > 2) umma_tile<DT, KSTEPS>(sb.z, adesc, bdesc + (uint64_t)sb.w, sc.x);
+                                if (hdr.z > 3) umma_tile<DT, KSTEPS>(sc.y, adesc, bdesc + (uint64_t)sc.z, sc.w);
+                            }
+                        }
+                    }
+                }
+                if (issuer) {
+                    umma_commit(bar_empty + 8u * stage);
+                    if (row_end) {
+                        // the accumulator this input row completed; on the block's last row also everything still open
+                        // (to be parked in the ring, or emitted if only bottom padding was missing)
+                        if (hdr.w) umma_commit(hdr.w);
+                        if (last_row)
+                            for (int orel = c_sched_rel; orel < c_n_orows; ++orel) umma_commit(bar_ready + 8u * (uint32_t)(orel % nslot));
+                    }
+                }
+                if (!next_ok && !mbar_wait(bar_full + 8u * n_stage, n_phase, abort_flag)) { ok = false; break; }
+                stage = n_stage; phase = n_phase; adesc_cur = adesc_nx; bdesc_cur = bdesc_nx; kb = n_kbi;
+                if (row_end) {
+                    if (last_row) break;
+                    if (!early_info) { nh = qn[0]; na = qn[1]; nb = qn[2]; nc = qn[3]; }   // (published with the tile just waited for)
+                    hdr = nh; sa = na; sb = nb; sc = nc;
+                    st = 0; ++ri;
+                    tc_fence_after();                            // the next row may start on a slot the epilogue has just cleared
+                } else {
+                    ++st;
+                }
             }
         }
         __syncwarp();
