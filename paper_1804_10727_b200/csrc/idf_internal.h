@@ -82,6 +82,7 @@ struct TcPlan {
     int nstage = 0;          // Δ-row tiles in flight
     int tmem_cols = 0;
     int out_groups = 0;
+    int out_bufs = 1;        // staging tiles per epilogue group (2: a row is laid out while the previous store still drains)
     int out_esize = 0, out_pwb = 0, out_panels = 0, out_stage_bytes = 0;   // staging of emitted rows for the TMA store
     int out_stage_rows = 0;  // rows of one staging panel: 128, or 64 in a plan for launches that emit pooled rows
     size_t smem_bytes = 0;

@@ -237,8 +237,9 @@ __device__ __forceinline__ void tmem_ld(uint32_t taddr, uint32_t (&v)[W])
               "=r"(v[28 % W]), "=r"(v[29 % W]), "=r"(v[30 % W]), "=r"(v[31 % W])
             : "r"(taddr) : "memory");
     }
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// (the registers of a tcgen05.ld are valid after this wait: several loads may be in flight before it)
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 template <int W>
 __device__ __forceinline__ void tmem_st_zero(uint32_t taddr)
 {
@@ -466,7 +467,8 @@ struct TcArgs {
     int a_stage_bytes;
     int out_esize, out_pwb, out_panels, out_stage_bytes;   // emitted rows: staging panels of out_pwb-byte rows
     int out_stage_rows;          // rows of one staging panel: 128, or 64 when only pooled rows are staged
-    int out_groups;              // epilogue groups at work (1 or 2), each with its own staging tile
+    int out_groups;              // epilogue groups at work, each with its own staging tile(s)
+    int out_bufs;                // staging tiles per group (1 or 2, used in turn)
     int out_row_dim;             // position of the row coordinate in the output tensor map (2 or 3)
     int out_row_first;           // tensor-map row index of relative output row 0
     // 2x2 max-pooling folded into the emission (the output tensor map then describes the pooled rows)
@@ -474,6 +476,11 @@ struct TcArgs {
     int pool_keep;               // 1: a trailing first row of a pair waits in pool_state for a later launch; 0: end of input, it is dropped
     void* pool_state;            // [S][Wout/2][Cout] in the output type: x-pooled first row of an open pair
     long long pool_row_base;     // pooled row p goes to tensor-map row p - pool_row_base
+    // small pieces of o_begin, so that the row loop needs no 64-bit arithmetic
+    int o_begin_par;             // o_begin & 1
+    int o_begin_half_mod;        // (o_begin >> 1) mod out_groups
+    int ring_slot0;              // o_begin mod ring_rows
+    int pool_row_first;          // (o_begin >> 1) - pool_row_base: tensor-map row of the pair that holds o_begin
 };
 
 template <int DT> struct Acc;
@@ -504,7 +511,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t sW = base;
     const uint32_t sA = (sW + (uint32_t)taps * a.n_kb * w_tile_bytes + 1023u) & ~1023u;
     const uint32_t sOut = sA + (uint32_t)a.nstage * a_stage_bytes;               // one staging tile per epilogue group
-    const uint32_t bars = sOut + (uint32_t)a.out_groups * (uint32_t)a.out_stage_bytes;
+    const uint32_t bars = sOut + (uint32_t)(a.out_groups * a.out_bufs) * (uint32_t)a.out_stage_bytes;
     const uint32_t bar_full = bars;
     const uint32_t bar_empty = bar_full + 8u * a.nstage;
     const uint32_t bar_w = bar_empty + 8u * a.nstage;
@@ -527,7 +534,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (c_ra < 0) c_ra = 0;
     int c_rb = (c_ob - 1) * a.stride - a.base_ty + a.Kh;                                           // one past the last
     if (c_rb > a.n_rows || chunk == a.n_chunks - 1) c_rb = a.n_rows;
-    const long long c_o_begin = a.o_begin + c_oa;
     const int c_base_ty = a.base_ty + c_ra - c_oa * a.stride;
     const int c_n_orows = c_ob - c_oa;
     const int c_done_rel = min(max(a.done_rel - c_oa, 0), c_n_orows);
@@ -787,10 +793,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         StageSink sink;
         sink.pwb_log2 = 31u - (uint32_t)__clz(a.out_pwb);
         sink.panel_bytes = (uint32_t)a.out_stage_rows * (uint32_t)a.out_pwb;
-        sink.row_base = sOut + (uint32_t)grp * a.out_stage_bytes + (uint32_t)md * a.out_pwb;
+        sink.row_base = sOut + (uint32_t)(grp * a.out_bufs) * a.out_stage_bytes + (uint32_t)md * a.out_pwb;
         sink.phase = a.out_pwb == 128 ? (uint32_t)(md & 7) : (a.out_pwb == 64 ? (uint32_t)((md >> 1) & 3)
                    : (a.out_pwb == 32 ? (uint32_t)((md >> 2) & 1) : 0u));
-        const uint32_t stg = sOut + (uint32_t)grp * a.out_stage_bytes;
+        uint32_t stg = sOut + (uint32_t)(grp * a.out_bufs) * a.out_stage_bytes;     // the staging tile in use
+        uint32_t buf_step = a.out_bufs > 1 ? (uint32_t)a.out_stage_bytes : 0u;      // to the group's other tile (sign flips per store)
         const int panel_cols = a.out_pwb / a.out_esize;
         PoolCtx pc;
         pc.on = a.pool; pc.second = 0; pc.from_state = 0; pc.to_state = 0; pc.drop = 0;
@@ -817,61 +824,68 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // those left open by this one) may share a ring slot; group 0 takes them all, in order, so a
         // slot is read before it is rewritten.  The other rows go round the groups.
         const int n_cin = c_r0_positive ? (c_base_ty + a.stride - 1) / a.stride : 0;
-        for (int orel = 0; orel < c_n_orows && ok && grp < a.out_groups; ++orel) {
+        // Per-row bookkeeping is kept with small counters that step from row to row (a division or a 64-bit
+        // operation per row and thread costs more than the row's arithmetic): TMEM slot and barrier parity of the row,
+        // its ring slot in global memory, the parity of its absolute index, the group whose turn it is.
+        const int G = a.out_groups;
+        int slot_c = 0;                                       // orel mod nslot
+        uint32_t par_c = 0;                                   // (orel div nslot) & 1
+        int turn = 0;                                         // orel mod G
+        int absp = (a.o_begin_par + c_oa) & 1;                // parity of the row's absolute index
+        int pair_turn = (a.o_begin_half_mod + ((a.o_begin_par + c_oa) >> 1)) % G;   // (absolute index div 2) mod G
+        int rslot_c = (a.ring_slot0 + c_oa) % a.ring_rows;    // absolute index mod ring_rows
+        for (int orel = 0; orel < c_n_orows && ok && grp < G; ++orel) {
             int owner;
             if (!a.pool) {
-                owner = (orel < n_cin || orel >= c_done_rel) ? 0 : orel % a.out_groups;
+                owner = (orel < n_cin || orel >= c_done_rel) ? 0 : turn;
             } else {
                 // both rows of a pooling pair go to one group; pairs touching the global ring or the pool layer's state
                 // (first < 0: the pair's first row came with an earlier launch) go to group 0
-                const int first = orel - (int)((c_o_begin + orel) & 1);
-                owner = (first < 0 || first < n_cin || first + 1 >= c_done_rel) ? 0 : (int)(((c_o_begin + orel) >> 1) % a.out_groups);
+                const int first = orel - absp;
+                owner = (first < 0 || first < n_cin || first + 1 >= c_done_rel) ? 0 : pair_turn;
             }
+            const int slot = slot_c, rslot = rslot_c, row_odd = absp;
+            const uint32_t par = par_c;
+            // the counters move on to the next row
+            if (++slot_c == a.nslot) { slot_c = 0; par_c ^= 1u; }
+            if (++turn == G) turn = 0;
+            if (++rslot_c == a.ring_rows) rslot_c = 0;
+            if (absp && ++pair_turn == G) pair_turn = 0;
+            absp ^= 1;
             if (owner != grp) continue;
-            const int slot = orel % a.nslot;
-            const uint32_t par = (uint32_t)((orel / a.nslot) & 1);
             const bool emit = orel < c_done_rel;
-            // one thread of the group polls the barrier; the named barrier below releases the other warps
+            // one thread of the group polls the barrier; the named barrier below releases the other warps.
+            // The tile must have been drained by the group's previous store before anyone writes it again: that
+            // wait comes first, it overlaps the wait for the row.
             int got = 1;
-            if (leader) got = mbar_wait_relaxed(bar_ready + 8u * slot, par, abort_flag) ? 1 : 0;
-            // the tile must have been drained by the group's previous store before anyone writes it again;
-            // the barrier also makes the whole group leave together if any of its waits ran out
-            if (emit && leader) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            if (leader) {
+                // (with two tiles the latest store may still be draining: it reads the other one)
+                if (emit) {
+                    if (a.out_bufs > 1) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                }
+                got = mbar_wait_relaxed(bar_ready + 8u * slot, par, abort_flag) ? 1 : 0;
+            }
+            // (the barrier also makes the whole group leave together if any of its waits ran out)
             if (!named_bar_and(1 + grp, 128, got != 0)) { ok = false; break; }
             tc_fence_after();
             const bool carried_in = c_r0_positive && (orel * a.stride - c_base_ty < 0);
             const bool pool_emit = a.pool && emit;
             if (pool_emit) {
-                pc.second = (int)((c_o_begin + orel) & 1);
+                pc.second = row_odd;
                 pc.from_state = pc.second && orel == 0;
                 const bool trailing = !pc.second && orel == c_done_rel - 1 && c_oa + c_done_rel == a.done_rel;   // the block's last emitted row
                 pc.to_state = trailing && a.pool_keep;
                 pc.drop = trailing && !a.pool_keep;
             }
-            TS* rp = ring_pos + (long long)((c_o_begin + orel) % a.ring_rows) * ring_slot_stride;
+            TS* rp = ring_pos + (long long)rslot * ring_slot_stride;
             const uint32_t trow = tlane + (uint32_t)(slot * a.Ntile);
-            if (a.Ntile == 64 || a.Ntile == 32) {
-                // the whole row fits in registers: take it, clear and release the slot at once, then finalise
-                uint32_t v0[32], v1[32];
-                tmem_ld<32>(trow, v0);
-                if (a.Ntile == 64) tmem_ld<32>(trow + 32, v1);
-                tmem_st_zero<32>(trow);
-                if (a.Ntile == 64) tmem_st_zero<32>(trow + 32);
-                tmem_st_wait();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_free + 8u * slot);   // one arrival per warp
-                if (pool_emit || (emit ? in_tile : valid)) {
-                    finalise_chunk<DT, 32, TS>(v0, carried_in && valid, emit, rp, bias, sink, 0u, a.out_elem, a.relu, a.shift, pc, state_ok, carry_off);
-                    if (a.Ntile == 64)
-                        finalise_chunk<DT, 32, TS>(v1, carried_in && valid, emit, rp + 32, bias ? bias + 32 : nullptr, sink,
-                                                   (uint32_t)(32 * a.out_esize), a.out_elem, a.relu, a.shift, pc, state_ok, carry_off);
-                }
-            } else {
+            {
                 if (wide) {
                     for (int c = 0; c < a.Ntile; c += 32) {
                         uint32_t v[32];
                         tmem_ld<32>(trow + c, v);
+                        tmem_ld_wait();
                         tmem_st_zero<32>(trow + c);           // the slot's next row starts from zero
                         if (pool_emit || (emit ? in_tile : valid))
                             finalise_chunk<DT, 32, TS>(v, carried_in && valid, emit, rp + c, bias ? bias + c : nullptr, sink,
@@ -881,6 +895,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int c = 0; c < a.Ntile; c += 16) {
                         uint32_t v[16];
                         tmem_ld<16>(trow + c, v);
+                        tmem_ld_wait();
                         tmem_st_zero<16>(trow + c);
                         if (pool_emit || (emit ? in_tile : valid))
                             finalise_chunk<DT, 16, TS>(v, carried_in && valid, emit, rp + c, bias ? bias + c : nullptr, sink,
@@ -896,7 +911,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 named_bar_sync(1 + grp, 128);
                 if (leader) {
-                    const int orow = a.pool ? (int)(((c_o_begin + orel) >> 1) - a.pool_row_base) : a.out_row_first + c_oa + orel;
+                    const int orow = a.pool ? a.pool_row_first + ((a.o_begin_par + c_oa + orel) >> 1) : a.out_row_first + c_oa + orel;
                     const int xc = a.pool ? (x0 >> 1) : x0;
                     for (int pnl = 0; pnl < a.out_panels; ++pnl) {
                         if (a.out_row_dim == 3)
@@ -906,6 +921,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
+                // the group's next row is laid out in its other tile
+                stg += buf_step; sink.row_base += buf_step; pc.sink.row_base += buf_step;
+                buf_step = 0u - buf_step;
             }
         }
         if (leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
@@ -1033,15 +1051,18 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     p->out_stage_bytes = p->out_panels * stage_rows * p->out_pwb;
     // as many epilogue groups (one staging tile each) as still leave three Δ-row stages
     p->out_groups = 1;
+    p->out_bufs = 1;
     // layers with many short K blocks per row (little MMA work per tile) need a deeper pipeline to cover the
     // copy latency more than they need a second epilogue group
     const size_t want_stages = p->n_kb >= 4 ? 4 : 3;
     for (int g = MAX_GROUPS; g > 1; --g)
         if (wb + want_stages * a_stage + (size_t)g * p->out_stage_bytes + 10240 <= SMEM_LIMIT) { p->out_groups = g; break; }
+    // a second staging tile per group where it still leaves one more Δ-row stage than wanted
+    if (wb + (want_stages + 1) * a_stage + 2 * (size_t)p->out_groups * p->out_stage_bytes + 10240 <= SMEM_LIMIT) p->out_bufs = 2;
     // the MMAs' run past a small box (see a_stage) must end inside this CTA's shared memory: what follows the
     // last stage (the staging tiles) covers it, or padding is added behind them
     const size_t overrun = (size_t)(128 + halo) * p->swb > a_stage ? (size_t)(128 + halo) * p->swb - a_stage : 0;
-    const size_t tail_have = (size_t)p->out_groups * p->out_stage_bytes;
+    const size_t tail_have = (size_t)p->out_groups * p->out_bufs * p->out_stage_bytes;
     const size_t tail_pad = overrun > tail_have ? (overrun - tail_have + 1023) / 1024 * 1024 : 0;
     if (SMEM_LIMIT < 8192 + wb + 1024 + tail_have + tail_pad + 2 * a_stage) return false;
     const size_t room = SMEM_LIMIT - 8192 - wb - 1024 - tail_have - tail_pad;   // static shared memory and alignment slack stay free
@@ -1049,7 +1070,7 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     if (nstage > 8) nstage = 8;
     if (nstage < 2) return false;
     p->nstage = nstage;
-    p->smem_bytes = 1024 + wb + (size_t)nstage * a_stage + (size_t)p->out_groups * p->out_stage_bytes + tail_pad + 8 * (2 * nstage + taps + 2 * p->nslot) + 64;
+    p->smem_bytes = 1024 + wb + (size_t)nstage * a_stage + tail_have + tail_pad + 8 * (2 * nstage + taps + 2 * p->nslot) + 64;
     p->w_bytes = (size_t)taps * Cout * Cin * esize;
     p->ok = 1;
     return true;
@@ -1137,9 +1158,13 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     t.BX = p.BX; t.BS = p.BS; t.n_xt = p.n_xt; t.Ntile = p.Ntile; t.n_nt = p.n_nt; t.KB = p.KB; t.n_kb = p.n_kb;
     t.swb = p.swb; t.nslot = p.nslot; t.nstage = p.nstage; t.tmem_cols = p.tmem_cols;
     t.BXP = p.BXP; t.shift_mode = p.shift_mode; t.sx = p.sx; t.a_stage_bytes = p.a_stage_bytes;
-    t.out_esize = p.out_esize; t.out_pwb = p.out_pwb; t.out_panels = p.out_panels; t.out_stage_bytes = p.out_stage_bytes; t.out_stage_rows = p.out_stage_rows; t.out_groups = p.out_groups;
+    t.out_esize = p.out_esize; t.out_pwb = p.out_pwb; t.out_panels = p.out_panels; t.out_stage_bytes = p.out_stage_bytes; t.out_stage_rows = p.out_stage_rows; t.out_groups = p.out_groups; t.out_bufs = p.out_bufs;
     t.out_row_dim = row_dim; t.out_row_first = (int)(a.o_begin - a.out_row_base);
     t.pool = a.pool_fused; t.pool_keep = a.pool_keep; t.pool_state = a.pool_state; t.pool_row_base = a.out_row_base;
+    t.o_begin_par = (int)(a.o_begin & 1);
+    t.o_begin_half_mod = (int)((a.o_begin >> 1) % p.out_groups);
+    t.ring_slot0 = (int)(a.o_begin % a.ring_rows);
+    t.pool_row_first = (int)((a.o_begin >> 1) - a.out_row_base);
     // row chunks: a layer with few tiles (few streams, narrow rows) spreads the block's rows over more CTAs
     t.n_chunks = 1; t.chunk_rows = t.n_orows; t.chunk_shift = 0;
     {

@@ -58,3 +58,92 @@ def test_full_size_state_bytes_are_the_ring_formula():
         w = workloads.get(name)
         net = idf.net_from_workload(w, *workloads.make_params(w))
         assert net.state_bytes == b
+
+
+# ---- strict bf16 parity, layer by layer, in the tile plans the full-size batch uses -----------------------
+def _layer_inputs(w):
+    """(index, layer, H, W, C of its input, pool follows?, is it the net's last conv?) for every conv layer."""
+    H, W, C = w.H, w.W, w.C
+    convs = [i for i, l in enumerate(w.layers) if l.kind == "conv"]
+    out = []
+    for i, l in enumerate(w.layers):
+        if l.kind == "conv":
+            pool_next = i + 1 < len(w.layers) and w.layers[i + 1].kind == "pool"
+            out.append((i, l, H, W, C, pool_next, i == convs[-1]))
+            H = (H + 2 * l.pad - l.kh) // l.stride + 1
+            W = 1 if W == 1 else (W + 2 * l.pad - l.kw) // l.stride + 1
+            C = l.cout
+        else:
+            H, W = H // 2, (1 if W == 1 else W // 2)
+    return out
+
+
+def _bf16_down_up(v):
+    """The bfloat16 values just below-or-equal and just above-or-equal every entry of v (float64 in, float64 out)."""
+    f = np.asarray(v, dtype=np.float64)
+    r = torch.from_numpy(f).float().bfloat16().float().numpy()          # nearest bf16 (as float32)
+    bits = r.view(np.uint32).astype(np.int64)
+    mag, neg = bits & 0x7FFFFFFF, (bits >> 31) != 0
+    tiny = np.float32(2.0 ** -133)
+
+    def from_parts(m, n):
+        return ((m.astype(np.uint32)) | (n.astype(np.uint32) << 31)).view(np.float32)
+    # one bf16 step toward +inf / toward -inf
+    up_mag = np.where(neg, mag - 0x10000, mag + 0x10000)
+    up = np.where(mag == 0, tiny, from_parts(np.maximum(up_mag, 0), neg & (up_mag > 0)))
+    dn_mag = np.where(neg, mag + 0x10000, mag - 0x10000)
+    dn = np.where(mag == 0, -tiny, from_parts(np.maximum(dn_mag, 0), neg | (dn_mag < 0)))
+    dn = np.where((~neg) & (dn_mag == 0), np.float32(0.0), dn)
+    r64 = r.astype(np.float64)
+    lo = np.where(r64 <= f, r64, dn.astype(np.float64))
+    hi = np.where(r64 >= f, r64, up.astype(np.float64))
+    return lo, hi
+
+
+@pytest.mark.parametrize("name,sample", [("vgg2d", [0, 37, 63]), ("audio1d", [0, 700, 1023])])
+def test_bf16_layers_strict_in_the_full_size_plans(orc, name, sample):
+    """Every conv layer of the bf16 workloads at the FULL stream count (so that the kernel picks the tiles, stream
+    packing, row chunks and pool folding it uses in the benchmarked batch), fed a seeded bf16 map of the layer's real
+    input shape; the oracle recomputes sampled streams.  The net's last conv layer emits unrounded fp32 and is held
+    to |g - o| <= 1e-4 + 1e-3 |o| directly.  A hidden layer must round to bf16 (so that its tile plan is the one of
+    the full net); a 1x1 identity conv behind it passes the rounded values through exactly, and each must be the
+    bf16 rounding of SOME value within that tolerance of the oracle's unrounded result."""
+    w = workloads.get(name)
+    ws, bs = workloads.make_params(w)
+    S = w.n_streams
+    for i, l, H, W, C, pool_next, is_last in _layer_inputs(w):
+        g = torch.Generator().manual_seed(1000 + 17 * i)
+        # post-ReLU-like activations (the first layer sees the signed input): bf16 values, segment layout [H][S][W][C]
+        seg = torch.empty((H, S, W, C), dtype=torch.bfloat16)
+        for h0 in range(0, H, 64):
+            blk = torch.randn((min(64, H - h0), S, W, C), generator=g)
+            seg[h0:h0 + 64] = (blk if i == 0 else blk.abs()).bfloat16()
+        layers = [l] + ([workloads.POOL] if pool_next else [])
+        wts, bias = [ws[i]] + ([None] if pool_next else []), [bs[i]] + ([None] if pool_next else [])
+        if not is_last:
+            layers.append(workloads.conv(l.cout, l.cout, 1, one_d=(W == 1), relu=0))
+            wts.append(np.eye(l.cout, dtype=np.float32).reshape(l.cout, 1, 1, l.cout)); bias.append(None)
+        net = idf.Net("bf16", tuple(layers), W, C, S, wts, bias)
+        out = net.alloc_out(H)
+        net.open()
+        rows = net.push_last(seg.cuda(), out)
+        tc = net.status()
+        assert tc[0] > 0 or C * 2 < 32, f"{name} layer {i}: not on the tensor-core path"
+        for s in sample:
+            a = seg[:, s].float().numpy()[None]                              # [1][H][W][C]
+            want = orc.conv_layer("bf16", l, a, ws[i], bs[i])                # unrounded f(c), float64
+            if pool_next:
+                want = orc.pool_layer("bf16", want)
+            got = out[s, :rows].cpu().numpy().astype(np.float64)
+            assert got.shape == want[0].shape, (got.shape, want.shape)
+            tol = 1e-4 + 1e-3 * np.abs(want[0])
+            if is_last:
+                bad = np.abs(got - want[0]) > tol
+            else:
+                lo, _ = _bf16_down_up(want[0] - tol)
+                _, hi = _bf16_down_up(want[0] + tol)
+                bad = (got < lo) | (got > hi)
+            assert not bad.any(), f"{name} layer {i} stream {s}: {bad.sum()} of {bad.size} outside the strict tolerance"
+        net.close()
+        del seg, out
+        torch.cuda.empty_cache()
