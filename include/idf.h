@@ -67,6 +67,27 @@ typedef enum {
  * state, and every arriving row adds its share w * dh at once. */
 typedef enum { IDF_PATH_AUTO = 0, IDF_PATH_DENSE = 1, IDF_PATH_SPARSE = 2 } idf_path;
 
+/* When a unit passes a change of its activation on.
+ *   IDF_EMIT_DEFERRED  once, when no present or future segment can reach it any more (see the file header): state of
+ *                      ceil(Kh/stride) rows per conv layer, the operation count of conventional inference, every
+ *                      kernel of the library.  Output rows appear when they are final.
+ *   IDF_EMIT_EAGER     the paper's literal rule (Eq. 3-5): after every segment each unit whose activation f(c) has
+ *                      changed announces dh = h(t) - h(t-1), the layer above adds w * dh to its states (Eq. 4) and
+ *                      re-evaluates in turn, within the same push.  The net's output is then an ANYTIME output: after
+ *                      every idf_stream_push, d_out holds, below the finished rows, also the rows a later segment can
+ *                      still reach, with the activation they have announced so far, and converges to the conventional
+ *                      result as the input arrives (Section "Experimental verification", Fig. 3-4); rows_emitted still
+ *                      counts finished rows only, and out_capacity_rows must cover every row touched.  A unit
+ *                      announces partial sums, so a layer keeps all rows of its input cone (state and announced
+ *                      activation: idf_net_state_bytes reports them) and a unit is updated once per segment of its
+ *                      receptive field.  Units of rows that turn out to lie beyond the end of the input (known only
+ *                      at idf_stream_finish) take back what they announced.  A max-pool unit holds its four current
+ *                      inputs (0 for units that have announced nothing) and announces max_new - max_old.  Runs on
+ *                      CUDA cores, one launch per layer and segment; IDF_GLOBAL_AVG, idf_stream_set_out_base and the
+ *                      snapshot calls are not available (IDF_ERR_UNSUPPORTED), the first layer must be a conv
+ *                      layer.  idf_event_counts: events[i] = non-zero changes layer i has received. */
+typedef enum { IDF_EMIT_DEFERRED = 0, IDF_EMIT_EAGER = 1 } idf_emission;
+
 typedef enum {
     IDF_OK = 0,
     IDF_ERR_ARG = -1,          /* null pointer, negative count, ...                                   */
@@ -97,6 +118,7 @@ typedef struct {
     int n_streams;             /* streams advanced together by every call */
     int row_block;             /* most segments pushed through all layers at once (bounds the   */
                                /* transient workspace); 0 = library default                     */
+    int emission;              /* idf_emission; 0 = IDF_EMIT_DEFERRED                           */
 } idf_spec;
 
 /* Build a net from a layer list and the parameters of a conventionally trained CNN
@@ -130,6 +152,11 @@ size_t idf_net_workspace_bytes(const idf_net* net);
  * Introduction).  out_rows may be 0.  Any out pointer may be NULL.  IDF_ERR_ARG for a NULL net or
  * negative in_rows. */
 int idf_out_shape(const idf_net* net, long long in_rows, long long* out_rows, int* out_w, int* out_c);
+
+/* Rows per stream the output buffer must hold (out_capacity_rows) for streams of in_rows segments: the rows of the
+ * final map (idf_out_shape) and, with IDF_EMIT_EAGER, also the rows above them that the last segments touch with
+ * partial activations before the end of input takes those back.  -1 for a NULL net or negative in_rows. */
+long long idf_out_rows_needed(const idf_net* net, long long in_rows);
 
 /* Start streams: every unit's state variable c and activation begin at zero (the paper's convention
  * in the paragraph after Eq. 3: all units start at 0, so the first events are the inputs themselves).

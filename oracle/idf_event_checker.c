@@ -13,8 +13,10 @@
  * nets the final maps produced here, one input component at a time, must equal
  * the layer-by-layer result (the equivalence stated after Eq. 5).
  *
- * Two emission policies:
- *   eager    - the paper's: a unit emits the moment its activation changes.
+ * Emission policies:
+ *   eager    - the paper's: a unit emits the moment its activation changes (one input component at a time).
+ *   eager, per segment (eager == 2) - the same rule with all components of a segment delivered before the
+ *              layers re-evaluate, one layer after the other: a unit emits h(after the segment) - h(before).
  *   deferred - a unit emits once, when no present or future input can reach
  *              it any more (its row has received its last kernel tap); this
  *              is the policy under which a layer needs only ceil(Kh/stride)
@@ -141,7 +143,7 @@ static void deliver(evc_net* N, int n, int y, int x, int ch, double d)
                     N->c[n][i] += N->w[n - 1][(((size_t)co * l->kh + ky) * l->kw + kx) * l->cin + ch] * d;
                     N->touched[n][i] = 1;
                     N->n_updates[n] += 1;
-                    if (N->eager) reevaluate(N, n, oy, ox, co);
+                    if (N->eager == 1) reevaluate(N, n, oy, ox, co);
                 }
             }
         }
@@ -152,13 +154,13 @@ static void deliver(evc_net* N, int n, int y, int x, int ch, double d)
         size_t i = ((size_t)oy * N->W[n] + ox) * N->C[n] + ch;
         N->touched[n][i] = 1;
         N->n_updates[n] += 1;
-        if (N->eager) reevaluate(N, n, oy, ox, ch);
+        if (N->eager == 1) reevaluate(N, n, oy, ox, ch);
     } else { /* global average over all positions of a channel */
         size_t i = (size_t)ch;
         N->c[n][i] += d / ((double)N->H[n - 1] * N->W[n - 1]);
         N->touched[n][i] = 1;
         N->n_updates[n] += 1;
-        if (N->eager) reevaluate(N, n, 0, 0, ch);
+        if (N->eager == 1) reevaluate(N, n, 0, 0, ch);
     }
 }
 
@@ -226,13 +228,27 @@ static void finalise_ready_rows(evc_net* N, int r_in, int flush, long long* live
  *   telescoping_err      max over all units of |sum of events - final activation|.
  * Returns 0, or -1 on bad arguments.
  */
-int evc_run(int mode, int eager, int n_layers, const evc_layer* layers,
-            const double* const* weights, const double* const* biases,
-            int H, int W, int C0, const double* input,
-            double* out, double* out_sum_dh,
-            long long* stats, long long* stats2,
-            long long* live_between, long long* live_peak, double* telescoping_err)
+/* every unit of layer n re-evaluates once (per-segment eager policy) */
+static void reevaluate_layer(evc_net* N, int n)
 {
+    for (int y = 0; y < N->H[n]; ++y)
+        for (int x = 0; x < N->W[n]; ++x)
+            for (int ch = 0; ch < N->C[n]; ++ch) reevaluate(N, n, y, x, ch);
+}
+
+/*
+ * As evc_run, but only the first n_feed rows of the H-row input are presented (the maps are sized for H rows:
+ * a stream that does not know yet where its input ends), and after every presented row the activation map of
+ * the last layer is copied to steps_out[r] (n_feed maps; may be NULL).  With n_feed == H this is evc_run.
+ */
+int evc_run_steps(int mode, int eager, int n_layers, const evc_layer* layers,
+                  const double* const* weights, const double* const* biases,
+                  int H, int W, int C0, const double* input, int n_feed, double* steps_out,
+                  double* out, double* out_sum_dh,
+                  long long* stats, long long* stats2,
+                  long long* live_between, long long* live_peak, double* telescoping_err)
+{
+    if (n_feed < 0 || n_feed > H) return -1;
     if (n_layers < 1 || n_layers > 62) return -1;
     evc_net N; memset(&N, 0, sizeof N);
     N.n_layers = n_layers; N.mode = mode; N.eager = eager; N.L = layers; N.w = weights; N.b = biases;
@@ -270,12 +286,9 @@ int evc_run(int mode, int eager, int n_layers, const evc_layer* layers,
             }
     }
     if (eager)   /* units whose f(b) is non-zero announce it before any input arrives */
-        for (int n = 1; n <= n_layers; ++n)
-            for (int y = 0; y < N.H[n]; ++y)
-                for (int x = 0; x < N.W[n]; ++x)
-                    for (int ch = 0; ch < N.C[n]; ++ch) reevaluate(&N, n, y, x, ch);
+        for (int n = 1; n <= n_layers; ++n) reevaluate_layer(&N, n);
 
-    for (int r = 0; r < H; ++r) {
+    for (int r = 0; r < n_feed; ++r) {
         /* present the components of this segment one by one; zero components send nothing */
         for (int x = 0; x < W; ++x)
             for (int ch = 0; ch < C0; ++ch) {
@@ -289,6 +302,12 @@ int evc_run(int mode, int eager, int n_layers, const evc_layer* layers,
                 }
             }
         if (!eager) finalise_ready_rows(&N, r, 0, live_peak);
+        if (eager == 2)   /* the segment is in: the layers re-evaluate one after the other */
+            for (int n = 1; n <= n_layers; ++n) reevaluate_layer(&N, n);
+        if (steps_out) {
+            size_t tot = (size_t)N.H[n_layers] * N.W[n_layers] * N.C[n_layers];
+            memcpy(steps_out + (size_t)r * tot, N.h[n_layers], tot * sizeof(double));
+        }
         /* units that hold state and that a later segment can still influence */
         for (int n = 1; n <= n_layers; ++n) {
             long long live = 0;
@@ -305,7 +324,7 @@ int evc_run(int mode, int eager, int n_layers, const evc_layer* layers,
             if (live > live_between[n]) live_between[n] = live;
         }
     }
-    if (!eager) finalise_ready_rows(&N, H - 1, 1, live_peak);
+    if (!eager && n_feed == H) finalise_ready_rows(&N, H - 1, 1, live_peak);
 
     double terr = 0.0;
     for (int n = 0; n <= n_layers; ++n) {
@@ -327,4 +346,15 @@ int evc_run(int mode, int eager, int n_layers, const evc_layer* layers,
         free(N.c[n]); free(N.h[n]); free(N.sum_dh[n]); free(N.touched[n]); free(N.done[n]);
     }
     return 0;
+}
+
+int evc_run(int mode, int eager, int n_layers, const evc_layer* layers,
+            const double* const* weights, const double* const* biases,
+            int H, int W, int C0, const double* input,
+            double* out, double* out_sum_dh,
+            long long* stats, long long* stats2,
+            long long* live_between, long long* live_peak, double* telescoping_err)
+{
+    return evc_run_steps(mode, eager, n_layers, layers, weights, biases, H, W, C0, input, H, NULL, out, out_sum_dh,
+                         stats, stats2, live_between, live_peak, telescoping_err);
 }

@@ -186,15 +186,21 @@ class _EvcLayer(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("kind", "cin", "cout", "kh", "kw", "stride", "pad", "relu", "shift")]
 
 
-def event_run(mode: str, layers, x: np.ndarray, weights, biases=None, eager: bool = True):
+def event_run(mode: str, layers, x: np.ndarray, weights, biases=None, eager=True, n_feed=None, steps: bool = False):
     """Run ONE stream (x: [H][W][C]) through the event-by-event checker (Eq. 2-5).
+
+    ``eager``: False/0 = a unit emits once when nothing can reach it any more; True/1 = the paper's rule, one input
+    component at a time; 2 = the paper's rule with a whole segment delivered before the layers re-evaluate.
+    ``n_feed``: present only the first n_feed rows (the maps stay sized for all H rows: a stream that does not know
+    where its input ends).  ``steps``: also return the last layer's map after every presented row.
 
     Returns a dict: out (final map of the last layer), sum_dh (sum of the last
     layer's emitted events per unit), events / updates (per layer, index 0 =
     input), live_between, live_peak (units holding reachable state, per layer),
-    telescoping_err.
+    telescoping_err, and steps ([n_feed][Hout][Wout][C]) if asked for.
     """
     H, W, C0 = x.shape
+    n_feed = H if n_feed is None else int(n_feed)
     n = len(layers)
     arr = (_EvcLayer * n)()
     kinds = {"conv": 0, "pool": 1, "avg": 2}
@@ -223,12 +229,17 @@ def event_run(mode: str, layers, x: np.ndarray, weights, biases=None, eager: boo
     lp = np.zeros(n + 1, dtype=np.int64)
     terr = ctypes.c_double(0)
     xd = np.ascontiguousarray(x, dtype=np.float64)
+    snap = np.zeros((n_feed, oh, ow, oc), dtype=np.float64) if steps else None
     modes = {"f32": 0, "bf16": 1, "i8": 2}
-    rc = lib().evc_run(modes[mode], int(bool(eager)), n, arr, wptr, bptr, H, W, C0, _p(xd, ctypes.c_double),
-                       _p(out, ctypes.c_double), _p(sdh, ctypes.c_double), _p(st, ctypes.c_longlong),
-                       _p(st2, ctypes.c_longlong), _p(lb, ctypes.c_longlong), _p(lp, ctypes.c_longlong),
-                       ctypes.byref(terr))
+    rc = lib().evc_run_steps(modes[mode], int(eager), n, arr, wptr, bptr, H, W, C0, _p(xd, ctypes.c_double),
+                             ctypes.c_int(n_feed), _p(snap, ctypes.c_double) if steps else None,
+                             _p(out, ctypes.c_double), _p(sdh, ctypes.c_double), _p(st, ctypes.c_longlong),
+                             _p(st2, ctypes.c_longlong), _p(lb, ctypes.c_longlong), _p(lp, ctypes.c_longlong),
+                             ctypes.byref(terr))
     if rc != 0:
         raise ValueError("event checker rejected the net")
-    return dict(out=out, sum_dh=sdh, events=st, updates=st2, live_between=lb, live_peak=lp,
-                telescoping_err=float(terr.value))
+    res = dict(out=out, sum_dh=sdh, events=st, updates=st2, live_between=lb, live_peak=lp,
+               telescoping_err=float(terr.value))
+    if steps:
+        res["steps"] = snap
+    return res

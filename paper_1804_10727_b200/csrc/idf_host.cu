@@ -62,6 +62,10 @@ struct LayerPlan {
     long long pending = 0;                 // rows waiting in this layer's input buffer
     int fire_rows = 0;                     // the layer runs once this many rows wait (or when a push ends)
     int fuse_pool = 0;                     // conv layer whose tensor-core launch may emit the following 2x2 max-pool's rows
+    // eager emission: rings of e_cap rows for the state, the announced activation and the change of the current step
+    int e_cap = 0, e_window = 0;           // ring capacity in rows; most rows one segment can touch (the input cone)
+    size_t e_c_off = 0, e_h_off = 0, e_d_off = 0;
+    long long e_hi = -1;                   // last row touched so far
 };
 
 enum Phase { CREATED = 0, OPEN = 1, FINISHED = 2 };
@@ -70,6 +74,8 @@ enum Phase { CREATED = 0, OPEN = 1, FINISHED = 2 };
 
 struct idf_net {
     int dtype = 0, in_w = 0, in_c = 0, n_streams = 0, row_block = 0;
+    int eager = 0;                         // emission policy: 0 = once per unit (deferred), 1 = after every segment (eager)
+    size_t eager_in_off = 0;               // the pushed segment as words (the input layer's announcement)
     std::vector<LayerPlan> L;
     size_t workspace_bytes = 0, state_region_off = 0, state_region_bytes = 0, counters_off = 0, status_off = 0;
     size_t ring_scratch_off = 0;           // room for a copy of the largest tensor-core layer's ring (row-chunked launches)
@@ -342,6 +348,8 @@ int launch_conv_pool(idf_net* net, size_t i, const void* in_ptr, long long n_in,
 // push of one segment still walks every layer it can reach before the call returns.
 int fire(idf_net* net, size_t i, const void* in_ptr, long long n_in, bool flush, void* d_out, long long out_cap,
          long long* emitted);
+int run_segments_eager(idf_net* net, const void* d_segments, long long n_seg, bool flush, void* d_out, long long out_cap,
+                       long long* emitted);
 
 int ensure_space(idf_net* net, size_t m, long long need, void* d_out, long long out_cap, long long* emitted)
 {
@@ -404,6 +412,7 @@ int run_segments(idf_net* net, const void* d_segments, long long n_seg, bool flu
                  long long out_cap, long long* emitted)
 {
     const size_t nl = net->L.size();
+    if (net->eager) return run_segments_eager(net, d_segments, n_seg, flush, d_out, out_cap, emitted);
     // capacity of the caller's output first: the rows complete after this call do not depend on the schedule
     {
         long long r = net->L[0].rows_in + n_seg;
@@ -429,6 +438,156 @@ int run_segments(idf_net* net, const void* d_segments, long long n_seg, bool flu
             rc = fire(net, i, i ? net->ws + net->L[i - 1].out_off : nullptr, i ? net->L[i].pending : 0, true, d_out, out_cap, emitted);
     if (rc != IDF_OK) net->phase = FINISHED;      // counters and buffers are no longer consistent: reopen to go on
     return rc;
+}
+
+}  // namespace
+
+namespace {
+
+// Rows of layer P reached by rows [lo, hi] of the layer below (its input cone, clipped at the top of the map).
+void reach(const LayerPlan& P, long long lo, long long hi, long long* o_lo, long long* o_hi)
+{
+    if (P.l.kind == IDF_CONV) {
+        const long long a = lo + P.l.pad - P.l.kh + 1;
+        *o_lo = a <= 0 ? 0 : (a + P.l.stride - 1) / P.l.stride;
+        *o_hi = (hi + P.l.pad) / P.l.stride;
+    } else {
+        *o_lo = lo / 2;
+        *o_hi = hi / 2;
+    }
+}
+
+// Eager emission, one segment at a time: the segment is the input layer's announcement; every layer in turn takes up
+// the changes of the rows below that moved, re-evaluates the rows of its cone and announces their changes.
+int eager_step(idf_net* net, const void* seg, long long r, void* d_out, long long out_cap)
+{
+    const long long S = net->n_streams;
+    const bool int_net = net->dtype == IDF_I8_I32;
+    unsigned long long* counters = (unsigned long long*)(net->ws + net->counters_off);
+    cudaError_t ce = launch_eager_input(seg, net->L[0].in_elem, net->ws + net->eager_in_off, S * net->in_w * net->in_c,
+                                        counters, net->stream);
+    if (ce != cudaSuccess) return fail(IDF_ERR_CUDA, "kernel launch failed (eager input): %s", cudaGetErrorString(ce));
+    net->launches += 1;
+    long long lo = r, hi = r;
+    for (size_t i = 0; i < net->L.size(); ++i) {
+        LayerPlan& P = net->L[i];
+        const bool last = i + 1 == net->L.size();
+        long long o_lo, o_hi;
+        reach(P, lo, hi, &o_lo, &o_hi);
+        EagerArgs a{};
+        a.din = i == 0 ? net->ws + net->eager_in_off : net->ws + net->L[i - 1].e_d_off;
+        a.hin = i == 0 ? nullptr : net->ws + net->L[i - 1].e_h_off;
+        a.c = net->ws + P.e_c_off; a.h = net->ws + P.e_h_off; a.d = net->ws + P.e_d_off;
+        a.w = net->ws + P.w_off;
+        a.bias = P.b_packed.empty() ? nullptr : net->ws + P.b_off;
+        a.out = last ? d_out : nullptr;
+        a.out_row_stride = (long long)P.out_w * P.out_c;
+        a.out_stream_stride = out_cap * a.out_row_stride;
+        a.events = last ? nullptr : counters + i + 1;
+        a.S = (int)S; a.Win = P.in_w; a.Wout = P.out_w; a.Cin = P.in_c; a.Cout = P.out_c;
+        a.Kh = P.l.kh; a.Kw = P.l.kw; a.stride = P.l.stride; a.pad = P.l.pad;
+        a.stride_x = P.in_w == 1 ? 1 : P.l.stride; a.pad_x = P.in_w == 1 ? 0 : P.l.pad;
+        a.relu = P.l.relu; a.shift = P.l.shift; a.round_bf16 = P.out_elem == E_BF16;
+        a.cap_in = i == 0 ? 1 : net->L[i - 1].e_cap; a.cap = P.e_cap;
+        a.in_lo = lo; a.in_hi = P.l.kind == IDF_MAXPOOL2 ? net->L[i - 1].e_hi : hi;
+        a.o_lo = o_lo; a.o_hi = o_hi; a.o_new = P.e_hi + 1; a.o_cut = (1LL << 62);
+        if (o_hi - o_lo + 1 > P.e_window) return fail(IDF_ERR_CAPACITY, "internal: layer %zu cone of %lld rows exceeds %d", i, o_hi - o_lo + 1, P.e_window);
+        ce = launch_eager_layer(a, P.l.kind == IDF_MAXPOOL2, int_net, net->stream);
+        if (ce != cudaSuccess) return fail(IDF_ERR_CUDA, "kernel launch failed at layer %zu: %s", i, cudaGetErrorString(ce));
+        net->launches += 1;
+        if (o_hi > P.e_hi) P.e_hi = o_hi;
+        lo = o_lo; hi = o_hi;
+    }
+    return IDF_OK;
+}
+
+// Rows of the last layer that no later segment can reach once `rows` segments have arrived.
+long long eager_final_rows(const idf_net* net, long long rows)
+{
+    long long lo = rows, hi = rows;
+    for (const auto& P : net->L) reach(P, lo, hi, &lo, &hi);
+    return lo;
+}
+
+// End of input: units of rows that turn out to lie beyond the maps (their receptive field was cut off by the end of
+// the input, or they only existed as a first half of a pooling pair) take back what they announced, layer by layer.
+int eager_finish(idf_net* net, void* d_out, long long out_cap)
+{
+    const long long S = net->n_streams;
+    const bool int_net = net->dtype == IDF_I8_I32;
+    unsigned long long* counters = (unsigned long long*)(net->ws + net->counters_off);
+    long long h = net->L[0].rows_in;
+    bool changed = false;
+    long long lo = 0, hi = -1;
+    for (size_t i = 0; i < net->L.size(); ++i) {
+        LayerPlan& P = net->L[i];
+        const bool last = i + 1 == net->L.size();
+        h = layer_rows_at_flush(P, h);                       // rows this layer's map really has
+        long long p_lo = (1LL << 62), p_hi = -1;
+        if (changed) reach(P, lo, hi, &p_lo, &p_hi);
+        if (p_hi > P.e_hi) p_hi = P.e_hi;
+        if (P.e_hi >= h) { p_lo = std::min(p_lo, h); p_hi = P.e_hi; }
+        if (p_hi < p_lo) { changed = false; continue; }
+        EagerArgs a{};
+        a.din = i == 0 ? net->ws + net->eager_in_off : net->ws + net->L[i - 1].e_d_off;
+        a.hin = i == 0 ? nullptr : net->ws + net->L[i - 1].e_h_off;
+        a.c = net->ws + P.e_c_off; a.h = net->ws + P.e_h_off; a.d = net->ws + P.e_d_off;
+        a.w = net->ws + P.w_off;
+        a.bias = P.b_packed.empty() ? nullptr : net->ws + P.b_off;
+        a.out = last ? d_out : nullptr;
+        a.out_row_stride = (long long)P.out_w * P.out_c;
+        a.out_stream_stride = out_cap * a.out_row_stride;
+        a.events = last ? nullptr : counters + i + 1;
+        a.S = (int)S; a.Win = P.in_w; a.Wout = P.out_w; a.Cin = P.in_c; a.Cout = P.out_c;
+        a.Kh = P.l.kh; a.Kw = P.l.kw; a.stride = P.l.stride; a.pad = P.l.pad;
+        a.stride_x = P.in_w == 1 ? 1 : P.l.stride; a.pad_x = P.in_w == 1 ? 0 : P.l.pad;
+        a.relu = P.l.relu; a.shift = P.l.shift; a.round_bf16 = P.out_elem == E_BF16;
+        a.cap_in = i == 0 ? 1 : net->L[i - 1].e_cap; a.cap = P.e_cap;
+        a.in_lo = changed ? lo : 1; a.in_hi = changed ? hi : 0;
+        if (P.l.kind == IDF_MAXPOOL2) a.in_hi = net->L[i - 1].e_hi;
+        a.o_lo = p_lo; a.o_hi = p_hi; a.o_new = P.e_hi + 1; a.o_cut = h;
+        // (rows beyond the caller's buffer are not written: they hold nothing the caller will read)
+        if (last && a.o_hi >= out_cap) a.o_hi = out_cap - 1;
+        cudaError_t ce = launch_eager_layer(a, P.l.kind == IDF_MAXPOOL2, int_net, net->stream);
+        if (ce != cudaSuccess) return fail(IDF_ERR_CUDA, "kernel launch failed at layer %zu: %s", i, cudaGetErrorString(ce));
+        net->launches += 1;
+        changed = true; lo = p_lo; hi = p_hi;
+    }
+    return IDF_OK;
+}
+
+int run_segments_eager(idf_net* net, const void* d_segments, long long n_seg, bool flush, void* d_out, long long out_cap,
+                       long long* emitted)
+{
+    const size_t seg_bytes = (size_t)net->n_streams * net->in_w * net->in_c * elem_size(net->L[0].in_elem);
+    const long long r0 = net->L[0].rows_in;
+    // every row the pushed segments touch in the last layer is written (finished rows and, above them, the rows of
+    // the cone with their current partial activations): all of them must fit the caller's buffer
+    if (n_seg > 0) {
+        long long lo = r0 + n_seg - 1, hi = lo;
+        for (const auto& P : net->L) reach(P, lo, hi, &lo, &hi);
+        if (hi + 1 > out_cap)
+            return fail(IDF_ERR_CAPACITY, "eager emission writes output rows up to %lld: out_capacity_rows=%lld is too small", hi, out_cap);
+    }
+    int rc = IDF_OK;
+    for (long long k = 0; k < n_seg && rc == IDF_OK; ++k) {
+        rc = eager_step(net, (const unsigned char*)d_segments + (size_t)k * seg_bytes, r0 + k, d_out, out_cap);
+        if (rc == IDF_OK) net->L[0].rows_in = r0 + k + 1;
+    }
+    long long done = eager_final_rows(net, net->L[0].rows_in);
+    if (rc == IDF_OK && flush) {
+        rc = eager_finish(net, d_out, out_cap);
+        long long h = net->L[0].rows_in;
+        for (const auto& P : net->L) h = layer_rows_at_flush(P, h);
+        done = h;
+        if (rc == IDF_OK && done > out_cap) rc = fail(IDF_ERR_CAPACITY, "output row %lld does not fit out_capacity_rows=%lld", done - 1, out_cap);
+    }
+    if (rc != IDF_OK) { net->phase = FINISHED; return rc; }
+    LayerPlan& Z = net->L.back();
+    if (done < Z.rows_done) done = Z.rows_done;
+    *emitted += done - Z.rows_done;
+    Z.rows_done = done;
+    return IDF_OK;
 }
 
 }  // namespace
@@ -463,10 +622,17 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
     if (spec->in_w < 1 || spec->in_c < 1) return fail(IDF_ERR_SPEC, "in_w and in_c must be positive");
     if (spec->n_streams < 1) return fail(IDF_ERR_SPEC, "n_streams must be positive");
     if (spec->row_block < 0 || spec->row_block > 4096) return fail(IDF_ERR_SPEC, "row_block must be 0..4096");
+    if (spec->emission != IDF_EMIT_DEFERRED && spec->emission != IDF_EMIT_EAGER) return fail(IDF_ERR_SPEC, "unknown emission policy %d", spec->emission);
+    if (spec->emission == IDF_EMIT_EAGER) {
+        if (spec->layers[0].kind != IDF_CONV) return fail(IDF_ERR_UNSUPPORTED, "eager emission: the first layer must be a conv layer");
+        for (int i = 0; i < spec->n_layers; ++i)
+            if (spec->layers[i].kind == IDF_GLOBAL_AVG) return fail(IDF_ERR_UNSUPPORTED, "eager emission: no global-average sink (use a whole-map conv layer as the output unit)");
+    }
 
     idf_net* net = new (std::nothrow) idf_net();
     if (!net) return fail(IDF_ERR_ARG, "out of host memory");
     net->dtype = spec->dtype; net->in_w = spec->in_w; net->in_c = spec->in_c; net->n_streams = spec->n_streams;
+    net->eager = spec->emission == IDF_EMIT_EAGER;
     // default: about 25 000 positions per stream and block (112 rows of a 224-wide image, 1024 samples of a 1D
     // signal): long enough that a launch's fixed cost (weights into shared memory, ring rows in and out) is small
     net->row_block = spec->row_block > 0 ? spec->row_block : std::min(1024, std::max(32, 25088 / spec->in_w));
@@ -533,7 +699,7 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
             }
             // tensor-core layout [tap][Cout][Cin], activation type, when the layer qualifies
             const int in_cap = i == 0 ? net->row_block : net->L[i - 1].out_cap_rows;
-            const bool tc_allowed = !P.use_sparse && !(debug_flags() & IDF_DEBUG_NO_TENSOR_CORES) && spec->dtype != IDF_F32;
+            const bool tc_allowed = !P.use_sparse && !(debug_flags() & IDF_DEBUG_NO_TENSOR_CORES) && spec->dtype != IDF_F32 && !net->eager;
             const size_t es = spec->dtype == IDF_I8_I32 ? 1 : 2;
             const int taps = l.kh * l.kw;
             const bool pool_next = i + 1 < spec->n_layers && spec->layers[i + 1].kind == IDF_MAXPOOL2;
@@ -605,13 +771,31 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
         net->state_bytes_stream += P.state_bytes_stream;
         w = P.out_w; c = P.out_c; elem = P.out_elem;
     }
+    if (net->eager) {
+        // rows of every layer that one segment can touch (its input cone): the most over a long run of segments
+        for (long long r = 0; r < 4096; ++r) {
+            long long lo = r, hi = r;
+            for (auto& P : net->L) {
+                reach(P, lo, hi, &lo, &hi);
+                P.e_window = std::max<long long>(P.e_window, hi - lo + 1);
+            }
+        }
+        net->state_bytes_stream = 0;
+        for (auto& P : net->L) {
+            P.e_cap = P.e_window + 2;      // (a pooling layer above still reads the two rows below its oldest open pair)
+            P.out_cap_rows = 0;
+            P.state_bytes_stream = (size_t)P.e_window * P.out_w * P.out_c * 8;       // state and announced activation
+            P.state_bytes_all = (size_t)3 * P.e_cap * net->n_streams * P.out_w * P.out_c * 4;
+            net->state_bytes_stream += P.state_bytes_stream;
+        }
+    }
     // a dense tensor-core conv layer directly followed by a 2x2 max-pool emits the pooled rows itself
     {
         const bool no_fuse = (debug_flags() & IDF_DEBUG_NO_POOL_FUSION) != 0;
         for (size_t i = 0; i + 1 < net->L.size(); ++i) {
             LayerPlan& P = net->L[i];
             P.fuse_pool = P.l.kind == IDF_CONV && net->L[i + 1].l.kind == IDF_MAXPOOL2 && P.tc.ok && P.tc_pool.ok && !P.use_sparse &&
-                          P.out_w >= 2 && (P.tc_pool.BX % 2) == 0 && !no_fuse;
+                          P.out_w >= 2 && (P.tc_pool.BX % 2) == 0 && !no_fuse && !net->eager;
         }
     }
     // workspace: [parameters][state of all streams][rows travelling between layers][counters]
@@ -622,8 +806,16 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
         P.wtc_off = off; off = align_up(off + P.wtc_packed.size(), 1024);
     }
     net->state_region_off = off;
-    for (auto& P : net->L) { P.state_off = off; off = align_up(off + P.state_bytes_all); }
+    for (auto& P : net->L) {
+        P.state_off = off;
+        if (net->eager) {
+            const size_t ring = P.state_bytes_all / 3;
+            P.e_c_off = off; P.e_h_off = off + ring; P.e_d_off = off + 2 * ring;
+        }
+        off = align_up(off + P.state_bytes_all);
+    }
     net->state_region_bytes = off - net->state_region_off;
+    if (net->eager) { net->eager_in_off = off; off = align_up(off + (size_t)net->n_streams * net->in_w * net->in_c * 4); }
     for (size_t i = 0; i + 1 < net->L.size(); ++i) {
         LayerPlan& P = net->L[i];
         P.out_off = off;
@@ -678,6 +870,19 @@ int idf_out_shape(const idf_net* net, long long in_rows, long long* out_rows, in
     return IDF_OK;
 }
 
+long long idf_out_rows_needed(const idf_net* net, long long in_rows)
+{
+    if (!net || in_rows < 0) return -1;
+    long long h = in_rows;
+    for (const auto& P : net->L) h = layer_rows_at_flush(P, h);
+    if (net->eager && in_rows > 0) {
+        long long lo = in_rows - 1, hi = lo;
+        for (const auto& P : net->L) reach(P, lo, hi, &lo, &hi);
+        h = std::max(h, hi + 1);
+    }
+    return h;
+}
+
 int idf_stream_open(idf_net* net, void* d_workspace, size_t workspace_bytes, void* cuda_stream)
 {
     if (!net || !d_workspace) return fail(IDF_ERR_ARG, "net and d_workspace must not be NULL");
@@ -711,7 +916,7 @@ int idf_stream_reset(idf_net* net)
 {
     if (!net) return fail(IDF_ERR_ARG, "net must not be NULL");
     if (net->phase == CREATED) return fail(IDF_ERR_STATE, "reset before stream_open");
-    for (auto& P : net->L) { P.rows_in = 0; P.rows_done = 0; P.tc_launches = 0; P.pending = 0; }
+    for (auto& P : net->L) { P.rows_in = 0; P.rows_done = 0; P.tc_launches = 0; P.pending = 0; P.e_hi = -1; }
     cudaError_t e = cudaMemsetAsync(net->ws + net->status_off, 0, sizeof(unsigned int), net->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(net->ws + net->state_region_off, 0, net->state_region_bytes, net->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(net->ws + net->counters_off, 0, net->L.size() * sizeof(unsigned long long), net->stream);
@@ -744,6 +949,7 @@ int idf_stream_set_out_base(idf_net* net, long long first_row)
 {
     if (!net) return fail(IDF_ERR_ARG, "net must not be NULL");
     if (net->phase != OPEN) return fail(IDF_ERR_STATE, "set_out_base needs open streams");
+    if (net->eager && first_row != 0) return fail(IDF_ERR_UNSUPPORTED, "eager emission keeps the output window at row 0");
     if (first_row < 0 || first_row > net->out_rows_total)
         return fail(IDF_ERR_ARG, "first_row=%lld: only rows emitted so far (%lld) can be left behind", first_row, net->out_rows_total);
     net->out_base = first_row;
@@ -918,6 +1124,7 @@ size_t idf_state_snapshot_bytes(const idf_net* net) { return net ? snapshot_byte
 int idf_state_save(idf_net* net, void* h_snapshot, size_t bytes)
 {
     if (!net || !h_snapshot) return fail(IDF_ERR_ARG, "net and h_snapshot must not be NULL");
+    if (net->eager) return fail(IDF_ERR_UNSUPPORTED, "state snapshots are not available with eager emission");
     if (net->phase != OPEN) return fail(IDF_ERR_STATE, "state_save needs open streams (after open/reset/push, before finish)");
     if (bytes < snapshot_bytes(net)) return fail(IDF_ERR_CAPACITY, "snapshot needs %zu bytes, %zu given", snapshot_bytes(net), bytes);
     for (const auto& P : net->L)
@@ -943,6 +1150,7 @@ int idf_state_save(idf_net* net, void* h_snapshot, size_t bytes)
 int idf_state_restore(idf_net* net, const void* h_snapshot, size_t bytes)
 {
     if (!net || !h_snapshot) return fail(IDF_ERR_ARG, "net and h_snapshot must not be NULL");
+    if (net->eager) return fail(IDF_ERR_UNSUPPORTED, "state snapshots are not available with eager emission");
     if (net->phase == CREATED) return fail(IDF_ERR_STATE, "state_restore before stream_open");
     if (bytes < sizeof(SnapshotHeader)) return fail(IDF_ERR_ARG, "not a snapshot (too short)");
     SnapshotHeader h;

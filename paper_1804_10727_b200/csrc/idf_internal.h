@@ -66,6 +66,30 @@ struct AvgArgs {
     long long rows_total;  // rows received since open, these included
 };
 
+// Eager emission (one segment per step): how one layer re-evaluates the rows of its input cone.
+// Rings hold 32-bit words (fp32 for float nets, int32 for int nets), slot = row mod capacity.
+struct EagerArgs {
+    const void* din;       // changes announced by the layer below in this step: [cap_in][S][Win][Cin] (conv)
+    const void* hin;       // activations announced so far by the layer below: [cap_in][S][Win][Cin] (pool)
+    void* c;               // state variables: [cap][S][Wout][Cout] (conv)
+    void* h;               // activations this layer has announced: [cap][S][Wout][Cout]
+    void* d;               // the change it announces in this step: [cap][S][Wout][Cout]
+    const void* w;         // [Kh][Kw][Cin][Cout] fp32 or int8
+    const void* bias;      // [Cout] words or nullptr
+    void* out;             // last layer: the caller's output [S][rows][Wout][Cout] (fp32 / int8), else nullptr
+    long long out_row_stride, out_stream_stride;
+    unsigned long long* events;   // count of non-zero changes announced (or nullptr)
+    int S, Win, Wout, Cin, Cout, Kh, Kw, stride, pad, stride_x, pad_x, relu, shift, round_bf16;
+    int cap_in, cap;       // ring capacities in rows
+    long long in_lo, in_hi;   // rows of the layer below that changed in this step (conv; empty if in_lo > in_hi);
+                              // pool: in_hi = last row of the layer below that has announced anything
+    long long o_lo, o_hi;     // rows of this layer to re-evaluate
+    long long o_new;          // rows >= o_new are touched for the first time (their slots hold an older row)
+    long long o_cut;          // rows >= o_cut turn out not to exist (end of input): their activation goes back to 0
+};
+cudaError_t launch_eager_input(const void* in, int in_elem, void* d, long long n, unsigned long long* events, cudaStream_t st);
+cudaError_t launch_eager_layer(const EagerArgs& a, int is_pool, int int_net, cudaStream_t st);
+
 // Static plan of the tensor-core path for one conv layer (tile shapes, shared-memory budget).
 struct TcPlan {
     int ok = 0;

@@ -28,7 +28,7 @@ EXPORTS = (
     "idf_net_create", "idf_net_destroy", "idf_net_state_bytes", "idf_net_workspace_bytes", "idf_out_shape",
     "idf_stream_open", "idf_stream_reset", "idf_stream_push", "idf_stream_push_last", "idf_stream_finish", "idf_run_host", "idf_event_counts",
     "idf_launch_count", "idf_stream_status", "idf_set_timing", "idf_layer_times", "idf_conv_rows_noalloc", "idf_last_error",
-    "idf_state_snapshot_bytes", "idf_state_save", "idf_state_restore", "idf_stream_set_out_base", "idf_set_debug_flags",
+    "idf_state_snapshot_bytes", "idf_state_save", "idf_state_restore", "idf_stream_set_out_base", "idf_set_debug_flags", "idf_out_rows_needed",
 )
 DEBUG_NO_TENSOR_CORES, DEBUG_NO_POOL_FUSION, DEBUG_NO_ROW_CHUNKS, DEBUG_NO_PDL = 1, 2, 4, 8
 
@@ -41,7 +41,7 @@ class IdfLayer(ctypes.Structure):
 class IdfSpec(ctypes.Structure):
     _fields_ = [("n_layers", ctypes.c_int), ("layers", ctypes.POINTER(IdfLayer)), ("dtype", ctypes.c_int),
                 ("in_w", ctypes.c_int), ("in_c", ctypes.c_int), ("n_streams", ctypes.c_int),
-                ("row_block", ctypes.c_int)]
+                ("row_block", ctypes.c_int), ("emission", ctypes.c_int)]
 
 
 class IdfError(RuntimeError):
@@ -83,6 +83,7 @@ def lib():
         L.idf_state_save.argtypes = [vp, vp, sz]
         L.idf_state_restore.argtypes = [vp, vp, sz]
         L.idf_set_debug_flags.argtypes = [ctypes.c_uint]
+        L.idf_out_rows_needed.argtypes = [vp, ll]; L.idf_out_rows_needed.restype = ll
         L.idf_last_error.restype = ctypes.c_char_p
         _lib = L
     return _lib
@@ -122,12 +123,12 @@ class Net:
 
     def __init__(self, dtype, layers: Sequence, in_w: int, in_c: int, n_streams: int,
                  weights: Sequence[Optional[np.ndarray]], biases: Optional[Sequence[Optional[np.ndarray]]] = None,
-                 row_block: int = 0):
+                 row_block: int = 0, eager: bool = False):
         self.dtype = DTYPES[dtype] if isinstance(dtype, str) else int(dtype)
         self.n_streams, self.in_w, self.in_c = int(n_streams), int(in_w), int(in_c)
         n = len(layers)
         self._layers = (IdfLayer * n)(*[_layer_struct(l) for l in layers])
-        spec = IdfSpec(n, self._layers, self.dtype, in_w, in_c, n_streams, row_block)
+        spec = IdfSpec(n, self._layers, self.dtype, in_w, in_c, n_streams, row_block, 1 if eager else 0)
         keep = []
         wptr = (ctypes.c_void_p * n)()
         bptr = (ctypes.c_void_p * n)()
@@ -212,7 +213,8 @@ class Net:
         _check(lib().idf_stream_reset(self._h))
 
     def alloc_out(self, in_rows: int, device="cuda:0") -> torch.Tensor:
-        r, w, c = self.out_shape(in_rows)
+        _, w, c = self.out_shape(in_rows)
+        r = int(lib().idf_out_rows_needed(self._h, in_rows))
         return torch.zeros((self.n_streams, max(r, 1), w, c), dtype=self.out_torch_dtype, device=device)
 
     def push(self, segments: torch.Tensor, out: torch.Tensor) -> int:

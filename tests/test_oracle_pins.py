@@ -353,3 +353,52 @@ def test_output_sinks_reduce_to_matrix_product_and_mean(orc, mode):
             vals = pre[s, :, :, c].reshape(-1)
             exact = sum(Fraction(float(v)) for v in vals) / len(vals)
             assert abs(Fraction(float(avg[s, 0, 0, c])) - exact) <= abs(exact) * Fraction(1, 10 ** 12)
+
+
+# ---- the per-segment form of the paper's eager rule (what the device's eager mode computes) --------------------
+@pytest.mark.parametrize("mode", ["f32", "i8"])
+@pytest.mark.parametrize("name", ["valid3", "same_pool", "stride2", "stride2_pad", "k5", "oned_k9", "oned_pad", "k3s3"])
+def test_per_segment_eager_equals_component_eager_after_every_segment(orc, name, mode):
+    """Delivering a whole segment before the layers re-evaluate changes when events are sent, not what the units
+    hold once the segment has been absorbed (Eq. 3-5 telescope): after every segment the last layer's map equals
+    that of the one-component-at-a-time rule, the final map equals Eq. 1, no more events are sent than one at a time,
+    the input events are the same, and a stream that has seen only its first rows shows, in the rows nothing can reach
+    any more, exactly the rows of the conventional result."""
+    from helpers import SMALL_NETS, small_dims, with_shifts
+    layers = SMALL_NETS[name]
+    if mode == "i8":
+        layers = with_shifts(layers, 6)
+    H, W = small_dims(name)
+    H = min(H, 25)
+    C0 = next(l.cin for l in layers if l.kind == "conv")
+    x, ws, _ = _rand_net(mode, layers, H, W, C0, S=1, bias=False, seed=31)
+    want = orc.forward(mode, layers, x, ws, None)[0]
+    one = orc.event_run(mode, layers, x[0], ws, None, eager=1, steps=True)
+    seg = orc.event_run(mode, layers, x[0], ws, None, eager=2, steps=True)
+    tol = 0 if mode == "i8" else 1e-9
+    assert np.abs(seg["out"] - want).max() <= tol and np.abs(one["out"] - want).max() <= tol
+    assert np.abs(seg["steps"] - one["steps"]).max() <= tol
+    assert seg["telescoping_err"] <= tol
+    assert seg["events"][0] == one["events"][0] == int((x != 0).sum())
+    assert all(a <= b for a, b in zip(seg["events"], one["events"]))
+    # presenting only the first rows gives the same snapshots as the full run (causality) ...
+    part = orc.event_run(mode, layers, x[0], ws, None, eager=2, n_feed=H // 2, steps=True)
+    assert np.array_equal(part["steps"], seg["steps"][:H // 2])
+    # ... and rows that are final after r segments already hold the conventional values
+    for r in range(H):
+        rows = r + 1
+        for l in layers:
+            if l.kind == "conv":
+                q = rows + l.pad - l.kh
+                rows = 0 if q < 0 else q // l.stride + 1
+            else:
+                rows //= 2
+        rows = min(rows, want.shape[0])
+        assert np.abs(seg["steps"][r][:rows] - want[:rows]).max(initial=0) <= tol
+
+
+def test_per_segment_eager_zero_input_sends_nothing(orc):
+    layers = (conv(2, 3, 3, pad=1), POOL, conv(3, 2, 3))
+    x, ws, _ = _rand_net("f32", layers, 12, 10, 2, S=1, bias=False, seed=2)
+    res = orc.event_run("f32", layers, np.zeros_like(x[0]), ws, None, eager=2, steps=True)
+    assert not res["events"].any() and not res["steps"].any()
