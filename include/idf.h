@@ -96,7 +96,10 @@ typedef enum {
     IDF_ERR_CAPACITY = -4,     /* workspace or output buffer too small                                */
     IDF_ERR_UNSUPPORTED = -5,  /* valid request this build cannot serve                               */
     IDF_ERR_CUDA = -6,         /* a CUDA call failed                                                  */
-    IDF_ERR_TIMEOUT = -7       /* a bounded device-side wait ran out                                  */
+    IDF_ERR_TIMEOUT = -7,      /* a bounded device-side wait ran out                                  */
+    IDF_ERR_BOUNDS = -8        /* range-checked build only (libidf_bounds.so): an index lay outside   */
+                               /* the ring, row buffer, shared or tensor memory it addresses; the     */
+                               /* access was skipped and recorded, never performed                    */
 } idf_status;
 
 typedef struct {
@@ -240,7 +243,10 @@ int idf_event_counts(idf_net* net, long long* events);
 long long idf_launch_count(const idf_net* net);
 
 /* Wait for the stream and report whether any kernel of this handle gave up on a bounded device-side
- * wait since idf_stream_open (IDF_ERR_TIMEOUT; results are then invalid).  tensor_core_launches
+ * wait since idf_stream_open (IDF_ERR_TIMEOUT; results are then invalid) or, in the range-checked build
+ * of the library (compiled with -DIDF_BOUNDS: every index into a ring, row buffer, shared or tensor
+ * memory is compared with its extent before the access), skipped an access whose index was out of range
+ * (IDF_ERR_BOUNDS).  tensor_core_launches
  * (host, n_layers entries, may be NULL) receives per layer how many launches took the tcgen05 path. */
 int idf_stream_status(idf_net* net, long long* tensor_core_launches);
 

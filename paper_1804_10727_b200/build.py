@@ -13,6 +13,7 @@ from pathlib import Path
 HERE = Path(__file__).resolve().parent
 CSRC = HERE / "csrc"
 LIB = HERE / "libidf.so"
+BOUNDS_LIB = HERE / "libidf_bounds.so"      # the same sources with every index range-checked (-DIDF_BOUNDS)
 INCLUDE = HERE.parent / "include"
 
 NVCC_FLAGS = [
@@ -26,9 +27,9 @@ def sources():
 
 
 def _stale() -> bool:
-    if not LIB.exists():
+    if not LIB.exists() or not BOUNDS_LIB.exists():
         return True
-    t = LIB.stat().st_mtime
+    t = min(LIB.stat().st_mtime, BOUNDS_LIB.stat().st_mtime)
     deps = list(CSRC.glob("*")) + list(INCLUDE.glob("*.h"))
     return any(p.stat().st_mtime > t for p in deps)
 
@@ -37,15 +38,16 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    objs = []
+    objs = {LIB: [], BOUNDS_LIB: []}
     procs = []
-    for src in sources():
-        obj = src.with_suffix(".o")
-        cmd = [nvcc, *NVCC_FLAGS, "-I", str(INCLUDE), "-c", str(src), "-o", str(obj)]
-        if verbose:
-            cmd.insert(1, "-Xptxas=-v")
-        procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
-        objs.append(obj)
+    for lib, extra, suffix in ((LIB, [], ".o"), (BOUNDS_LIB, ["-DIDF_BOUNDS"], ".bounds.o")):
+        for src in sources():
+            obj = src.with_suffix(suffix)
+            cmd = [nvcc, *NVCC_FLAGS, *extra, "-I", str(INCLUDE), "-c", str(src), "-o", str(obj)]
+            if verbose:
+                cmd.insert(1, "-Xptxas=-v")
+            procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
+            objs[lib].append(obj)
     failed = False
     for src, p in procs:
         out, _ = p.communicate()
@@ -54,9 +56,10 @@ def build(force: bool = False, verbose: bool = False) -> Path:
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
-    subprocess.run([nvcc, "-shared", "-o", str(tmp), *map(str, objs)], check=True)
-    os.replace(tmp, LIB)
+    for lib, lib_objs in objs.items():
+        tmp = lib.with_suffix(f".tmp{os.getpid()}.so")
+        subprocess.run([nvcc, "-shared", "-o", str(tmp), *map(str, lib_objs)], check=True)
+        os.replace(tmp, lib)
     return LIB
 
 

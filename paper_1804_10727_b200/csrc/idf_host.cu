@@ -179,6 +179,10 @@ int launch_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, boo
         row_stride = S * stream_stride;
         row_base = o_begin - out_slot;             // emitted rows are appended slot after slot
     }
+    // extents of the buffers this launch addresses (the range-checked build compares every index with them)
+    const long long in_elems = n_in * S * P.in_w * P.in_c;
+    const long long out_elems = last ? S * out_cap * P.out_w * P.out_c : (long long)P.out_cap_rows * S * P.out_w * P.out_c;
+    unsigned int* status = (unsigned int*)(net->ws + net->status_off);
     cudaError_t ce;
     cudaEvent_t ev_a = nullptr, ev_b = nullptr;
     if (net->timing) {
@@ -190,6 +194,8 @@ int launch_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, boo
     }
     if (P.l.kind == IDF_CONV) {
         ConvArgs a{};
+        a.in_elems = in_elems; a.out_elems = out_elems; a.status = status;
+        a.ring_elems = (long long)P.ring_rows * S * P.out_w * P.out_c;
         a.in = in_ptr;
         a.w = net->ws + P.w_off;
         a.bias = P.b_packed.empty() ? nullptr : net->ws + P.b_off;
@@ -224,6 +230,7 @@ int launch_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, boo
             ce = P.use_sparse ? launch_conv_sparse(a, net->dtype, net->stream) : launch_conv_simple(a, net->dtype, net->stream);
     } else if (P.l.kind == IDF_GLOBAL_AVG) {
         AvgArgs a{};
+        a.in_elems = in_elems; a.out_elems = out_elems; a.sum_elems = S * P.in_c; a.status = status;
         a.in = in_ptr;
         a.sum = net->ws + P.state_off;
         a.out = (float*)out_ptr;
@@ -233,6 +240,7 @@ int launch_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, boo
         ce = launch_avg(a, net->stream);
     } else {
         PoolArgs a{};
+        a.in_elems = in_elems; a.out_elems = out_elems; a.state_elems = S * P.out_w * P.out_c; a.status = status;
         a.in = in_ptr;
         a.state = net->ws + P.state_off;
         a.out = out_ptr;
@@ -302,6 +310,11 @@ int launch_conv_pool(idf_net* net, size_t i, const void* in_ptr, long long n_in,
     a.ring_rows = P.ring_rows; a.in_elem = P.in_elem; a.out_elem = P.out_elem;
     a.r0 = r0; a.r1 = r1; a.o_begin = o_begin; a.o_end = o_end; a.done_end = done_end;
     a.pool_fused = 1; a.pool_keep = flush ? 0 : 1; a.pool_state = net->ws + Q.state_off;
+    a.in_elems = n_in * S * P.in_w * P.in_c;
+    a.out_elems = last ? S * out_cap * Q.out_w * Q.out_c : (long long)Q.out_cap_rows * S * Q.out_w * Q.out_c;
+    a.ring_elems = (long long)P.ring_rows * S * P.out_w * P.out_c;
+    a.pool_state_elems = S * Q.out_w * Q.out_c;
+    a.status = (unsigned int*)(net->ws + net->status_off);
     if (a.out_rows_extent < 1) return 1;
     cudaEvent_t ev_a = nullptr, ev_b = nullptr;
     if (net->timing) {
@@ -491,6 +504,10 @@ int eager_step(idf_net* net, const void* seg, long long r, void* d_out, long lon
         a.cap_in = i == 0 ? 1 : net->L[i - 1].e_cap; a.cap = P.e_cap;
         a.in_lo = lo; a.in_hi = P.l.kind == IDF_MAXPOOL2 ? net->L[i - 1].e_hi : hi;
         a.o_lo = o_lo; a.o_hi = o_hi; a.o_new = P.e_hi + 1; a.o_cut = (1LL << 62);
+        a.in_elems = i == 0 ? S * net->in_w * net->in_c : (long long)net->L[i - 1].e_cap * S * P.in_w * P.in_c;
+        a.ring_elems = (long long)P.e_cap * S * P.out_w * P.out_c;
+        a.out_elems = S * out_cap * P.out_w * P.out_c;
+        a.status = (unsigned int*)(net->ws + net->status_off);
         if (o_hi - o_lo + 1 > P.e_window) return fail(IDF_ERR_CAPACITY, "internal: layer %zu cone of %lld rows exceeds %d", i, o_hi - o_lo + 1, P.e_window);
         ce = launch_eager_layer(a, P.l.kind == IDF_MAXPOOL2, int_net, net->stream);
         if (ce != cudaSuccess) return fail(IDF_ERR_CUDA, "kernel launch failed at layer %zu: %s", i, cudaGetErrorString(ce));
@@ -546,6 +563,10 @@ int eager_finish(idf_net* net, void* d_out, long long out_cap)
         a.in_lo = changed ? lo : 1; a.in_hi = changed ? hi : 0;
         if (P.l.kind == IDF_MAXPOOL2) a.in_hi = net->L[i - 1].e_hi;
         a.o_lo = p_lo; a.o_hi = p_hi; a.o_new = P.e_hi + 1; a.o_cut = h;
+        a.in_elems = i == 0 ? S * net->in_w * net->in_c : (long long)net->L[i - 1].e_cap * S * P.in_w * P.in_c;
+        a.ring_elems = (long long)P.e_cap * S * P.out_w * P.out_c;
+        a.out_elems = S * out_cap * P.out_w * P.out_c;
+        a.status = (unsigned int*)(net->ws + net->status_off);
         // (rows beyond the caller's buffer are not written: they hold nothing the caller will read)
         if (last && a.o_hi >= out_cap) a.o_hi = out_cap - 1;
         cudaError_t ce = launch_eager_layer(a, P.l.kind == IDF_MAXPOOL2, int_net, net->stream);
@@ -1079,6 +1100,7 @@ int idf_stream_status(idf_net* net, long long* tensor_core_launches)
     if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "stream_status: %s", cudaGetErrorString(e));
     if (tensor_core_launches)
         for (size_t i = 0; i < net->L.size(); ++i) tensor_core_launches[i] = net->L[i].tc_launches;
+    if (st & 2u) return fail(IDF_ERR_BOUNDS, "an index check of the range-checked build failed (the access was skipped; results are invalid)");
     if (st != 0) return fail(IDF_ERR_TIMEOUT, "a bounded device-side wait ran out (kernel gave up)");
     return IDF_OK;
 }

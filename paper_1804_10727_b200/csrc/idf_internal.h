@@ -10,6 +10,24 @@ namespace idf {
 // element types of activation rows travelling between layers
 enum Elem : int { E_F32 = 0, E_BF16 = 1, E_I8 = 2, E_I32 = 3 };
 
+// Range-checked build (-DIDF_BOUNDS): every index into a ring, a row buffer, shared memory or tensor memory is
+// compared with the extent of what it indexes before the access; a violation sets bit 1 of the handle's status
+// word (idf_stream_status then reports IDF_ERR_BOUNDS) and the access is skipped - never a trap, never a wild
+// access.  In the regular build the checks compile to nothing.
+#ifdef __CUDACC__
+#ifdef IDF_BOUNDS
+__device__ __forceinline__ bool bounds_ok(unsigned int* status, long long idx, long long extent)
+{
+    if (idx >= 0 && idx < extent) return true;
+    if (status) atomicOr(status, 2u);
+    return false;
+}
+#define IDF_OK_AT(status, idx, extent) idf::bounds_ok((status), (long long)(idx), (long long)(extent))
+#else
+#define IDF_OK_AT(status, idx, extent) true
+#endif
+#endif
+
 // process-wide debug switches (bits of idf_debug_flag), set through idf_set_debug_flags
 unsigned debug_flags();
 
@@ -43,6 +61,9 @@ struct ConvArgs {
     int pool_fused;        // 1: emit pooled rows
     int pool_keep;         // 1: more input may follow (a trailing first row of a pair waits in pool_state); 0: end of input
     void* pool_state;      // the pool layer's state: [S][Wout/2][Cout] in the output type
+    // extents in elements of what the pointers above address (range-checked build) and the handle's status word
+    long long in_elems, out_elems, ring_elems, pool_state_elems;
+    unsigned int* status;
 };
 
 struct PoolArgs {
@@ -52,6 +73,8 @@ struct PoolArgs {
     long long out_row_stride, out_stream_stride, out_row_base;
     int S, Win, Wout, C, elem;
     long long r0, r1, o_begin, o_end, done_end;
+    long long in_elems, out_elems, state_elems;   // extents (range-checked build)
+    unsigned int* status;
 };
 
 // Global-average sink: every arriving row is added into one running sum per (stream, channel); the
@@ -64,6 +87,8 @@ struct AvgArgs {
     int S, W, C, elem;
     long long n_rows;      // rows arriving in this launch
     long long rows_total;  // rows received since open, these included
+    long long in_elems, out_elems, sum_elems;     // extents (range-checked build)
+    unsigned int* status;
 };
 
 // Eager emission (one segment per step): how one layer re-evaluates the rows of its input cone.
@@ -86,6 +111,8 @@ struct EagerArgs {
     long long o_lo, o_hi;     // rows of this layer to re-evaluate
     long long o_new;          // rows >= o_new are touched for the first time (their slots hold an older row)
     long long o_cut;          // rows >= o_cut turn out not to exist (end of input): their activation goes back to 0
+    long long in_elems, ring_elems, out_elems;    // extents of din/hin, of each of c/h/d, of out (range-checked build)
+    unsigned int* status;
 };
 cudaError_t launch_eager_input(const void* in, int in_elem, void* d, long long n, unsigned long long* events, cudaStream_t st);
 cudaError_t launch_eager_layer(const EagerArgs& a, int is_pool, int int_net, cudaStream_t st);

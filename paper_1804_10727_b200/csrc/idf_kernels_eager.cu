@@ -45,11 +45,13 @@ __device__ __forceinline__ void count_events(unsigned long long* counter, bool n
 
 __device__ __forceinline__ void write_out(const EagerArgs& a, long long o, int s, int x, int co, float h)
 {
-    ((float*)a.out)[(long long)s * a.out_stream_stride + o * a.out_row_stride + (long long)x * a.Cout + co] = h;
+    const long long i = (long long)s * a.out_stream_stride + o * a.out_row_stride + (long long)x * a.Cout + co;
+    if (IDF_OK_AT(a.status, i, a.out_elems)) ((float*)a.out)[i] = h;
 }
 __device__ __forceinline__ void write_out(const EagerArgs& a, long long o, int s, int x, int co, int h)
 {
-    ((int8_t*)a.out)[(long long)s * a.out_stream_stride + o * a.out_row_stride + (long long)x * a.Cout + co] = (int8_t)h;
+    const long long i = (long long)s * a.out_stream_stride + o * a.out_row_stride + (long long)x * a.Cout + co;
+    if (IDF_OK_AT(a.status, i, a.out_elems)) ((int8_t*)a.out)[i] = (int8_t)h;
 }
 
 // The pushed segment as the input layer's announcement: input units start at 0, so dh = x (paragraph after Eq. 3).
@@ -98,6 +100,7 @@ __global__ void __launch_bounds__(256) eager_conv_kernel(EagerArgs a)
                     const long long i = o * a.stride - a.pad + ky;
                     if (i < a.in_lo || i > a.in_hi) continue;
                     const TS* drow = din + ((i % a.cap_in) * a.S + s) * (long long)a.Win * a.Cin;
+                    if (!IDF_OK_AT(a.status, (drow - din) + (long long)a.Win * a.Cin - 1, a.in_elems)) continue;
                     for (int kx = 0; kx < a.Kw; ++kx) {
                         const int ix = x * a.stride_x - a.pad_x + kx;
                         if (ix < 0 || ix >= a.Win) continue;
@@ -110,6 +113,7 @@ __global__ void __launch_bounds__(256) eager_conv_kernel(EagerArgs a)
                     }
                 }
             const long long e = (((o % a.cap) * a.S + s) * a.Wout + x) * (long long)a.Cout + co;
+            if (!IDF_OK_AT(a.status, e, a.ring_elems)) continue;
             const bool fresh = o >= a.o_new;                        // first touch: the slot still holds an older row
             const TS cn = (fresh ? (TS)0 : cr[e]) + acc;
             const TS hold = fresh ? (TS)0 : hr[e];
@@ -151,12 +155,14 @@ __global__ void __launch_bounds__(256) eager_pool_kernel(EagerArgs a)
                 const long long i = 2 * o + dy;
                 for (int dx = 0; dx < px; ++dx) {
                     TS v = 0;                                          // a unit that has announced nothing stands at 0
-                    if (i <= a.in_hi) v = hin[(((i % a.cap_in) * a.S + s) * a.Win + (px * x + dx)) * (long long)a.Cin + c];
+                    const long long hi_at = (((i % a.cap_in) * a.S + s) * a.Win + (px * x + dx)) * (long long)a.Cin + c;
+                    if (i <= a.in_hi && IDF_OK_AT(a.status, hi_at, a.in_elems)) v = hin[hi_at];
                     m = have ? (v > m ? v : m) : v;
                     have = true;
                 }
             }
             const long long e = (((o % a.cap) * a.S + s) * a.Wout + x) * (long long)a.Cout + c;
+            if (!IDF_OK_AT(a.status, e, a.ring_elems)) continue;
             const TS hold = o >= a.o_new ? (TS)0 : hr[e];
             const TS hn = o >= a.o_cut ? (TS)0 : m;
             hr[e] = hn;

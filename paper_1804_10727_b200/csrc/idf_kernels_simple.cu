@@ -80,12 +80,13 @@ __global__ void __launch_bounds__(256) conv_rows_kernel(ConvArgs a, long long in
                     const int ix = x * a.stride_x - a.pad_x + kx;
                     if (ix < 0 || ix >= a.Win) continue;
                     const TI* ap = row + (long long)ix * a.Cin;
+                    if (!IDF_OK_AT(a.status, (ap - in) + a.Cin - 1, a.in_elems)) continue;
                     const TW* wp = w + ((long long)(ky * a.Kw + kx) * a.Cin) * a.Cout + co;
                     for (int ci = 0; ci < a.Cin; ++ci) acc += to_acc(ap[ci]) * to_acc(wp[(long long)ci * a.Cout]);
                 }
             }
-            out[(o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride + (long long)x * a.Cout + co] =
-                Emit<TO, TS>::run(acc, bias ? bias[co] : (TS)0, a.relu, a.shift);
+            const long long oi = (o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride + (long long)x * a.Cout + co;
+            if (IDF_OK_AT(a.status, oi, a.out_elems)) out[oi] = Emit<TO, TS>::run(acc, bias ? bias[co] : (TS)0, a.relu, a.shift);
         }
         return;
     }
@@ -104,6 +105,7 @@ __global__ void __launch_bounds__(256) conv_rows_kernel(ConvArgs a, long long in
         bool dirty = false;
         TS leave = 0;
         TS* rp = ring + ((long long)slot * a.S + s) * row_elems + (long long)x * a.Cout + co;
+        if (!IDF_OK_AT(a.status, rp - ring, a.ring_elems)) continue;
         for (; o < a.o_end; o += a.ring_rows) {
             if (o >= int_begin && o < int_end) continue;         // an interior row: another CTA's
             TS acc = 0;
@@ -115,6 +117,7 @@ __global__ void __launch_bounds__(256) conv_rows_kernel(ConvArgs a, long long in
                     const int ix = x * a.stride_x - a.pad_x + kx;
                     if (ix < 0 || ix >= a.Win) continue;
                     const TI* ap = row + (long long)ix * a.Cin;
+                    if (!IDF_OK_AT(a.status, (ap - in) + a.Cin - 1, a.in_elems)) continue;
                     const TW* wp = w + ((long long)(ky * a.Kw + kx) * a.Cin) * a.Cout + co;
                     for (int ci = 0; ci < a.Cin; ++ci) acc += to_acc(ap[ci]) * to_acc(wp[(long long)ci * a.Cout]);
                 }
@@ -122,8 +125,8 @@ __global__ void __launch_bounds__(256) conv_rows_kernel(ConvArgs a, long long in
             const bool carried_in = (a.r0 > 0) && (o * a.stride - a.pad < a.r0);
             const TS c = acc + (carried_in ? *rp : (TS)0);
             if (o < a.done_end) {
-                out[(o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride +
-                    (long long)x * a.Cout + co] = Emit<TO, TS>::run(c, b, a.relu, a.shift);
+                const long long oi = (o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride + (long long)x * a.Cout + co;
+                if (IDF_OK_AT(a.status, oi, a.out_elems)) out[oi] = Emit<TO, TS>::run(c, b, a.relu, a.shift);
                 if (carried_in) { dirty = true; leave = 0; }
             } else {
                 dirty = true;
@@ -155,11 +158,13 @@ __global__ void __launch_bounds__(256) conv_flush_kernel(ConvArgs a)
         const int s = (int)(t % a.S);
         const long long o = a.o_begin + t / a.S;
         TS* rp = ring + ((o % a.ring_rows) * a.S + s) * row_elems + (long long)x * a.Cout + co;
+        if (!IDF_OK_AT(a.status, (rp - ring) + 3, a.ring_elems)) continue;
         __align__(16) TS c[4];
         *(int4*)c = *(const int4*)rp;
         if (o >= a.done_end) continue;               // a row that can never complete: left as it is
         *(int4*)rp = make_int4(0, 0, 0, 0);
         TO* op = out + (o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride + (long long)x * a.Cout + co;
+        if (!IDF_OK_AT(a.status, (op - out) + 3, a.out_elems)) continue;
 #pragma unroll
         for (int j = 0; j < 4; ++j) op[j] = Emit<TO, TS>::run(c[j], bias ? bias[co + j] : (TS)0, a.relu, a.shift);
     }
@@ -268,7 +273,8 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
     if (RING_IN_SMEM) {
         for (int i = tid; i < a.ring_rows * row_elems; i += SPARSE_THREADS) {
             const int slot = i / row_elems, e = i - slot * row_elems;
-            ring[i] = gring[((long long)slot * a.S + s) * row_elems + e];
+            const long long gi = ((long long)slot * a.S + s) * row_elems + e;
+            if (IDF_OK_AT(a.status, gi, a.ring_elems)) ring[i] = gring[gi];
         }
     }
     __syncthreads();
@@ -282,6 +288,8 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
         for (; done < upto; ++done) {
             const long long slot = done % a.ring_rows;
             TO* orow = out + (done - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride;
+            if (!IDF_OK_AT(a.status, (orow - out) + row_elems - 1, a.out_elems) || !IDF_OK_AT(a.status, orow - out, a.out_elems) ||
+                !IDF_OK_AT(a.status, (slot + 1) * (long long)row_elems - 1, (long long)a.ring_rows * row_elems)) continue;
             if (sizeof(TO) == 1 && (a.Cout & 3) == 0 && (((uintptr_t)orow) & 3) == 0) {
                 // int8 rows: four channels per thread, one 4-byte store
                 const bool pow2 = (a.Cout & (a.Cout - 1)) == 0;
@@ -339,6 +347,7 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
             if (upto > a.done_end) upto = a.done_end;
         }
         const TI* row = in + ((r - a.r0) * a.S + s) * (long long)n_comp;
+        if (have && !IDF_OK_AT(a.status, (row - in) + n_comp - 1, a.in_elems)) continue;
         const int n_pass = have ? (n_comp + SPARSE_MAX_EVENTS - 1) / SPARSE_MAX_EVENTS : 1;
         for (int pass = 0; pass < n_pass; ++pass) {
             const int base = pass * SPARSE_MAX_EVENTS;
@@ -357,6 +366,7 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
                         off = __shfl_sync(0xffffffffu, off, 0);
                         if (v != (TS)0) {
                             const int k = off + __popc(m & ((1u << lane) - 1u));
+                            if (!IDF_OK_AT(a.status, k, SPARSE_MAX_EVENTS)) continue;
                             const int x = i / a.Cin;
                             ev_x[k] = (short)x;
                             ev_ci[k] = (short)(i - x * a.Cin);
@@ -393,6 +403,7 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
                             for (int kx = 0; kx < 3; ++kx) {
                                 const int ox = x - kx;
                                 if (ox < 0 || ox >= a.Wout) continue;
+                                if (!IDF_OK_AT(a.status, soff[ky] + ox * a.Cout + co, (long long)a.ring_rows * row_elems)) continue;
                                 atomic_add_shared(ring_s + soff[ky] + ox * a.Cout + co, val * wp[(ky * 3 + kx) * tap_w + co]);
                             }
                         }
@@ -419,6 +430,7 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
                         if (ox >= a.Wout) continue;
                         const int wofs = kx * a.Cin * a.Cout;
                         TS* dst = drow + ox * a.Cout;
+                        if (!IDF_OK_AT(a.status, (dst - ring) + a.Cout - 1, RING_IN_SMEM ? (long long)a.ring_rows * row_elems : a.ring_elems)) continue;
                         for (int co = lane; co < a.Cout; co += 32) {
                             const TS wv = w_in_smem ? w_s[wrow_i + wofs + co] : (TS)to_acc(wrow[wofs + co]);
                             if (RING_IN_SMEM) atomic_add_shared(dst + co, val * wv);
@@ -435,7 +447,8 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
     if (RING_IN_SMEM) {
         for (int i = tid; i < a.ring_rows * row_elems; i += SPARSE_THREADS) {
             const int slot = i / row_elems, e = i - slot * row_elems;
-            gring[((long long)slot * a.S + s) * row_elems + e] = ring[i];
+            const long long gi = ((long long)slot * a.S + s) * row_elems + e;
+            if (IDF_OK_AT(a.status, gi, a.ring_elems)) gring[gi] = ring[i];
         }
     }
     if (tid == 0 && a.event_counter && ev_total) atomicAdd(a.event_counter, ev_total);
@@ -481,7 +494,8 @@ cudaError_t launch_conv_sparse(const ConvArgs& a, int dtype, cudaStream_t st)
 // ------------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256) unfold_rows_kernel(const T* __restrict__ in, T* __restrict__ out, long long n_pos,
-                                                          int Win, int Wout, int Cin, int Kw, int stride_x, int pad_x, int kpad)
+                                                          int Win, int Wout, int Cin, int Kw, int stride_x, int pad_x, int kpad,
+                                                          long long in_elems, unsigned int* status)
 {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     constexpr int V = 16 / (int)sizeof(T);
@@ -502,7 +516,8 @@ __global__ void __launch_bounds__(256) unfold_rows_kernel(const T* __restrict__ 
             const int kx = k0 / Cin, ci = k0 - kx * Cin;
             const int ix = xo * stride_x - pad_x + kx;
             int4 q = make_int4(0, 0, 0, 0);
-            if (kx < Kw && ix >= 0 && ix < Win) q = *(const int4*)(row + (long long)ix * Cin + ci);
+            if (kx < Kw && ix >= 0 && ix < Win && IDF_OK_AT(status, (row - in) + (long long)ix * Cin + ci + V - 1, in_elems))
+                q = *(const int4*)(row + (long long)ix * Cin + ci);
             *(int4*)(out + p * kpad + (long long)v * V) = q;
             continue;
         }
@@ -513,7 +528,7 @@ __global__ void __launch_bounds__(256) unfold_rows_kernel(const T* __restrict__ 
 #pragma unroll
         for (int j = 0; j < V; ++j) {
             const int e = e0 + j;
-            vals[j] = (j < k_end && e >= 0 && e < e_end) ? row[e] : (T)0;
+            vals[j] = (j < k_end && e >= 0 && e < e_end && IDF_OK_AT(status, (row - in) + e, in_elems)) ? row[e] : (T)0;
         }
         *(int4*)(out + p * kpad + (long long)v * V) = *(const int4*)vals;
     }
@@ -529,10 +544,10 @@ cudaError_t launch_unfold(const ConvArgs& a, int n_rows, int kpad, void* out, cu
     if (blocks > 148LL * 32) blocks = 148LL * 32;
     if (a.in_elem == E_BF16)
         unfold_rows_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)a.in, (__nv_bfloat16*)out, n_pos,
-                                                                          a.Win, a.Wout, a.Cin, a.Kw, a.stride_x, a.pad_x, kpad);
+                                                                          a.Win, a.Wout, a.Cin, a.Kw, a.stride_x, a.pad_x, kpad, a.in_elems, a.status);
     else if (a.in_elem == E_I8)
         unfold_rows_kernel<int8_t><<<(unsigned)blocks, 256, 0, st>>>((const int8_t*)a.in, (int8_t*)out, n_pos, a.Win, a.Wout,
-                                                                   a.Cin, a.Kw, a.stride_x, a.pad_x, kpad);
+                                                                   a.Cin, a.Kw, a.stride_x, a.pad_x, kpad, a.in_elems, a.status);
     else
         return cudaErrorInvalidValue;
     return cudaGetLastError();
@@ -566,22 +581,22 @@ __global__ void __launch_bounds__(256) pool_rows_kernel(PoolArgs a)
         for (long long o = a.o_begin; o < a.o_end; ++o) {
             bool have = false;
             T m = (T)0;
+            if (!IDF_OK_AT(a.status, idx, a.state_elems)) continue;
             if (2 * o < a.r0) { m = state[idx]; have = true; }
             for (int dy = 0; dy < 2; ++dy) {
                 const long long r = 2 * o + dy;
                 if (r < a.r0 || r >= a.r1) continue;
                 const T* row = in + ((r - a.r0) * a.S + s) * (long long)a.Win * a.C;
                 for (int dx = 0; dx < px; ++dx) {
+                    if (!IDF_OK_AT(a.status, (row - in) + (long long)(px * ox + dx) * a.C + c, a.in_elems)) continue;
                     const T v = row[(long long)(px * ox + dx) * a.C + c];
                     m = have ? max_of(m, v) : v;
                     have = true;
                 }
             }
-            if (o < a.done_end)
-                out[(o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride +
-                    (long long)ox * a.C + c] = m;
-            else
-                state[idx] = m;
+            const long long oi = (o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride + (long long)ox * a.C + c;
+            if (o < a.done_end) { if (IDF_OK_AT(a.status, oi, a.out_elems)) out[oi] = m; }
+            else state[idx] = m;
         }
     }
 }
@@ -620,6 +635,7 @@ __global__ void __launch_bounds__(256) pool_rows_vec_kernel(PoolArgs a)
         for (int turn = 0; turn < 2; ++turn) {
             __align__(16) T m[V];
             bool have = false;
+            if (!IDF_OK_AT(a.status, sidx + V - 1, a.state_elems)) break;
             if (2 * o < a.r0) { *(int4*)m = *(const int4*)(state + sidx); have = true; }
             for (int dy = 0; dy < 2; ++dy) {
                 const long long r = 2 * o + dy;
@@ -627,17 +643,16 @@ __global__ void __launch_bounds__(256) pool_rows_vec_kernel(PoolArgs a)
                 const T* row = in + ((r - a.r0) * a.S + s) * (long long)a.Win * a.C;
                 for (int dx = 0; dx < px; ++dx) {
                     __align__(16) T v[V];
+                    if (!IDF_OK_AT(a.status, (row - in) + (long long)(px * ox + dx) * a.C + c + V - 1, a.in_elems)) continue;
                     *(int4*)v = *(const int4*)(row + (long long)(px * ox + dx) * a.C + c);
 #pragma unroll
                     for (int j = 0; j < V; ++j) m[j] = have ? max_of(m[j], v[j]) : v[j];
                     have = true;
                 }
             }
-            if (o < a.done_end)
-                *(int4*)(out + (o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride +
-                         (long long)ox * a.C + c) = *(const int4*)m;
-            else
-                *(int4*)(state + sidx) = *(const int4*)m;
+            const long long oi = (o - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride + (long long)ox * a.C + c;
+            if (o < a.done_end) { if (IDF_OK_AT(a.status, oi + V - 1, a.out_elems)) *(int4*)(out + oi) = *(const int4*)m; }
+            else *(int4*)(state + sidx) = *(const int4*)m;
             if (!(chained && o == a.o_begin)) break;
             o = a.o_end - 1;
         }
@@ -699,13 +714,15 @@ __global__ void __launch_bounds__(256) avg_rows_kernel(AvgArgs a)
          idx += (long long)gridDim.x * blockDim.x) {
         const int c = (int)(idx % a.C);
         const long long s = idx / a.C;
+        if (!IDF_OK_AT(a.status, idx, a.sum_elems)) continue;
         TS acc = sum[idx];
         for (long long r = 0; r < a.n_rows; ++r) {
             const TI* row = in + (r * a.S + s) * (long long)a.W * a.C + c;
+            if (!IDF_OK_AT(a.status, (row - in) + (long long)(a.W - 1) * a.C, a.in_elems)) continue;
             for (int x = 0; x < a.W; ++x) acc += avg_term(row[(long long)x * a.C]);
         }
         sum[idx] = acc;
-        a.out[s * a.out_stream_stride + c] = (float)((double)acc / count);
+        if (IDF_OK_AT(a.status, s * a.out_stream_stride + c, a.out_elems)) a.out[s * a.out_stream_stride + c] = (float)((double)acc / count);
     }
 }
 cudaError_t launch_avg(const AvgArgs& a, cudaStream_t st)

@@ -481,6 +481,8 @@ struct TcArgs {
     int o_begin_half_mod;        // (o_begin >> 1) mod out_groups
     int ring_slot0;              // o_begin mod ring_rows
     int pool_row_first;          // (o_begin >> 1) - pool_row_base: tensor-map row of the pair that holds o_begin
+    long long ring_elems, pool_state_bytes;   // extents of ring (state words) and pool_state (bytes): range-checked build
+    unsigned int smem_bytes;     // dynamic shared memory of the launch (range-checked build)
 };
 
 template <int DT> struct Acc;
@@ -545,6 +547,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (threadIdx.x == 0) {
         s_abort = 0;
         s_issued = 0;
+        if (!IDF_OK_AT(a.status, (bar_free - smem_u32(smem_raw)) + 8u * a.nslot - 1, a.smem_bytes)) s_abort = 1;
         for (int i = 0; i < a.nstage; ++i) { mbar_init(bar_full + 8u * i, 1); mbar_init(bar_empty + 8u * i, 1); }
         for (int i = 0; i < taps; ++i) mbar_init(bar_w + 8u * i, 1);
         for (int i = 0; i < a.nslot; ++i) { mbar_init(bar_ready + 8u * i, 1); mbar_init(bar_free + 8u * i, 4); }
@@ -644,6 +647,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int xl = 0; xl < n_xload && ok; ++xl)
                         for (int kb = 0; kb < a.n_kb; ++kb) {
                             if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                            if (!IDF_OK_AT(a.status, (sA - smem_u32(smem_raw)) + (uint32_t)stage * a_stage_bytes + a_box_bytes - 1, bars - smem_u32(smem_raw))) { ok = false; break; }
                             mbar_expect_tx(bar_full + 8u * stage, a_box_bytes);
                             tma_load_4d(sA + (uint32_t)stage * a_stage_bytes, &tmA, bar_full + 8u * stage,
                                         kb * a.KB, x0 * a.sx - a.pad_x + xl, s0, c_ra + ri);
@@ -880,10 +884,26 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             TS* rp = ring_pos + (long long)rslot * ring_slot_stride;
             const uint32_t trow = tlane + (uint32_t)(slot * a.Ntile);
+            bool fine = true;           // range-checked build: false skips this row's accesses (the barriers still run)
+#ifdef IDF_BOUNDS
+            {
+                fine = IDF_OK_AT(a.status, slot * a.Ntile + a.Ntile - 1, a.tmem_cols);
+                if (valid && (carried_in || !emit)) fine = fine && IDF_OK_AT(a.status, (rp - (TS*)a.ring) + a.Ntile - 1, a.ring_elems);
+                if (pool_emit && state_ok && (pc.from_state || pc.to_state))
+                    fine = fine && IDF_OK_AT(a.status, (pc.state - (unsigned char*)a.pool_state) + (long long)a.Ntile * a.out_esize - 1, a.pool_state_bytes);
+                // (a launch that emits pooled rows stages them in the half-size tile; the full-size addresses are not used then)
+                const uint32_t stage_row = a.pool ? pc.sink.row_base : sink.row_base;
+                if (emit && (a.pool ? pc.writer != 0 : in_tile))
+                    fine = fine && IDF_OK_AT(a.status, (stage_row - smem_u32(smem_raw)) + (uint32_t)(a.out_panels - 1) * sink.panel_bytes + a.out_pwb - 1,
+                                             bars - smem_u32(smem_raw));
+                fine = __all_sync(0xffffffffu, fine) != 0;     // (the tensor-memory loads below are warp-wide instructions)
+            }
+#endif
             {
                 if (wide) {
                     for (int c = 0; c < a.Ntile; c += 32) {
                         uint32_t v[32];
+                        if (!fine) continue;
                         tmem_ld<32>(trow + c, v);
                         tmem_ld_wait();
                         tmem_st_zero<32>(trow + c);           // the slot's next row starts from zero
@@ -894,6 +914,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 } else {
                     for (int c = 0; c < a.Ntile; c += 16) {
                         uint32_t v[16];
+                        if (!fine) continue;
                         tmem_ld<16>(trow + c, v);
                         tmem_ld_wait();
                         tmem_st_zero<16>(trow + c);
@@ -1165,6 +1186,7 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     t.o_begin_half_mod = (int)((a.o_begin >> 1) % p.out_groups);
     t.ring_slot0 = (int)(a.o_begin % a.ring_rows);
     t.pool_row_first = (int)((a.o_begin >> 1) - a.out_row_base);
+    t.ring_elems = a.ring_elems; t.pool_state_bytes = a.pool_state_elems * p.out_esize; t.smem_bytes = (unsigned int)p.smem_bytes;
     // row chunks: a layer with few tiles (few streams, narrow rows) spreads the block's rows over more CTAs
     t.n_chunks = 1; t.chunk_rows = t.n_orows; t.chunk_shift = 0;
     {

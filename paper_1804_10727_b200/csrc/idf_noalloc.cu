@@ -112,6 +112,10 @@ extern "C" int idf_conv_rows_noalloc(const float* d_in, int n_rows, int n_stream
         a.S = n_streams; a.Win = in_w; a.Wout = out_w; a.Cin = cin; a.Cout = cout; a.Kh = kh; a.Kw = kw;
         a.stride = stride; a.pad = pad; a.relu = relu; a.shift = 0; a.ring_rows = ring_rows;
         a.stride_x = stride_x; a.pad_x = pad_x; a.in_elem = E_F32; a.out_elem = E_F32;
+        a.in_elems = (r1 - r0) * (long long)n_streams * in_w * cin;
+        a.out_elems = (long long)n_streams * out_capacity_rows * out_w * cout;
+        a.ring_elems = (long long)ring_rows * n_streams * out_w * cout;
+        a.status = nullptr;          // (no handle, no status word: the range-checked build still skips what is out of range)
         a.r0 = r0; a.r1 = r1; a.o_begin = rows_done; a.o_end = started > done_end ? started : done_end; a.done_end = done_end;
         e = launch_conv_simple(a, IDF_F32, st);
         if (e != cudaSuccess) return set_last_error(IDF_ERR_CUDA, "noalloc: kernel launch failed");

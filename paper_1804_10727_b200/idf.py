@@ -15,14 +15,22 @@ import torch
 
 _HERE = Path(__file__).resolve().parent
 LIB_PATH = _HERE / "libidf.so"
+BOUNDS_LIB_PATH = _HERE / "libidf_bounds.so"      # the range-checked build of the same sources (-DIDF_BOUNDS)
 _lib = None
+
+
+def use_library(path) -> None:
+    """Load the library from ``path`` from now on (e.g. ``BOUNDS_LIB_PATH``); handles made before stay with theirs."""
+    global _lib, LIB_PATH
+    LIB_PATH = Path(path)
+    _lib = None
 
 F32, BF16_F32, I8_I32 = 0, 1, 2
 CONV, MAXPOOL2, GLOBAL_AVG = 0, 1, 2
 PATH_AUTO, PATH_DENSE, PATH_SPARSE = 0, 1, 2
 DTYPES = {"f32": F32, "bf16": BF16_F32, "i8": I8_I32}
 
-OK, ERR_ARG, ERR_SPEC, ERR_STATE, ERR_CAPACITY, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5, -6, -7
+OK, ERR_ARG, ERR_SPEC, ERR_STATE, ERR_CAPACITY, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_BOUNDS = 0, -1, -2, -3, -4, -5, -6, -7, -8
 
 EXPORTS = (
     "idf_net_create", "idf_net_destroy", "idf_net_state_bytes", "idf_net_workspace_bytes", "idf_out_shape",
