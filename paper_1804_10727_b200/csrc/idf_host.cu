@@ -45,6 +45,12 @@ struct LayerPlan {
     TcPlan tc_pool;                         // plan of the launches that also emit the following max-pool's rows
     alignas(64) unsigned char w_map_pool[128];
     long long tc_launches = 0;
+    // thin layers (the whole receptive field of an output position in one shared-memory row): a kernel of its own for
+    // the rows a block determines completely
+    ThinPlan thin;
+    std::vector<unsigned char> wthin_packed;   // [Cout][row bytes] in the activation type, zero padded
+    size_t wthin_off = 0;
+    alignas(64) unsigned char w_map_thin[128];
     // x-unfold in front of the tensor-core kernel (thin or x-strided layers): the Kw taps of every
     // output position are laid side by side as kpad channels, the conv then has Kw = 1, stride_x = 1
     int unfold = 0, kpad = 0, in_cap_rows = 0;
@@ -211,7 +217,22 @@ int launch_layer(idf_net* net, size_t i, const void* in_ptr, long long n_in, boo
         a.ring_rows = P.ring_rows; a.in_elem = P.in_elem; a.out_elem = P.out_elem;
         a.r0 = r0; a.r1 = r1; a.o_begin = o_begin; a.o_end = o_end; a.done_end = done_end;
         ce = cudaErrorNotSupported;
-        if (P.tc.ok && !P.use_sparse && n_in > 0) {
+        if (P.thin.ok && !P.use_sparse && n_in > 0) {
+            // rows not begun by an earlier block (first tap row o*stride - pad >= r0) and completed by this one: the
+            // thin-layer kernel computes them from the block's rows alone; the others exchange state with the ring
+            long long int_begin = r0 > 0 ? (r0 + P.l.pad + P.l.stride - 1) / P.l.stride : o_begin;
+            if (int_begin < o_begin) int_begin = o_begin;
+            const long long int_end = done_end;
+            if (int_end - int_begin >= 4) {
+                ce = launch_conv_thin(a, P.thin, net->dtype, P.w_map_thin, int_begin, int_end, status, net->stream);
+                if (ce == cudaSuccess) {
+                    net->launches += 1;
+                    P.tc_launches += 1;
+                    ce = launch_conv_edges(a, net->dtype, int_begin, int_end, net->stream);
+                }
+            }
+        }
+        if (ce == cudaErrorNotSupported && P.tc.ok && !P.use_sparse && n_in > 0) {
             ConvArgs t = a;
             if (P.unfold && n_in <= P.in_cap_rows) {
                 ce = launch_unfold(a, (int)n_in, P.kpad, net->ws + P.unf_off, net->stream);
@@ -627,7 +648,7 @@ const char* idf_last_error(void) { return g_err.c_str(); }
 
 int idf_set_debug_flags(unsigned int flags)
 {
-    if (flags & ~(unsigned)(IDF_DEBUG_NO_TENSOR_CORES | IDF_DEBUG_NO_POOL_FUSION | IDF_DEBUG_NO_ROW_CHUNKS | IDF_DEBUG_NO_PDL))
+    if (flags & ~(unsigned)(IDF_DEBUG_NO_TENSOR_CORES | IDF_DEBUG_NO_POOL_FUSION | IDF_DEBUG_NO_ROW_CHUNKS | IDF_DEBUG_NO_PDL | IDF_DEBUG_PREFER_THIN))
         return fail(IDF_ERR_ARG, "unknown debug flag in 0x%x", flags);
     g_debug_flags.store(flags, std::memory_order_relaxed);
     return IDF_OK;
@@ -756,6 +777,20 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
                                    (size_t)l.kw * l.cin * es);
                 }
             }
+            // A layer whose whole receptive field fits one 128-byte row gets the thin-layer kernel where the row-ring kernel
+            // has no good form for it: 1D nets (behind an x-unfold pass every tap row would carry Cin values padded to a
+            // K step: audio1d's first layer 1.68 -> 0.84 ms) and shapes it cannot take at all.  2D layers with kx taps stay
+            // with x-unfold + row ring (vgg2d conv1: 0.19 ms against 0.52 ms: building 27-value rows element by element
+            // costs more than the unfold pass saves).
+            const bool prefer_thin = (debug_flags() & IDF_DEBUG_PREFER_THIN) != 0;
+            if (tc_allowed && ((P.unfold && (w == 1 || prefer_thin)) || !P.tc.ok) && !(pool_next && P.tc_pool.ok) &&
+                thin_make_plan(spec->dtype, net->n_streams, P.out_w, l.cin, l.cout, l.kh, l.kw, l.stride, w == 1 ? 1 : l.stride,
+                               (int)elem_size(P.out_elem), &P.thin)) {
+                P.wthin_packed.assign((size_t)l.cout * P.thin.swb, 0);
+                for (int co = 0; co < l.cout; ++co)
+                    memcpy(P.wthin_packed.data() + (size_t)co * P.thin.swb, (const unsigned char*)weights[i] + (size_t)co * taps * l.cin * es,
+                           (size_t)taps * l.cin * es);
+            }
             if (biases && biases[i]) {
                 // an all-zero bias is no bias: the kernels then skip the add (state words: +0.0f and 0 are all-zero bits)
                 bool any = false;
@@ -825,6 +860,7 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
         P.w_off = off; off = align_up(off + P.w_packed.size());
         P.b_off = off; off = align_up(off + P.b_packed.size());
         P.wtc_off = off; off = align_up(off + P.wtc_packed.size(), 1024);
+        P.wthin_off = off; off = align_up(off + P.wthin_packed.size(), 1024);
     }
     net->state_region_off = off;
     for (auto& P : net->L) {
@@ -926,6 +962,10 @@ int idf_stream_open(idf_net* net, void* d_workspace, size_t workspace_bytes, voi
             if (P.tc_pool.ok && tc_encode_weights(P.tc_pool, net->dtype, net->ws + P.wtc_off, P.unfold ? P.l.kh : P.l.kh * P.l.kw,
                                                   P.unfold ? P.kpad : P.l.cin, P.l.cout, P.w_map_pool) != 0)
                 P.tc_pool.ok = 0;
+        }
+        if (!P.wthin_packed.empty() && e == cudaSuccess) {
+            e = cudaMemcpyAsync(net->ws + P.wthin_off, P.wthin_packed.data(), P.wthin_packed.size(), cudaMemcpyHostToDevice, net->stream);
+            if (thin_encode_weights(P.thin, net->dtype, net->ws + P.wthin_off, P.l.cout, P.w_map_thin) != 0) P.thin.ok = 0;
         }
     }
     if (e != cudaSuccess) { net->phase = CREATED; return fail(IDF_ERR_CUDA, "stream_open: %s", cudaGetErrorString(e)); }

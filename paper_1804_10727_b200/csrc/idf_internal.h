@@ -145,6 +145,26 @@ int tc_encode_weights(const TcPlan& p, int dtype, const void* d_w, int taps, int
 cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const void* w_map, int n_in_rows,
                            unsigned int* status, cudaStream_t st);
 
+// Static plan of the thin-layer kernel (the whole Kh*Kw*Cin-wide receptive field in one swizzled shared-memory row).
+struct ThinPlan {
+    int ok = 0;
+    int swb = 0;             // bytes of one im2col row: 32, 64 or 128 (the swizzle span)
+    int kelems = 0;          // Kh*Kw*Cin values of a row, zero padded to swb bytes
+    int ksteps = 0;          // 32-byte MMA K steps
+    int BX = 0, BS = 0, n_xt = 0, n_mt = 0;   // a 128-position tile = BS streams x BX consecutive x positions
+    int R = 0;               // output rows per work item
+    int nstage = 0, tmem_cols = 0;
+    int out_esize = 0, out_pwb = 0, out_panels = 0, out_tile_bytes = 0;
+    size_t smem_bytes = 0, w_bytes = 0;      // w_bytes: device weights [Cout][swb] in the activation type
+};
+bool thin_make_plan(int dtype, int S, int Wout, int Cin, int Cout, int Kh, int Kw, int stride, int stride_x, int out_esize, ThinPlan* p);
+int thin_encode_weights(const ThinPlan& p, int dtype, const void* d_w, int Cout, void* map_out);
+cudaError_t launch_conv_thin(const ConvArgs& a, const ThinPlan& p, int dtype, const void* w_map, long long o_first, long long o_end,
+                             unsigned int* status, cudaStream_t st);
+// CUDA-core conv kernel on the rows that exchange state with the ring only: rows [skip_begin, skip_end) are left to
+// another kernel
+cudaError_t launch_conv_edges(const ConvArgs& a, int dtype, long long skip_begin, long long skip_end, cudaStream_t st);
+
 // x-unfold: out[row][s][x'][kx*Cin + ci] = in[row][s][x'*stride_x - pad_x + kx][ci] (0 outside the row or
 // beyond Kw*Cin), kpad channels per position, in the activation type
 cudaError_t launch_unfold(const ConvArgs& a, int n_rows, int kpad, void* out, cudaStream_t st);

@@ -91,23 +91,36 @@ __global__ void __launch_bounds__(256) conv_rows_kernel(ConvArgs a, long long in
         return;
     }
     const long long total = (long long)a.ring_rows * a.S * row_elems;
+    const int slot_of_first = (int)(a.o_begin % a.ring_rows);      // (one 64-bit division per thread instead of five)
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (long long)edge_blocks * blockDim.x) {
-        const int co = (int)(idx % a.Cout);
-        long long t = idx / a.Cout;
-        const int x = (int)(t % a.Wout);
-        t /= a.Wout;
-        const int s = (int)(t % a.S);
-        const int slot = (int)(t / a.S);
+        int co, x, s, slot;
+        if (total <= 0x7fffffffLL) {
+            unsigned t = (unsigned)idx;
+            co = (int)(t % (unsigned)a.Cout); t /= (unsigned)a.Cout;
+            x = (int)(t % (unsigned)a.Wout); t /= (unsigned)a.Wout;
+            s = (int)(t % (unsigned)a.S);
+            slot = (int)(t / (unsigned)a.S);
+        } else {
+            co = (int)(idx % a.Cout);
+            long long t = idx / a.Cout;
+            x = (int)(t % a.Wout);
+            t /= a.Wout;
+            s = (int)(t % a.S);
+            slot = (int)(t / a.S);
+        }
         const TS b = bias ? bias[co] : (TS)0;
         // first visited row that lives in this slot
-        long long o = a.o_begin + ((slot - a.o_begin % a.ring_rows) + a.ring_rows) % a.ring_rows;
+        long long o = a.o_begin + ((slot - slot_of_first) + a.ring_rows) % a.ring_rows;
         bool dirty = false;
         TS leave = 0;
         TS* rp = ring + ((long long)slot * a.S + s) * row_elems + (long long)x * a.Cout + co;
         if (!IDF_OK_AT(a.status, rp - ring, a.ring_elems)) continue;
         for (; o < a.o_end; o += a.ring_rows) {
-            if (o >= int_begin && o < int_end) continue;         // an interior row: another CTA's
+            if (o >= int_begin && o < int_end) {                 // interior rows are another CTA's: on to the slot's first row behind them
+                o += (long long)((unsigned)(int_end - 1 - o) / (unsigned)a.ring_rows) * a.ring_rows;      // (a block has far fewer than 2^32 rows)
+                continue;
+            }
             TS acc = 0;
             for (int ky = 0; ky < a.Kh; ++ky) {
                 const long long r = o * a.stride - a.pad + ky;
@@ -200,6 +213,28 @@ static cudaError_t launch_rows(const ConvArgs& a, cudaStream_t st)
     }
     conv_rows_kernel<TI, TW, TS, TO><<<(unsigned)(blocks + int_blocks), 256, 0, st>>>(a, int_begin, int_end, (unsigned)blocks);
     return cudaGetLastError();
+}
+
+template <typename TI, typename TW, typename TS, typename TO>
+static cudaError_t launch_edges_t(const ConvArgs& a, long long skip_begin, long long skip_end, cudaStream_t st)
+{
+    const long long total = (long long)a.ring_rows * a.S * a.Wout * a.Cout;
+    if (total == 0 || a.o_end <= a.o_begin) return cudaSuccess;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148LL * 64) blocks = 148LL * 64;
+    conv_rows_kernel<TI, TW, TS, TO><<<(unsigned)blocks, 256, 0, st>>>(a, skip_begin, skip_end, (unsigned)blocks);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_conv_edges(const ConvArgs& a, int dtype, long long skip_begin, long long skip_end, cudaStream_t st)
+{
+    if (dtype == 0) return launch_edges_t<float, float, float, float>(a, skip_begin, skip_end, st);
+    if (dtype == 1) {
+        if (a.in_elem != E_BF16) return cudaErrorInvalidValue;
+        if (a.out_elem == E_BF16) return launch_edges_t<__nv_bfloat16, float, float, __nv_bfloat16>(a, skip_begin, skip_end, st);
+        return launch_edges_t<__nv_bfloat16, float, float, float>(a, skip_begin, skip_end, st);
+    }
+    return launch_edges_t<int8_t, int8_t, int, int8_t>(a, skip_begin, skip_end, st);
 }
 
 cudaError_t launch_conv_simple(const ConvArgs& a, int dtype, cudaStream_t st)

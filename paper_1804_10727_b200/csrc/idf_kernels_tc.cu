@@ -975,6 +975,323 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Thin layers: the whole receptive field of an output position (Kh*Kw*Cin values) fits ONE swizzled
+// shared-memory row of 32, 64 or 128 bytes - the first layers of nets that start from few channels.
+// Such a layer is a plain contraction over that row (Eq. 4 for all taps of a unit at once), with so
+// little arithmetic per output that the kernel is bound by the bytes it writes; what matters is that
+// every role pays its fixed cost per BATCH of rows, not per row:
+//   warps 0-3   build the im2col rows of R output rows of one 128-position tile in shared memory,
+//               straight from the layer's input rows (zero where a tap falls on padding);
+//   warp 4      issues R x ksteps tcgen05.mma (M = 128, N = Cout) into one of two accumulator sets;
+//   warps 5-12  two epilogue groups taking work items in turn: tcgen05.ld, f(c + b), rounding or
+//               requantisation, swizzled staging tile, one TMA store per row.
+// The kernel handles only rows that this block's input rows determine completely (no ring row is read
+// or written: rows begun by an earlier block or left open by this one go through the CUDA-core kernel),
+// so rows are independent work items: item i = (row group, position tile), dealt round robin to a
+// grid of one CTA per SM.
+// ------------------------------------------------------------------------------------------------
+constexpr int THIN_THREADS = 13 * 32;
+constexpr int THIN_MAX_K = 128;              // bytes of an im2col row
+constexpr int THIN_RAW_PER_THREAD = 16;      // input values a gather thread copies per work item (128 threads)
+constexpr int THIN_RAW_BYTES = 128 * THIN_RAW_PER_THREAD * 2;
+
+struct ThinArgs {
+    const void* in;              // input rows of the block: [n_in][S][Win][Cin] in the activation type
+    const void* bias;
+    unsigned int* status;
+    long long r0;                // absolute index of the first input row of the block
+    long long o_first;           // absolute index of the first output row this launch computes
+    int n_in, n_out;             // input rows in the block, output rows to compute: o_first + [0, n_out)
+    int S, Win, Wout, Cin, Cout, Kh, Kw, stride, pad, stride_x, pad_x, relu, shift, out_elem;
+    int kelems, swb, ksteps, BX, BS, n_xt, n_mt, R, nstage, tmem_cols;
+    int out_esize, out_pwb, out_panels, out_tile_bytes;
+    int out_row_dim, out_row_first;          // position of the row coordinate in the output tensor map; map row of o_first
+};
+
+template <int DT>
+__global__ void __launch_bounds__(THIN_THREADS, 1)
+conv_thin_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmO, const ThinArgs a)
+{
+    typedef typename Acc<DT>::S TS;
+    constexpr int ES = DT == 1 ? 2 : 1;              // bytes of an activation
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+    __shared__ short s_tab[THIN_MAX_K][2];            // value k of an im2col row: where it comes from, where it goes
+
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t row_tile_bytes = 128u * (uint32_t)a.swb;               // one im2col tile (128 positions)
+    const uint32_t stage_bytes = (uint32_t)a.R * row_tile_bytes;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sW = base;                                              // [Cout][swb]
+    const uint32_t sA = (sW + (uint32_t)a.Cout * a.swb + 1023u) & ~1023u;
+    const uint32_t sOut = sA + (uint32_t)a.nstage * stage_bytes;           // [group][buffer][R] staging tiles
+    const uint32_t bars = sOut + 2u * 2u * (uint32_t)a.R * a.out_tile_bytes;
+    const uint32_t bar_full = bars, bar_empty = bar_full + 8u * a.nstage, bar_w = bar_empty + 8u * a.nstage;
+    const uint32_t bar_accfull = bar_w + 8u, bar_accfree = bar_accfull + 16u;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        for (int i = 0; i < a.nstage; ++i) { mbar_init(bar_full + 8u * i, 4); mbar_init(bar_empty + 8u * i, 1); }
+        mbar_init(bar_w, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(bar_accfull + 8u * i, 1); mbar_init(bar_accfree + 8u * i, 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_expect_tx(bar_w, (uint32_t)a.Cout * a.swb);                   // the parameters do not depend on earlier kernels
+        tma_load_2d(sW, &tmW, bar_w, 0, 0);
+    }
+    for (int k = threadIdx.x; k < a.kelems; k += blockDim.x) {
+        // value k of an im2col row: tap (ky, kx), channel ci -> its offset (in elements) from the position's corner in the
+        // staging area [row][stream][position][channel], and its byte position in the row
+        const int ci = k % a.Cin, t = k / a.Cin, ky = t / a.Kw, kx = t % a.Kw;
+        const int XP = (a.BX - 1) * a.stride_x + a.Kw;
+        s_tab[k][0] = (short)((ky * a.BS * XP + kx) * a.Cin + ci);
+        s_tab[k][1] = (short)(k * ES);
+    }
+    if (warp == 4) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)), "r"((uint32_t)a.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // the zero padding behind the kelems values of every im2col row is written once
+    for (uint32_t i = threadIdx.x; i < (uint32_t)a.nstage * stage_bytes / 16u; i += blockDim.x)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(sA + 16u * i), "r"(0u) : "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const uint32_t tmem_base = s_tmem_base;
+    volatile int* abort_flag = &s_abort;
+    const int n_groups = (a.n_out + a.R - 1) / a.R;
+    const long long n_items = (long long)n_groups * a.n_mt;
+
+    if (warp < 4) {
+        // ------------------------------ im2col rows ---------------------------------------------
+        // Two steps per work item.  (1) The 128 threads copy the input rows the item's R output rows reach - for the
+        // tile's streams and positions, with the kx halo, zero where a tap falls on padding - into a small staging
+        // area [row][stream][position][channel]: consecutive threads read consecutive elements, and the copy of the
+        // NEXT item is already in flight (in registers) while the current one is worked on.  (2) Thread m builds the
+        // im2col row of position m for each of the R output rows from that area: element k of a row sits at a fixed
+        // offset from the position's corner (table s_tab), so a value costs two additions, a load and a store.
+        const int m = warp * 32 + lane;                       // row of the tile = position
+        const int bs = m / a.BX, bx = m - bs * a.BX;
+        const bool in_tile = bs < a.BS;
+        const uint32_t sw_phase = a.swb == 128 ? (uint32_t)(m & 7) : (a.swb == 64 ? (uint32_t)((m >> 1) & 3) : (uint32_t)((m >> 2) & 1));
+        const unsigned char* in = (const unsigned char*)a.in;
+        const int XP = (a.BX - 1) * a.stride_x + a.Kw;        // positions of a stream in the staging area
+        const int run_s = XP * a.Cin, run_r = a.BS * run_s;   // elements per (row, stream) and per row
+        const int n_r = (a.R - 1) * a.stride + a.Kh;
+        const int raw_elems = n_r * run_r;
+        const uint32_t m_r = 0xFFFFFFFFu / (uint32_t)run_r + 1u, m_s = 0xFFFFFFFFu / (uint32_t)run_s + 1u,
+                       m_c = 0xFFFFFFFFu / (uint32_t)a.Cin + 1u;        // q = umulhi(n, m): n / d for the small n here
+        const uint32_t corner = (uint32_t)((bs * XP + bx * a.stride_x) * a.Cin) * ES;
+        const uint32_t sRaw = bars + 256u;                    // behind the barriers
+        unsigned short held[THIN_RAW_PER_THREAD];             // the next item's share of the staging area
+        auto fetch = [&](long long item) {
+            const int g = (int)(item / a.n_mt), mt = (int)(item - (long long)g * a.n_mt);
+            const int xt = mt % a.n_xt, st = mt / a.n_xt;
+            const long long r_first = (a.o_first + (long long)g * a.R) * a.stride - a.pad - a.r0;     // row of the block
+            const int x_first = xt * a.BX * a.stride_x - a.pad_x;
+#pragma unroll
+            for (int i = 0; i < THIN_RAW_PER_THREAD; ++i) {
+                const uint32_t e = (uint32_t)(m + 128 * i);
+                unsigned short v = 0;
+                if (e < (uint32_t)raw_elems) {
+                    const uint32_t rr = __umulhi(e, m_r), e1 = e - rr * (uint32_t)run_r;
+                    const uint32_t ss = __umulhi(e1, m_s), e2 = e1 - ss * (uint32_t)run_s;
+                    const uint32_t xp = __umulhi(e2, m_c), ci = e2 - xp * (uint32_t)a.Cin;
+                    const long long r = r_first + rr;
+                    const int sg = st * a.BS + (int)ss, ix = x_first + (int)xp;
+                    if (r >= 0 && r < a.n_in && sg < a.S && ix >= 0 && ix < a.Win) {
+                        const long long at = ((r * a.S + sg) * a.Win + ix) * (long long)a.Cin + ci;
+                        if (IDF_OK_AT(a.status, at, (long long)a.n_in * a.S * a.Win * a.Cin))
+                            v = ES == 2 ? *(const unsigned short*)(in + 2 * at) : (unsigned short)in[at];
+                    }
+                }
+                held[i] = v;
+            }
+        };
+        int it = 0;
+        bool ok = true;
+        if ((long long)blockIdx.x < n_items) fetch(blockIdx.x);
+        for (long long item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
+            const int stage = it % a.nstage;
+            const uint32_t ph = (uint32_t)((it / a.nstage) & 1);
+            const int g = (int)(item / a.n_mt), mt = (int)(item - (long long)g * a.n_mt);
+            const int xt = mt % a.n_xt, st = mt / a.n_xt;
+            const bool valid = in_tile && st * a.BS + bs < a.S && xt * a.BX + bx < a.Wout;
+#pragma unroll
+            for (int i = 0; i < THIN_RAW_PER_THREAD; ++i) {
+                const uint32_t e = (uint32_t)(m + 128 * i);
+                if (e < (uint32_t)raw_elems) {
+                    if (ES == 2) asm volatile("st.shared.u16 [%0], %1;" ::"r"(sRaw + 2u * e), "h"(held[i]) : "memory");
+                    else asm volatile("st.shared.u8 [%0], %1;" ::"r"(sRaw + e), "r"((uint32_t)held[i]) : "memory");
+                }
+            }
+            named_bar_sync(3, 128);                               // the staging area is complete
+            if (item + gridDim.x < n_items) fetch(item + gridDim.x);
+            int got = 1;
+            if (lane == 0) got = mbar_wait_relaxed(bar_empty + 8u * stage, ph ^ 1u, abort_flag) ? 1 : 0;
+            got = __shfl_sync(0xffffffffu, got, 0);
+            if (got && valid) {
+                for (int j = 0; j < a.R; ++j) {
+                    if (g * a.R + j >= a.n_out) break;
+                    const uint32_t row_addr = sA + (uint32_t)stage * stage_bytes + (uint32_t)j * row_tile_bytes + (uint32_t)m * a.swb;
+                    const uint32_t from = sRaw + corner + (uint32_t)(j * a.stride * run_r) * ES;
+                    // eight values at a time: the loads of a batch are all issued before the first store needs its value
+                    for (int k0 = 0; k0 < a.kelems; k0 += 8) {
+                        uint32_t v[8], dst[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const int k = k0 + u < a.kelems ? k0 + u : a.kelems - 1;      // (the tail repeats the last value: same bytes, same place)
+                            const uint32_t off = (uint32_t)(unsigned short)s_tab[k][0] * ES, to = (uint32_t)(unsigned short)s_tab[k][1];
+                            dst[u] = row_addr + ((((to >> 4) ^ sw_phase)) << 4) + (to & 15u);
+                            if (ES == 2) { unsigned short h; asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(from + off)); v[u] = h; }
+                            else asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v[u]) : "r"(from + off));
+                        }
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            if (ES == 2) asm volatile("st.shared.u16 [%0], %1;" ::"r"(dst[u]), "h"((unsigned short)v[u]));
+                            else asm volatile("st.shared.u8 [%0], %1;" ::"r"(dst[u]), "r"(v[u]));
+                        }
+                    }
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the tensor core reads these rows through the async proxy
+            // nobody reads the staging area any more; and if any warp's wait ran out, all four leave together
+            if (!named_bar_and(3, 128, got != 0)) { ok = false; break; }
+            if (lane == 0) mbar_arrive(bar_full + 8u * stage);
+        }
+    } else if (warp == 4) {
+        // ------------------------------ MMA issuer ---------------------------------------------
+        const uint64_t desc_hi = make_smem_desc(0, a.swb);
+        const uint32_t idesc = (DT == 1 ? ((1u << 4) | (1u << 7) | (1u << 10)) : ((2u << 4) | (1u << 7) | (1u << 10))) |
+                               ((128u >> 4) << 24) | ((uint32_t)(a.Cout >> 3) << 17);
+        const uint64_t bdesc = desc_hi | (uint64_t)((sW & 0x3FFFFu) >> 4);
+        bool ok = mbar_wait(bar_w, 0, abort_flag);
+        const bool issuer = elect_one();
+        int it = 0;
+        for (long long item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
+            const int stage = it % a.nstage;
+            const uint32_t ph = (uint32_t)((it / a.nstage) & 1);
+            const int acc = it & 1;
+            const uint32_t aph = (uint32_t)((it >> 1) & 1);
+            if (!mbar_wait(bar_accfree + 8u * acc, aph ^ 1u, abort_flag)) { ok = false; break; }   // the epilogue has read this accumulator set
+            if (!mbar_wait(bar_full + 8u * stage, ph, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            if (issuer) {
+                for (int j = 0; j < a.R; ++j) {
+                    const uint64_t adesc = desc_hi | (uint64_t)(((sA + (uint32_t)stage * stage_bytes + (uint32_t)j * row_tile_bytes) & 0x3FFFFu) >> 4);
+                    const uint32_t d = tmem_base + (uint32_t)((acc * a.R + j) * a.Cout);
+                    for (int k = 0; k < a.ksteps; ++k) umma<DT>(d, adesc + 2u * k, bdesc + 2u * k, idesc, k > 0 ? 1u : 0u);
+                }
+                umma_commit(bar_empty + 8u * stage);
+                umma_commit(bar_accfull + 8u * acc);
+            }
+            __syncwarp();
+        }
+    } else {
+        // ------------------------------ epilogue -----------------------------------------------
+        const int q = warp & 3;                           // TMEM lane quarter this warp may read
+        const int grp = (warp - 5) >> 2;
+        const bool leader = (warp - 5) == grp * 4 && lane == 0;
+        const int m = q * 32 + lane;
+        const int bs = m / a.BX, bx = m - bs * a.BX;
+        const bool in_tile = bs < a.BS;
+        const TS* bias = (const TS*)a.bias;
+        const uint32_t tlane = tmem_base + ((uint32_t)(q * 32) << 16);
+        StageSink sink;
+        sink.pwb_log2 = 31u - (uint32_t)__clz(a.out_pwb);
+        sink.panel_bytes = 128u * (uint32_t)a.out_pwb;
+        const int md = bs * a.BX + bx;
+        sink.phase = a.out_pwb == 128 ? (uint32_t)(md & 7) : (a.out_pwb == 64 ? (uint32_t)((md >> 1) & 3)
+                   : (a.out_pwb == 32 ? (uint32_t)((md >> 2) & 1) : 0u));
+        PoolCtx pc;
+        pc.on = 0; pc.writer = 0; pc.second = 0; pc.from_state = 0; pc.to_state = 0; pc.drop = 0; pc.sink = sink; pc.state = nullptr;
+        const int panel_cols = a.out_pwb / a.out_esize;
+        const uint32_t grp_base = sOut + (uint32_t)grp * 2u * (uint32_t)a.R * a.out_tile_bytes;
+        int buf = 0;
+        bool ok = true;
+        int it = 0;
+        for (long long item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
+            if ((it & 1) != grp) continue;
+            const uint32_t aph = (uint32_t)((it >> 1) & 1);
+            const int g = (int)(item / a.n_mt), mt = (int)(item - (long long)g * a.n_mt);
+            const int xt = mt % a.n_xt, st = mt / a.n_xt;
+            int got = 1;
+            if (leader) {
+                asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");     // the tiles of the store before last are free again
+                got = mbar_wait_relaxed(bar_accfull + 8u * grp, aph, abort_flag) ? 1 : 0;
+            }
+            if (!named_bar_and(1 + grp, 128, got != 0)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t tiles = grp_base + (uint32_t)buf * (uint32_t)a.R * a.out_tile_bytes;
+            for (int j = 0; j < a.R; ++j) {
+                if (g * a.R + j >= a.n_out) break;
+                sink.row_base = tiles + (uint32_t)j * a.out_tile_bytes + (uint32_t)md * a.out_pwb;
+                const bool fine = IDF_OK_AT(a.status, (sink.row_base - smem_u32(smem_raw)) + (uint32_t)(a.out_panels - 1) * sink.panel_bytes + a.out_pwb - 1,
+                                            bars - smem_u32(smem_raw));
+                const uint32_t trow = tlane + (uint32_t)((grp * a.R + j) * a.Cout);
+                if ((a.Cout & 31) == 0) {
+                    for (int c = 0; c < a.Cout; c += 32) {
+                        uint32_t v[32];
+                        tmem_ld<32>(trow + c, v);
+                        tmem_ld_wait();
+                        if (in_tile && fine)
+                            finalise_chunk<DT, 32, TS>(v, false, true, (TS*)nullptr, bias ? bias + c : nullptr, sink, (uint32_t)(c * a.out_esize),
+                                                       a.out_elem, a.relu, a.shift, pc, false, 0);
+                    }
+                } else {
+                    for (int c = 0; c < a.Cout; c += 16) {
+                        uint32_t v[16];
+                        tmem_ld<16>(trow + c, v);
+                        tmem_ld_wait();
+                        if (in_tile && fine)
+                            finalise_chunk<DT, 16, TS>(v, false, true, (TS*)nullptr, bias ? bias + c : nullptr, sink, (uint32_t)(c * a.out_esize),
+                                                       a.out_elem, a.relu, a.shift, pc, false, 0);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_accfree + 8u * grp);           // one arrival per warp: the accumulator set may be overwritten
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            named_bar_sync(1 + grp, 128);
+            if (leader) {
+                for (int j = 0; j < a.R; ++j) {
+                    const int orel = g * a.R + j;
+                    if (orel >= a.n_out) break;
+                    const uint32_t tile = tiles + (uint32_t)j * a.out_tile_bytes;
+                    for (int pnl = 0; pnl < a.out_panels; ++pnl) {
+                        if (a.out_row_dim == 3)
+                            tma_store_4d(&tmO, tile + (uint32_t)pnl * sink.panel_bytes, pnl * panel_cols, xt * a.BX, st * a.BS, a.out_row_first + orel);
+                        else
+                            tma_store_4d(&tmO, tile + (uint32_t)pnl * sink.panel_bytes, pnl * panel_cols, xt * a.BX, a.out_row_first + orel, st * a.BS);
+                    }
+                }
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
+            buf ^= 1;
+        }
+        if (leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (s_abort) {
+        if (threadIdx.x == 0) {
+            for (uint32_t i = 0; i < 4096 && !mbar_try_wait(bar_w, 0); ++i) __nanosleep(64);   // the CTA's own copy must land first
+            atomicOr(a.status, 1u);
+        }
+        __syncthreads();
+    }
+    if (warp == 4) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)a.tmem_cols) : "memory");
+    }
+}
+
 // ---- host side ---------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -1243,6 +1560,132 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     const bool use_pdl = (debug_flags() & IDF_DEBUG_NO_PDL) == 0;
     cfg.attrs = attr; cfg.numAttrs = use_pdl ? 1 : 0;
     cudaError_t le = cudaLaunchKernelEx(&cfg, fn, tmA, *(const CUtensorMap*)w_map, tmO, t);
+    if (le != cudaSuccess) return le;
+    return cudaGetLastError();
+}
+
+
+// ---- thin layers: host side ----------------------------------------------------------------------
+bool thin_make_plan(int dtype, int S, int Wout, int Cin, int Cout, int Kh, int Kw, int stride, int stride_x, int out_esize, ThinPlan* p)
+{
+    *p = ThinPlan{};
+    if (dtype != 1 && dtype != 2) return false;
+    const int esize = dtype == 1 ? 2 : 1;
+    const int kbytes = Kh * Kw * Cin * esize;
+    if (kbytes > THIN_MAX_K || Cout % 16 != 0 || Cout > 256 || Kh * Kw * Cin > THIN_MAX_K) return false;
+    p->swb = kbytes <= 32 ? 32 : (kbytes <= 64 ? 64 : 128);
+    p->kelems = Kh * Kw * Cin;
+    p->ksteps = p->swb / 32;
+    if (Wout >= 128) {
+        p->n_xt = (Wout + 127) / 128;
+        p->BX = (Wout + p->n_xt - 1) / p->n_xt;
+        p->BS = 1;
+    } else {
+        p->n_xt = 1;
+        p->BX = Wout;
+        p->BS = 128 / Wout;
+        if (p->BS > S) p->BS = S;
+    }
+    p->n_mt = p->n_xt * ((S + p->BS - 1) / p->BS);
+    p->out_esize = out_esize;
+    p->out_pwb = Cout * out_esize >= 128 ? 128 : Cout * out_esize;
+    p->out_panels = Cout * out_esize / p->out_pwb;
+    p->out_tile_bytes = p->out_panels * 128 * p->out_pwb;
+    // rows per work item: as many as two accumulator sets in tensor memory and two staging sets per group allow
+    const size_t wb = ((size_t)Cout * p->swb + 1023) / 1024 * 1024;
+    int R = 256 / Cout;
+    if (R > 4) R = 4;
+    for (; R >= 1; --R) {
+        const size_t need = 2048 + wb + 3 * (size_t)R * 128 * p->swb + 4 * (size_t)R * p->out_tile_bytes + 512 + THIN_RAW_BYTES + 4096;
+        // the input values behind the item's rows (with the kx halo) must fit the staging area
+        const long long raw = (long long)((R - 1) * stride + Kh) * p->BS * ((p->BX - 1) * stride_x + Kw) * Cin;
+        if (need <= SMEM_LIMIT && raw <= 128 * THIN_RAW_PER_THREAD && raw * 4 < 32767) break;
+    }
+    if (R < 1) return false;
+    p->R = R;
+    p->nstage = 3;
+    int cols = 32;
+    while (cols < 2 * R * Cout) cols <<= 1;
+    if (cols > 512) return false;
+    p->tmem_cols = cols;
+    p->smem_bytes = 1024 + wb + (size_t)p->nstage * R * 128 * p->swb + 4 * (size_t)R * p->out_tile_bytes + 256 + THIN_RAW_BYTES + 64;
+    p->w_bytes = (size_t)Cout * p->swb;
+    p->ok = 1;
+    return true;
+}
+
+int thin_encode_weights(const ThinPlan& p, int dtype, const void* d_w, int Cout, void* map_out)
+{
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return -1;
+    const int esize = dtype == 1 ? 2 : 1;
+    cuuint64_t dims[2] = {(cuuint64_t)(p.swb / esize), (cuuint64_t)Cout};
+    cuuint64_t strides[1] = {(cuuint64_t)p.swb};
+    cuuint32_t box[2] = {(cuuint32_t)(p.swb / esize), (cuuint32_t)Cout};
+    cuuint32_t es[2] = {1, 1};
+    CUresult r = enc((CUtensorMap*)map_out, dtype == 1 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
+                     const_cast<void*>(d_w), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(p.swb),
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : -1;
+}
+
+// Output rows [o_first, o_end) of the layer, each determined completely by the block's input rows a.in (rows
+// a.r0 .. a.r1-1; taps outside them fall on zero padding).  cudaErrorNotSupported: use another kernel.
+cudaError_t launch_conv_thin(const ConvArgs& a, const ThinPlan& p, int dtype, const void* w_map, long long o_first, long long o_end,
+                             unsigned int* status, cudaStream_t st)
+{
+    EncodeTiledFn enc = encode_fn();
+    if (!enc || !p.ok || o_end <= o_first) return cudaErrorNotSupported;
+    if (((uintptr_t)a.out & 15) != 0 || a.out_rows_extent < 1 || a.pool_fused) return cudaErrorNotSupported;
+    CUtensorMap tmO;
+    const int row_dim = a.out_row_stride > a.out_stream_stride ? 3 : 2;
+    {
+        const int oes = p.out_esize;
+        cuuint64_t od[4] = {(cuuint64_t)a.Cout, (cuuint64_t)a.Wout, 0, 0};
+        cuuint64_t os[3] = {(cuuint64_t)a.Cout * oes, 0, 0};
+        cuuint32_t ob[4] = {(cuuint32_t)(p.out_pwb / oes), (cuuint32_t)p.BX, 1, 1};
+        cuuint32_t es[4] = {1, 1, 1, 1};
+        od[row_dim] = (cuuint64_t)a.out_rows_extent; od[5 - row_dim] = (cuuint64_t)a.S;
+        os[row_dim - 1] = (cuuint64_t)a.out_row_stride * oes; os[4 - row_dim] = (cuuint64_t)a.out_stream_stride * oes;
+        ob[5 - row_dim] = (cuuint32_t)p.BS;
+        const CUtensorMapDataType odt = a.out_elem == E_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                      : (a.out_elem == E_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
+        const CUtensorMapSwizzle osw = p.out_pwb == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                     : (p.out_pwb == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                     : (p.out_pwb == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE));
+        if (enc(&tmO, odt, 4, a.out, od, os, ob, es, CU_TENSOR_MAP_INTERLEAVE_NONE, osw, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorNotSupported;
+    }
+    ThinArgs t{};
+    t.in = a.in; t.bias = a.bias; t.status = status;
+    t.r0 = a.r0; t.o_first = o_first; t.n_in = (int)(a.r1 - a.r0); t.n_out = (int)(o_end - o_first);
+    t.S = a.S; t.Win = a.Win; t.Wout = a.Wout; t.Cin = a.Cin; t.Cout = a.Cout; t.Kh = a.Kh; t.Kw = a.Kw;
+    t.stride = a.stride; t.pad = a.pad; t.stride_x = a.stride_x; t.pad_x = a.pad_x; t.relu = a.relu; t.shift = a.shift;
+    t.out_elem = a.out_elem;
+    t.kelems = p.kelems; t.swb = p.swb; t.ksteps = p.ksteps; t.BX = p.BX; t.BS = p.BS; t.n_xt = p.n_xt; t.n_mt = p.n_mt;
+    t.R = p.R; t.nstage = p.nstage; t.tmem_cols = p.tmem_cols;
+    t.out_esize = p.out_esize; t.out_pwb = p.out_pwb; t.out_panels = p.out_panels; t.out_tile_bytes = p.out_tile_bytes;
+    t.out_row_dim = row_dim; t.out_row_first = (int)(o_first - a.out_row_base);
+    const long long n_items = (long long)((t.n_out + p.R - 1) / p.R) * p.n_mt;
+    const unsigned grid = (unsigned)(n_items < 148 ? n_items : 148);
+    typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const ThinArgs);
+    const KernelFn fn = dtype == 1 ? (KernelFn)conv_thin_kernel<1> : (KernelFn)conv_thin_kernel<2>;
+    static bool attr_set[2][64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dtype - 1][dev]) {
+        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_LIMIT - 6144));
+        if (e != cudaSuccess) return e;
+        attr_set[dtype - 1][dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(THIN_THREADS); cfg.dynamicSmemBytes = p.smem_bytes; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = (debug_flags() & IDF_DEBUG_NO_PDL) ? 0 : 1;
+    cudaError_t le = cudaLaunchKernelEx(&cfg, fn, *(const CUtensorMap*)w_map, tmO, t);
     if (le != cudaSuccess) return le;
     return cudaGetLastError();
 }

@@ -38,7 +38,7 @@ EXPORTS = (
     "idf_launch_count", "idf_stream_status", "idf_set_timing", "idf_layer_times", "idf_conv_rows_noalloc", "idf_last_error",
     "idf_state_snapshot_bytes", "idf_state_save", "idf_state_restore", "idf_stream_set_out_base", "idf_set_debug_flags", "idf_out_rows_needed",
 )
-DEBUG_NO_TENSOR_CORES, DEBUG_NO_POOL_FUSION, DEBUG_NO_ROW_CHUNKS, DEBUG_NO_PDL = 1, 2, 4, 8
+DEBUG_NO_TENSOR_CORES, DEBUG_NO_POOL_FUSION, DEBUG_NO_ROW_CHUNKS, DEBUG_NO_PDL, DEBUG_PREFER_THIN = 1, 2, 4, 8, 16
 
 
 class IdfLayer(ctypes.Structure):

@@ -188,3 +188,46 @@ def test_row_chunks_match_oracle(orc, debug_flags, name, mode, layers, H, W, S):
         debug_flags(idf.DEBUG_NO_ROW_CHUNKS)
         net = idf.Net(mode, layers, W, layers[0].cin, S, ws, bs)
         assert_equal(idf.infer(net, x, last=True), want, name + "/unchunked")
+
+
+# ---- thin layers: the whole receptive field in one shared-memory row, a kernel of its own ------------------------
+THIN_CASES = [
+    # (name, mode, layers, H, W, S)
+    ("bf16_rgb_3x3_same", "bf16", (conv(3, 64, 3, pad=1), conv(64, 16, 3, pad=1)), 30, 40, 5),
+    ("i8_rgb_3x3_valid", "i8", (conv(3, 32, 3, path=1), conv(32, 32, 3, pad=1)), 26, 37, 4),
+    ("bf16_1d_k9_stride2", "bf16", (conv(1, 32, 9, stride=2, one_d=True), conv(32, 32, 9, one_d=True)), 300, 1, 200),
+    ("i8_1d_k9", "i8", (conv(2, 16, 9, one_d=True, path=1),), 120, 1, 70),                   # 16 channels: 16-column chunks
+    ("bf16_wide_three_x_tiles", "bf16", (conv(2, 32, 3, pad=1),), 12, 300, 2),
+    ("i8_many_channels", "i8", (conv(4, 256, 3, pad=1, path=1), conv(256, 16, 1)), 14, 20, 3),   # one row per work item
+    ("i8_5x5_stride2", "i8", (conv(4, 32, 5, stride=2, pad=2, path=1), conv(32, 16, 3)), 41, 30, 3),   # 100-byte rows
+    ("bf16_last_layer_fp32", "bf16", (conv(3, 32, 3, pad=1),), 20, 24, 6),
+]
+
+
+@pytest.mark.parametrize("name,mode,layers,H,W,S", THIN_CASES, ids=[c[0] for c in THIN_CASES])
+def test_thin_layers_match_oracle(orc, debug_flags, name, mode, layers, H, W, S):
+    debug_flags(idf.DEBUG_PREFER_THIN)          # (2D layers take x-unfold + row ring by default; here every case runs the thin kernel)
+    if mode == "i8":
+        layers = with_shifts(layers, 8)
+    x, ws, bs = rand_net(mode, layers, H, W, layers[0].cin, S=S, seed=7 + len(name))
+    want = orc.forward(mode, layers, x, ws, bs)
+    n_conv = sum(l.kind == "conv" for l in layers)
+    # whole streams at once, blocks that begin / continue / end streams (rows carried through the ring at both ends of
+    # a block), row by row (no row is determined by one block alone: the ring kernel takes everything)
+    for chunks, rb, last in ((None, 0, True), (None, 0, False), ([H // 2 + 1], 0, True), ([7, 9, 5], 8, False), ([1] * min(H, 30), 0, True)):
+        got, tc = _run(mode, layers, x, ws, bs, chunks=chunks, row_block=rb) if not last else (None, None)
+        if last:
+            net = idf.Net(mode, layers, W, layers[0].cin, S, ws, bs, row_block=rb)
+            got = idf.infer(net, x, chunks=chunks, last=True)
+            tc = net.status()
+        what = f"{name}/chunks={chunks}/rb={rb}/last={last}"
+        if chunks is None:
+            assert tc[0] > 0, f"{what}: the first layer did not take a tensor-core kernel: {tc}"
+        if mode == "i8":
+            assert_equal(got, want, what)
+        elif n_conv == 1:
+            assert_close(got, want, what)
+        else:
+            err = np.abs(got - want)
+            ok = err <= 1e-4 + 1e-3 * np.abs(want)
+            assert ok.mean() > 0.97 and err.max() < 0.05, (what, ok.mean(), err.max())
