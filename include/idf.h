@@ -319,15 +319,17 @@ int idf_conv_rows_noalloc(const float* d_in, int n_rows, int n_streams, int in_w
  * the paths with one another; results are the same with any combination (bit-exact for int nets), only the
  * kernels and launch counts differ.  Not for production use; the paper has no counterpart.  flags is a
  * combination of the bits below (0 = defaults); IDF_DEBUG_NO_TENSOR_CORES, IDF_DEBUG_NO_POOL_FUSION and
- * IDF_DEBUG_PREFER_THIN are read by idf_net_create (they affect nets created afterwards), the other two at every launch.
+ * IDF_DEBUG_PREFER_THIN are read by idf_net_create (they affect nets created afterwards), the others at every push or launch.
  * IDF_ERR_ARG for an unknown bit (nothing changes). */
 typedef enum {
     IDF_DEBUG_NO_TENSOR_CORES = 1,  /* dense layers stay on the CUDA-core kernel                              */
     IDF_DEBUG_NO_POOL_FUSION = 2,   /* max-pool layers run as launches of their own                           */
     IDF_DEBUG_NO_ROW_CHUNKS = 4,    /* a block's rows stay in one CTA per tile                                */
     IDF_DEBUG_NO_PDL = 8,           /* no programmatic dependent launch                                       */
-    IDF_DEBUG_PREFER_THIN = 16      /* thin layers (receptive field of at most 128 bytes) take the thin-layer */
+    IDF_DEBUG_PREFER_THIN = 16,     /* thin layers (receptive field of at most 128 bytes) take the thin-layer */
                                     /* kernel also where x-unfold + row ring is the default (2D nets)          */
+    IDF_DEBUG_NO_FUSED = 32,        /* never the single launch over all layers (state in shared memory)       */
+    IDF_DEBUG_FORCE_FUSED = 64      /* ... always, where a stream's state fits (by default: small pushes only) */
 } idf_debug_flag;
 int idf_set_debug_flags(unsigned int flags);
 

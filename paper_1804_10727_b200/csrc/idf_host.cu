@@ -80,6 +80,11 @@ enum Phase { CREATED = 0, OPEN = 1, FINISHED = 2 };
 
 struct idf_net {
     int dtype = 0, in_w = 0, in_c = 0, n_streams = 0, row_block = 0;
+    // depth-first over all layers in one launch (nets whose per-stream state is small): plan made at create
+    int fused_ok = 0, fused_G = 0, fused_threads = 0, fused_in_soff = 0;
+    size_t fused_smem = 0;
+    std::vector<int> fused_state_soff, fused_rowbuf_soff;
+    double macs_per_row = 0;               // multiply-accumulates one segment of one stream costs (all layers, steady state)
     int eager = 0;                         // emission policy: 0 = once per unit (deferred), 1 = after every segment (eager)
     size_t eager_in_off = 0;               // the pushed segment as words (the input layer's announcement)
     std::vector<LayerPlan> L;
@@ -384,6 +389,8 @@ int fire(idf_net* net, size_t i, const void* in_ptr, long long n_in, bool flush,
          long long* emitted);
 int run_segments_eager(idf_net* net, const void* d_segments, long long n_seg, bool flush, void* d_out, long long out_cap,
                        long long* emitted);
+int run_segments_fused(idf_net* net, const void* d_segments, long long n_seg, bool flush, void* d_out, long long out_cap,
+                       long long* emitted);
 
 int ensure_space(idf_net* net, size_t m, long long need, void* d_out, long long out_cap, long long* emitted)
 {
@@ -447,6 +454,12 @@ int run_segments(idf_net* net, const void* d_segments, long long n_seg, bool flu
 {
     const size_t nl = net->L.size();
     if (net->eager) return run_segments_eager(net, d_segments, n_seg, flush, d_out, out_cap, emitted);
+    if (net->fused_ok && !(debug_flags() & IDF_DEBUG_NO_FUSED) && n_seg <= 65535) {
+        // pushes that the per-layer kernels could only answer with a handful of nearly empty launches take the single
+        // launch that keeps the state on chip: few segments, or little arithmetic altogether
+        const bool small = n_seg <= 2 || net->macs_per_row * (double)n_seg * net->n_streams < 5e7;
+        if (small || (debug_flags() & IDF_DEBUG_FORCE_FUSED)) return run_segments_fused(net, d_segments, n_seg, flush, d_out, out_cap, emitted);
+    }
     // capacity of the caller's output first: the rows complete after this call do not depend on the schedule
     {
         long long r = net->L[0].rows_in + n_seg;
@@ -635,6 +648,58 @@ int run_segments_eager(idf_net* net, const void* d_segments, long long n_seg, bo
 }  // namespace
 
 namespace {
+
+// One launch for the whole push: every segment through every layer, state in shared memory (depth_first_kernel).
+int run_segments_fused(idf_net* net, const void* d_segments, long long n_seg, bool flush, void* d_out, long long out_cap,
+                       long long* emitted)
+{
+    const size_t nl = net->L.size();
+    // rows complete after this call, layer by layer (the schedule inside the kernel follows the same closed forms)
+    std::vector<long long> in_after(nl), done_after(nl);
+    long long r = net->L[0].rows_in + n_seg;
+    for (size_t i = 0; i < nl; ++i) {
+        in_after[i] = r;
+        r = flush ? layer_rows_at_flush(net->L[i], r) : layer_done_after(net->L[i], r);
+        r = std::max(r, net->L[i].rows_done);
+        done_after[i] = r;
+    }
+    if (r - net->out_base > out_cap)
+        return fail(IDF_ERR_CAPACITY, "output row %lld does not fit out_capacity_rows=%lld", r - 1, out_cap);
+    if (n_seg == 0 && !flush) return IDF_OK;
+    FusedArgs a{};
+    a.n_layers = (int)nl; a.S = net->n_streams; a.G = net->fused_G;
+    a.in = d_segments; a.n_seg = (int)n_seg; a.in_w = net->in_w; a.in_c = net->in_c; a.in_elem = net->L[0].in_elem;
+    a.in_soff = net->fused_in_soff; a.flush = flush ? 1 : 0;
+    a.weights = net->ws;
+    a.out = d_out; a.out_cap = out_cap; a.out_base = net->out_base; a.out_elem = net->L.back().out_elem;
+    a.counters = (unsigned long long*)(net->ws + net->counters_off);
+    a.status = (unsigned int*)(net->ws + net->status_off);
+    for (size_t i = 0; i < nl; ++i) {
+        const LayerPlan& P = net->L[i];
+        FusedLayer& F = a.layer[i];
+        F.kind = P.l.kind == IDF_CONV ? 0 : 1;
+        F.Cin = P.in_c; F.Cout = P.out_c; F.Kh = P.l.kh; F.Kw = P.l.kw; F.stride = P.l.stride; F.pad = P.l.pad;
+        F.stride_x = P.in_w == 1 ? 1 : P.l.stride; F.pad_x = P.in_w == 1 ? 0 : P.l.pad;
+        F.relu = P.l.relu; F.shift = P.l.shift; F.round_bf16 = P.out_elem == E_BF16;
+        F.Win = P.in_w; F.Wout = P.out_w; F.ring_rows = P.ring_rows; F.count_events = P.use_sparse; F.out_elem = P.out_elem;
+        F.state_soff = net->fused_state_soff[i]; F.rowbuf_soff = net->fused_rowbuf_soff[i];
+        F.w_off = (long long)(net->dtype == IDF_I8_I32 ? P.w_off : P.w_off / 4);
+        F.bias_off = P.b_packed.empty() ? -1 : (long long)P.b_off;
+        F.state = net->ws + P.state_off;
+        F.rows_in = P.rows_in; F.rows_done = P.rows_done;
+    }
+    cudaError_t ce = launch_depth_first(a, net->dtype == IDF_I8_I32, net->fused_threads, net->fused_smem, net->stream);
+    if (ce != cudaSuccess) { net->phase = FINISHED; return fail(IDF_ERR_CUDA, "kernel launch failed (all layers in one): %s", cudaGetErrorString(ce)); }
+    net->launches += 1;
+    const long long before = net->L.back().rows_done;
+    for (size_t i = 0; i < nl; ++i) { net->L[i].rows_in = in_after[i]; net->L[i].rows_done = done_after[i]; net->L[i].pending = 0; }
+    *emitted += net->L.back().rows_done - before;
+    return IDF_OK;
+}
+
+}  // namespace
+
+namespace {
 std::atomic<unsigned> g_debug_flags{0};
 }
 namespace idf {
@@ -648,7 +713,7 @@ const char* idf_last_error(void) { return g_err.c_str(); }
 
 int idf_set_debug_flags(unsigned int flags)
 {
-    if (flags & ~(unsigned)(IDF_DEBUG_NO_TENSOR_CORES | IDF_DEBUG_NO_POOL_FUSION | IDF_DEBUG_NO_ROW_CHUNKS | IDF_DEBUG_NO_PDL | IDF_DEBUG_PREFER_THIN))
+    if (flags & ~(unsigned)(IDF_DEBUG_NO_TENSOR_CORES | IDF_DEBUG_NO_POOL_FUSION | IDF_DEBUG_NO_ROW_CHUNKS | IDF_DEBUG_NO_PDL | IDF_DEBUG_PREFER_THIN | IDF_DEBUG_NO_FUSED | IDF_DEBUG_FORCE_FUSED))
         return fail(IDF_ERR_ARG, "unknown debug flag in 0x%x", flags);
     g_debug_flags.store(flags, std::memory_order_relaxed);
     return IDF_OK;
@@ -852,6 +917,41 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
             LayerPlan& P = net->L[i];
             P.fuse_pool = P.l.kind == IDF_CONV && net->L[i + 1].l.kind == IDF_MAXPOOL2 && P.tc.ok && P.tc_pool.ok && !P.use_sparse &&
                           P.out_w >= 2 && (P.tc_pool.BX % 2) == 0 && !no_fuse && !net->eager;
+        }
+    }
+    // one launch for all layers, state in shared memory: possible when a stream's rings, pooling rows and one row per
+    // layer boundary are small enough for at least one stream per CTA
+    if (!net->eager && (int)net->L.size() <= FUSED_MAX_LAYERS) {
+        bool ok = true;
+        size_t words = (size_t)net->in_w * net->in_c;
+        double macs = 0, rate = 1;
+        for (const auto& P : net->L) {
+            if (P.l.kind == IDF_GLOBAL_AVG) { ok = false; break; }
+            words += (size_t)(P.l.kind == IDF_CONV ? P.ring_rows : 1) * P.out_w * P.out_c + (size_t)P.out_w * P.out_c;
+            if (P.l.kind == IDF_CONV) { rate /= P.l.stride; macs += rate * P.out_w * P.out_c * (double)P.l.kh * P.l.kw * P.l.cin; }
+            else rate /= 2;
+        }
+        net->macs_per_row = macs;
+        const size_t per_stream = words * 4;
+        if (ok && per_stream <= FUSED_SMEM_LIMIT) {
+            int G = (int)std::min<size_t>(FUSED_SMEM_LIMIT / per_stream, 32);
+            G = std::min(G, net->n_streams);
+            // (enough CTAs for the SMs before more streams per CTA)
+            while (G > 1 && (net->n_streams + G - 1) / G < 148) --G;
+            net->fused_G = G;
+            size_t off = 0;
+            net->fused_in_soff = 0; off += (size_t)G * net->in_w * net->in_c;
+            size_t widest = (size_t)G * net->in_w * net->in_c;
+            for (const auto& P : net->L) {
+                net->fused_state_soff.push_back((int)off);
+                off += (size_t)(P.l.kind == IDF_CONV ? P.ring_rows : 1) * G * P.out_w * P.out_c;
+                net->fused_rowbuf_soff.push_back((int)off);
+                off += (size_t)G * P.out_w * P.out_c;
+                widest = std::max(widest, (size_t)G * P.out_w * P.out_c);
+            }
+            net->fused_smem = off * 4;
+            net->fused_threads = (int)std::min<size_t>(512, std::max<size_t>(64, (widest + 31) / 32 * 32));
+            net->fused_ok = 1;
         }
     }
     // workspace: [parameters][state of all streams][rows travelling between layers][counters]

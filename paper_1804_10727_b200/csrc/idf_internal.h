@@ -117,6 +117,35 @@ struct EagerArgs {
 cudaError_t launch_eager_input(const void* in, int in_elem, void* d, long long n, unsigned long long* events, cudaStream_t st);
 cudaError_t launch_eager_layer(const EagerArgs& a, int is_pool, int int_net, cudaStream_t st);
 
+// Depth-first over all layers in one launch (state of a group of streams in shared memory).
+constexpr int FUSED_MAX_LAYERS = 12;
+constexpr size_t FUSED_SMEM_LIMIT = 200 * 1024;
+struct FusedLayer {
+    int kind;              // 0 conv, 1 max-pool
+    int Cin, Cout, Kh, Kw, stride, pad, stride_x, pad_x, relu, shift, round_bf16, Win, Wout, ring_rows;
+    int count_events;      // the layer reports its input events (sparse-path layers)
+    int out_elem;          // element type of the rows the layer emits (pool state in global memory has this type)
+    int state_soff, rowbuf_soff;   // shared memory, in words: ring [slot][G][Wout][Cout] or pool row [G][Wout][C]; emitted row [G][Wout][Cout]
+    long long w_off;       // weights [Kh][Kw][Cin][Cout]: element offset from FusedArgs::weights (fp32 or int8 elements)
+    long long bias_off;    // bias [Cout] words: BYTE offset from FusedArgs::weights, or -1
+    void* state;           // the layer's state in global memory
+    long long rows_in, rows_done;   // progress at launch
+};
+struct FusedArgs {
+    FusedLayer layer[FUSED_MAX_LAYERS];
+    int n_layers, S, G;    // streams in all, streams per CTA
+    const void* in;        // pushed segments [n_seg][S][in_w][in_c] in the element type in_elem
+    int n_seg, in_w, in_c, in_elem, in_soff;
+    int flush;             // the input ends with these segments
+    const void* weights;   // base of the parameter area
+    void* out;             // [S][out_cap][Wout][Cout] in out_elem (fp32 / int8)
+    long long out_cap, out_base;
+    int out_elem;
+    unsigned long long* counters;   // per layer: input events applied (sparse-path layers)
+    unsigned int* status;
+};
+cudaError_t launch_depth_first(const FusedArgs& a, int int_net, int threads, size_t smem_bytes, cudaStream_t st);
+
 // Static plan of the tensor-core path for one conv layer (tile shapes, shared-memory budget).
 struct TcPlan {
     int ok = 0;

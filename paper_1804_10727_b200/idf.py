@@ -39,6 +39,7 @@ EXPORTS = (
     "idf_state_snapshot_bytes", "idf_state_save", "idf_state_restore", "idf_stream_set_out_base", "idf_set_debug_flags", "idf_out_rows_needed",
 )
 DEBUG_NO_TENSOR_CORES, DEBUG_NO_POOL_FUSION, DEBUG_NO_ROW_CHUNKS, DEBUG_NO_PDL, DEBUG_PREFER_THIN = 1, 2, 4, 8, 16
+DEBUG_NO_FUSED, DEBUG_FORCE_FUSED = 32, 64
 
 
 class IdfLayer(ctypes.Structure):
