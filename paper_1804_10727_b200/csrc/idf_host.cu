@@ -47,6 +47,8 @@ struct LayerPlan {
     long long tc_launches = 0;
     // thin layers (the whole receptive field of an output position in one shared-memory row): a kernel of its own for
     // the rows a block determines completely
+    std::vector<unsigned char> wq_packed;      // int nets, Cin % 4 == 0: [Kh][Kw][Cin/4][Cout] words of four int8 (all-layers launch)
+    size_t wq_off = 0;
     ThinPlan thin;
     std::vector<unsigned char> wthin_packed;   // [Cout][row bytes] in the activation type, zero padded
     size_t wthin_off = 0;
@@ -455,9 +457,12 @@ int run_segments(idf_net* net, const void* d_segments, long long n_seg, bool flu
     const size_t nl = net->L.size();
     if (net->eager) return run_segments_eager(net, d_segments, n_seg, flush, d_out, out_cap, emitted);
     if (net->fused_ok && !(debug_flags() & IDF_DEBUG_NO_FUSED) && n_seg <= 65535) {
-        // pushes that the per-layer kernels could only answer with a handful of nearly empty launches take the single
-        // launch that keeps the state on chip: few segments, or little arithmetic altogether
-        const bool small = n_seg <= 2 || net->macs_per_row * (double)n_seg * net->n_streams < 5e7;
+        // Pushes of one or two segments with so little arithmetic that the per-layer kernels' launches are all there is to
+        // them (a small net, a stream or two) take the single launch that keeps the state on chip (measured, one segment
+        // per push: toy1d 17.2 -> 12.3 us per push).  Anything larger is better off with the per-layer kernels, which work
+        // on all rows and streams of a layer at once, on the tensor cores (mnist2d, one image row per push: 8 streams
+        // 26 us per-layer against 30 us in one launch; 4096 streams 114 against 425 us).
+        const bool small = n_seg <= 2 && net->macs_per_row * (double)n_seg * net->n_streams < 2e5;
         if (small || (debug_flags() & IDF_DEBUG_FORCE_FUSED)) return run_segments_fused(net, d_segments, n_seg, flush, d_out, out_cap, emitted);
     }
     // capacity of the caller's output first: the rows complete after this call do not depend on the schedule
@@ -671,7 +676,8 @@ int run_segments_fused(idf_net* net, const void* d_segments, long long n_seg, bo
     a.in = d_segments; a.n_seg = (int)n_seg; a.in_w = net->in_w; a.in_c = net->in_c; a.in_elem = net->L[0].in_elem;
     a.in_soff = net->fused_in_soff; a.flush = flush ? 1 : 0;
     a.weights = net->ws;
-    a.out = d_out; a.out_cap = out_cap; a.out_base = net->out_base; a.out_elem = net->L.back().out_elem;
+    a.out = d_out; a.out_cap = out_cap; a.out_elem = net->L.back().out_elem;
+    a.out_row0 = (int)(net->L.back().rows_done - net->out_base);
     a.counters = (unsigned long long*)(net->ws + net->counters_off);
     a.status = (unsigned int*)(net->ws + net->status_off);
     for (size_t i = 0; i < nl; ++i) {
@@ -684,9 +690,23 @@ int run_segments_fused(idf_net* net, const void* d_segments, long long n_seg, bo
         F.Win = P.in_w; F.Wout = P.out_w; F.ring_rows = P.ring_rows; F.count_events = P.use_sparse; F.out_elem = P.out_elem;
         F.state_soff = net->fused_state_soff[i]; F.rowbuf_soff = net->fused_rowbuf_soff[i];
         F.w_off = (long long)(net->dtype == IDF_I8_I32 ? P.w_off : P.w_off / 4);
+        F.wq_off = net->dtype == IDF_I8_I32 ? (P.wq_packed.empty() ? -1 : (long long)P.wq_off) : 0;
         F.bias_off = P.b_packed.empty() ? -1 : (long long)P.b_off;
         F.state = net->ws + P.state_off;
-        F.rows_in = P.rows_in; F.rows_done = P.rows_done;
+        if (F.kind == 0) {
+            const long long t0 = P.rows_in + P.l.pad, hi = t0 / P.l.stride, tf = t0 - (P.l.kh - 1);
+            F.ph0 = (int)(t0 % P.l.stride);
+            F.hi_slot0 = (int)(hi % P.ring_rows);
+            F.hi_sat0 = (int)std::min<long long>(hi, 1 << 20);
+            F.tf_neg0 = tf < 0 ? (int)-tf : 0;
+            F.phf0 = tf < 0 ? 0 : (int)(tf % P.l.stride);
+            F.done_slot0 = (int)(P.rows_done % P.ring_rows);
+            // rows that complete only because the input ends: those of the final map that the rows received do not complete
+            F.n_flush = flush ? (int)std::max<long long>(0, conv_rows_at_flush(P.l, in_after[i]) -
+                                                             std::max(conv_done_after(P.l, in_after[i]), P.rows_done)) : 0;
+        } else {
+            F.ph0 = (int)(P.rows_in & 1);
+        }
     }
     cudaError_t ce = launch_depth_first(a, net->dtype == IDF_I8_I32, net->fused_threads, net->fused_smem, net->stream);
     if (ce != cudaSuccess) { net->phase = FINISHED; return fail(IDF_ERR_CUDA, "kernel launch failed (all layers in one): %s", cudaGetErrorString(ce)); }
@@ -856,6 +876,15 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
                     memcpy(P.wthin_packed.data() + (size_t)co * P.thin.swb, (const unsigned char*)weights[i] + (size_t)co * taps * l.cin * es,
                            (size_t)taps * l.cin * es);
             }
+            if (spec->dtype == IDF_I8_I32 && l.cin % 4 == 0) {
+                P.wq_packed.resize((size_t)taps * l.cin * l.cout);
+                const int8_t* src = (const int8_t*)weights[i];
+                for (int co = 0; co < l.cout; ++co)
+                    for (int k = 0; k < taps; ++k)
+                        for (int ci = 0; ci < l.cin; ++ci)
+                            P.wq_packed[((((size_t)k * (l.cin / 4) + ci / 4) * l.cout + co) * 4) + (ci & 3)] =
+                                (unsigned char)src[((size_t)co * taps + k) * l.cin + ci];
+            }
             if (biases && biases[i]) {
                 // an all-zero bias is no bias: the kernels then skip the add (state words: +0.0f and 0 are all-zero bits)
                 bool any = false;
@@ -932,26 +961,33 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
             else rate /= 2;
         }
         net->macs_per_row = macs;
-        const size_t per_stream = words * 4;
-        if (ok && per_stream <= FUSED_SMEM_LIMIT) {
-            int G = (int)std::min<size_t>(FUSED_SMEM_LIMIT / per_stream, 32);
+        // rows between layers: fp32 values or int8; rings: words
+        const size_t rs = spec->dtype == IDF_I8_I32 ? 1 : 4;
+        size_t per_stream = (size_t)net->in_w * net->in_c * rs;
+        for (const auto& P : net->L)
+            per_stream += (P.l.kind == IDF_CONV ? (size_t)P.ring_rows * P.out_w * P.out_c * 4 : (size_t)P.out_w * P.out_c * rs) +
+                          (size_t)P.out_w * P.out_c * rs;
+        (void)words;
+        if (ok && per_stream + 64 * net->L.size() <= FUSED_SMEM_LIMIT) {
+            int G = (int)std::min<size_t>((FUSED_SMEM_LIMIT - 64 * net->L.size()) / per_stream, 32);
             G = std::min(G, net->n_streams);
             // (enough CTAs for the SMs before more streams per CTA)
-            while (G > 1 && (net->n_streams + G - 1) / G < 148) --G;
+            while (G > 1 && (net->n_streams + G - 1) / G < 2 * 148) --G;
             net->fused_G = G;
+            auto up16 = [](size_t v) { return (v + 15) / 16 * 16; };
             size_t off = 0;
-            net->fused_in_soff = 0; off += (size_t)G * net->in_w * net->in_c;
+            net->fused_in_soff = 0; off = up16((size_t)G * net->in_w * net->in_c * rs);
             size_t widest = (size_t)G * net->in_w * net->in_c;
             for (const auto& P : net->L) {
                 net->fused_state_soff.push_back((int)off);
-                off += (size_t)(P.l.kind == IDF_CONV ? P.ring_rows : 1) * G * P.out_w * P.out_c;
+                off = up16(off + (P.l.kind == IDF_CONV ? (size_t)P.ring_rows * G * P.out_w * P.out_c * 4 : (size_t)G * P.out_w * P.out_c * rs));
                 net->fused_rowbuf_soff.push_back((int)off);
-                off += (size_t)G * P.out_w * P.out_c;
+                off = up16(off + (size_t)G * P.out_w * P.out_c * rs);
                 widest = std::max(widest, (size_t)G * P.out_w * P.out_c);
             }
-            net->fused_smem = off * 4;
+            net->fused_smem = off;
             net->fused_threads = (int)std::min<size_t>(512, std::max<size_t>(64, (widest + 31) / 32 * 32));
-            net->fused_ok = 1;
+            net->fused_ok = off <= FUSED_SMEM_LIMIT;
         }
     }
     // workspace: [parameters][state of all streams][rows travelling between layers][counters]
@@ -961,6 +997,7 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
         P.b_off = off; off = align_up(off + P.b_packed.size());
         P.wtc_off = off; off = align_up(off + P.wtc_packed.size(), 1024);
         P.wthin_off = off; off = align_up(off + P.wthin_packed.size(), 1024);
+        P.wq_off = off; off = align_up(off + P.wq_packed.size());
     }
     net->state_region_off = off;
     for (auto& P : net->L) {
@@ -1063,6 +1100,8 @@ int idf_stream_open(idf_net* net, void* d_workspace, size_t workspace_bytes, voi
                                                   P.unfold ? P.kpad : P.l.cin, P.l.cout, P.w_map_pool) != 0)
                 P.tc_pool.ok = 0;
         }
+        if (!P.wq_packed.empty() && e == cudaSuccess)
+            e = cudaMemcpyAsync(net->ws + P.wq_off, P.wq_packed.data(), P.wq_packed.size(), cudaMemcpyHostToDevice, net->stream);
         if (!P.wthin_packed.empty() && e == cudaSuccess) {
             e = cudaMemcpyAsync(net->ws + P.wthin_off, P.wthin_packed.data(), P.wthin_packed.size(), cudaMemcpyHostToDevice, net->stream);
             if (thin_encode_weights(P.thin, net->dtype, net->ws + P.wthin_off, P.l.cout, P.w_map_thin) != 0) P.thin.ok = 0;

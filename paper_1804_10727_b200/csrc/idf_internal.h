@@ -125,11 +125,14 @@ struct FusedLayer {
     int Cin, Cout, Kh, Kw, stride, pad, stride_x, pad_x, relu, shift, round_bf16, Win, Wout, ring_rows;
     int count_events;      // the layer reports its input events (sparse-path layers)
     int out_elem;          // element type of the rows the layer emits (pool state in global memory has this type)
-    int state_soff, rowbuf_soff;   // shared memory, in words: ring [slot][G][Wout][Cout] or pool row [G][Wout][C]; emitted row [G][Wout][Cout]
+    int state_soff, rowbuf_soff;   // shared memory, in bytes: ring [slot][G][Wout][Cout] words or pool row [G][Wout][C]; emitted row [G][Wout][Cout]
     long long w_off;       // weights [Kh][Kw][Cin][Cout]: element offset from FusedArgs::weights (fp32 or int8 elements)
+    long long wq_off;      // int nets: the same weights, four input channels to a word [Kh][Kw][Cin/4][Cout], BYTE offset; -1: none
     long long bias_off;    // bias [Cout] words: BYTE offset from FusedArgs::weights, or -1
     void* state;           // the layer's state in global memory
-    long long rows_in, rows_done;   // progress at launch
+    // the layer's progress when the launch begins, as the small counters the kernel steps (see LayerClock)
+    int ph0, hi_slot0, hi_sat0, phf0, tf_neg0, done_slot0;
+    int n_flush;           // rows the layer completes on bottom padding if the input ends with this launch
 };
 struct FusedArgs {
     FusedLayer layer[FUSED_MAX_LAYERS];
@@ -139,7 +142,8 @@ struct FusedArgs {
     int flush;             // the input ends with these segments
     const void* weights;   // base of the parameter area
     void* out;             // [S][out_cap][Wout][Cout] in out_elem (fp32 / int8)
-    long long out_cap, out_base;
+    long long out_cap;
+    int out_row0;          // index in the caller's buffer of the next output row
     int out_elem;
     unsigned long long* counters;   // per layer: input events applied (sparse-path layers)
     unsigned int* status;

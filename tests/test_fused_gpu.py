@@ -80,8 +80,9 @@ def test_per_layer_kernels_and_the_single_launch_take_turns_on_one_stream(orc, m
 
 
 def test_small_pushes_take_the_single_launch_by_default(orc):
-    """One image row per push on the mnist2d net: one launch per push (the per-layer kernels need three to five)."""
-    w = workloads.get("mnist2d", n_streams=300)
+    """One image row per push on the mnist2d net with a single stream: one launch per push (the per-layer kernels
+    need three to five); with hundreds of streams a push is real work and stays with the per-layer kernels."""
+    w = workloads.get("mnist2d", n_streams=1)
     x = workloads.make_input(w)
     ws, bs = workloads.make_params(w)
     want = orc.forward(w.dtype, w.layers, x, ws, bs)
@@ -92,19 +93,21 @@ def test_small_pushes_take_the_single_launch_by_default(orc):
     assert net.event_counts()[0] == int((x != 0).sum())          # the sparse first layer still reports its events
     assert net.state_bytes == 18432
     net.close()
-    # whole images in one push: per-layer kernels (tensor cores for the dense layers)
+    w = workloads.get("mnist2d", n_streams=300)
+    x = workloads.make_input(w)
+    want = orc.forward(w.dtype, w.layers, x, ws, bs)
     net = idf.net_from_workload(w, ws, bs)
-    got = idf.infer(net, x, last=True)
-    assert any(t > 0 for t in net.status())
-    assert_equal(got, want, "mnist2d, whole images")
+    got = idf.infer(net, x, chunks=[1] * w.H, last=True)
+    assert net.launches > w.H and any(t > 0 for t in net.status())
+    assert_equal(got, want, "mnist2d, 300 streams, one row per push")
     net.close()
-    # toy1d: so little arithmetic that the whole signal is one launch
-    t = workloads.get("toy1d")
+    # toy1d, a few samples per push
+    t = workloads.get("toy1d", H=301)
     xt = workloads.make_input(t)
     wt, bt = workloads.make_params(t)
     net = idf.net_from_workload(t, wt, bt)
-    got = idf.infer(net, xt, last=True)
-    assert net.launches == 1
+    got = idf.infer(net, xt, chunks=[2] * 150, last=True)
+    assert net.launches == 151
     assert_close(got, orc.forward(t.dtype, t.layers, xt, wt, bt), "toy1d")
     net.close()
 
