@@ -762,7 +762,8 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
     net->eager = spec->emission == IDF_EMIT_EAGER;
     // default: about 25 000 positions per stream and block (112 rows of a 224-wide image, 1024 samples of a 1D
     // signal): long enough that a launch's fixed cost (weights into shared memory, ring rows in and out) is small
-    net->row_block = spec->row_block > 0 ? spec->row_block : std::min(1024, std::max(32, 25088 / spec->in_w));
+    // (1D signals: 4096 samples - fewer launches and fewer rows read twice at the edges of row chunks; audio1d 2.9 -> 2.3 ms)
+    net->row_block = spec->row_block > 0 ? spec->row_block : (spec->in_w == 1 ? 4096 : std::min(1024, std::max(32, 25088 / spec->in_w)));
     const int act_elem = spec->dtype == IDF_F32 ? E_F32 : (spec->dtype == IDF_BF16_F32 ? E_BF16 : E_I8);
     const size_t state_word = 4;
 

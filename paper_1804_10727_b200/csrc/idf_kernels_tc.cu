@@ -1361,6 +1361,7 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     // a launch that emits pooled rows stages half a tile of positions
     const int stage_rows = pooled ? 64 : 128;
     int best = 0, best_units = -1;
+    const bool wide_for_1d = true;
     for (int nt = 256; nt >= 16; nt >>= 1) {
         if (Cout % nt) continue;
         if ((ring_rows + 1) * nt > 512) continue;
@@ -1369,6 +1370,10 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
         if (wb + 3 * a_stage + (size_t)stage_rows * nt * out_esize + 10240 > SMEM_LIMIT) continue;   // one staging tile at least
         const int units = p->n_mt * (Cout / nt);
         if (units >= 120) { best = nt; break; }          // enough CTAs for the 148 SMs: take the widest such tile
+        // 1D nets come in long blocks of rows, which row chunks spread over the SMs: there the widest tile that fits
+        // wins, because every channel slice fetches the Δ-rows again (audio1d's 128-channel layers with 16-channel
+        // tiles moved 4.2 GB per layer through the L2)
+        if (Win == 1 && wide_for_1d) { best = nt; break; }
         if (units > best_units) { best_units = units; best = nt; }
     }
     if (!best) return false;
