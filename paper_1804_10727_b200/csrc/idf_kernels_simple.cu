@@ -317,12 +317,18 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
     const int n_comp = a.Win * a.Cin;
     const int taps = a.Kh * a.Kw;
     const int slot0 = (int)(a.o_begin % a.ring_rows);     // ring slot of the first visited row
-    long long done = a.o_begin;                      // rows below `done` have been emitted
-    // finalisation of the ring rows below `upto`: emit f(c + b), zero the slot
-    auto finalise_upto = [&](long long upto) {
+    // Row bookkeeping relative to the block (32-bit, stepping counters: a 64-bit division per row and thread costs as
+    // much as the row's own work): rows are counted from o_begin, input rows from r0.
+    int done = 0;                                    // visited rows below `done` have been emitted
+    int done_slot = slot0;                           // ring slot of visited row `done`
+    const int done_end_rel = (int)(a.done_end - a.o_begin), n_in = (int)(a.r1 - a.r0);
+    const int c_q = (int)(a.r0 + a.pad - a.Kh - a.o_begin * a.stride);       // r + pad - Kh - o_begin*stride for r = r0
+    // finalisation of the visited rows below `upto`: emit f(c + b), zero the slot
+    auto finalise_upto = [&](int upto) {
         for (; done < upto; ++done) {
-            const long long slot = done % a.ring_rows;
-            TO* orow = out + (done - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride;
+            const int slot = done_slot;
+            if (++done_slot == a.ring_rows) done_slot = 0;
+            TO* orow = out + (a.o_begin + done - a.out_row_base) * a.out_row_stride + (long long)s * a.out_stream_stride;
             if (!IDF_OK_AT(a.status, (orow - out) + row_elems - 1, a.out_elems) || !IDF_OK_AT(a.status, orow - out, a.out_elems) ||
                 !IDF_OK_AT(a.status, (slot + 1) * (long long)row_elems - 1, (long long)a.ring_rows * row_elems)) continue;
             if (sizeof(TO) == 1 && (a.Cout & 3) == 0 && (((uintptr_t)orow) & 3) == 0) {
@@ -372,16 +378,19 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
     // hide behind the arithmetic of the other); (B) the events are scattered into the ring.  The event
     // counter is double-buffered so that it can be cleared for the next pass while this one's is still read.
     int cb = 0;
-    for (long long r = a.r0; r <= a.r1; ++r) {
-        // r == r1 is the closing pass: no input, everything below done_end is finalised
-        const bool have = r < a.r1;
-        long long upto = a.done_end;
+    for (int rr = 0; rr <= n_in; ++rr) {
+        // rr == n_in is the closing pass: no input, everything below done_end is finalised
+        const bool have = rr < n_in;
+        int upto = done_end_rel;
         if (have) {
-            const long long q = r + a.pad - a.Kh;        // row o completes at input row o*stride - pad + Kh - 1, here: <= r - 1
-            upto = q < 0 ? 0 : q / a.stride + 1;
-            if (upto > a.done_end) upto = a.done_end;
+            // row o completes at input row o*stride - pad + Kh - 1, here: <= r - 1; relative to o_begin:
+            // floor((r + pad - Kh) / stride) + 1 - o_begin, not below 0
+            const int q = rr + c_q;
+            upto = q < 0 ? -((-q + a.stride - 1) / a.stride) + 1 : q / a.stride + 1;
+            if (upto < 0) upto = 0;
+            if (upto > done_end_rel) upto = done_end_rel;
         }
-        const TI* row = in + ((r - a.r0) * a.S + s) * (long long)n_comp;
+        const TI* row = in + ((long long)rr * a.S + s) * (long long)n_comp;
         if (have && !IDF_OK_AT(a.status, (row - in) + n_comp - 1, a.in_elems)) continue;
         const int n_pass = have ? (n_comp + SPARSE_MAX_EVENTS - 1) / SPARSE_MAX_EVENTS : 1;
         for (int pass = 0; pass < n_pass; ++pass) {
@@ -417,7 +426,7 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
             // scatter: a warp takes one event at a time and walks its kernel taps, the lanes take the output
             // channels; target row, ring slot and target x are worked out once per tap row / tap (no
             // per-channel index arithmetic, no division when the stride is 1)
-            const int ty0 = (int)(r - a.o_begin * a.stride) + a.pad;          // tap ky reaches relative row (ty0 - ky) / stride
+            const int ty0 = rr + c_q + a.Kh;                                  // = r + pad - o_begin*stride: tap ky reaches relative row (ty0 - ky) / stride
             if (RING_IN_SMEM && w_in_smem && a.stride == 1 && a.stride_x == 1 && a.Kh == 3 && a.Kw == 3) {
                 // the common 3x3, stride-1 case with everything in shared memory, unrolled: the three target rows'
                 // slot offsets are worked out once per input row, a tap costs an address, a weight, a reduction
