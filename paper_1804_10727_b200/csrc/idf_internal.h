@@ -158,6 +158,7 @@ struct TcPlan {
     int shift_mode = 0;      // kx taps read one haloed tile at row offsets instead of one box per kx
     int sx = 1;              // x stride (> 1 only without shift_mode: the tensor map walks the input row in steps of sx)
     int a_stage_bytes = 0;
+    int n_box = 1, a_box_pitch = 0;   // TMA boxes per stage (one per kx tap where the taps cannot share a haloed box), their distance
     int n_xt = 0, n_mt = 0;  // x tiles per row, M tiles in all
     int Ntile = 0, n_nt = 0; // output channels per CTA, N tiles
     int KB = 0, n_kb = 0;    // input channels per K block (one swizzled shared-memory row), K blocks

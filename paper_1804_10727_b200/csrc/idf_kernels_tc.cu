@@ -465,6 +465,7 @@ struct TcArgs {
     int n_chunks, chunk_rows, chunk_shift;   // the block's output rows are cut into n_chunks runs of chunk_rows rows (the first one
                                  // chunk_shift shorter), one CTA each: see the kernel's prologue
     int a_stage_bytes;
+    int n_box, a_box_pitch;      // TMA boxes per stage (one per kx tap when the taps cannot share a haloed box) and their distance in bytes
     int out_esize, out_pwb, out_panels, out_stage_bytes;   // emitted rows: staging panels of out_pwb-byte rows
     int out_stage_rows;          // rows of one staging panel: 128, or 64 when only pooled rows are staged
     int out_groups;              // epilogue groups at work, each with its own staging tile(s)
@@ -507,7 +508,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t w_tile_bytes = (uint32_t)a.Ntile * a.swb;
     const uint32_t a_stage_bytes = (uint32_t)a.a_stage_bytes;
     const uint32_t a_box_bytes = (uint32_t)a.BXP * a.BS * a.swb;
-    const int n_xload = a.shift_mode ? 1 : a.Kw;
+    // (rows of 128 bytes always share one haloed box: for that instantiation the compiler sees the constant)
+    const int n_box = KSTEPS == 4 ? 1 : a.n_box;
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sW = base;
@@ -644,16 +646,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     // barrier and has one barrier less to look at.
                     const uint32_t* qr = s_rowq[ri & (ROWQ - 1)];
                     if (qr[0] && !mbar_wait(qr[0], qr[1], abort_flag)) { ok = false; break; }
-                    for (int xl = 0; xl < n_xload && ok; ++xl)
-                        for (int kb = 0; kb < a.n_kb; ++kb) {
-                            if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-                            if (!IDF_OK_AT(a.status, (sA - smem_u32(smem_raw)) + (uint32_t)stage * a_stage_bytes + a_box_bytes - 1, bars - smem_u32(smem_raw))) { ok = false; break; }
-                            mbar_expect_tx(bar_full + 8u * stage, a_box_bytes);
-                            tma_load_4d(sA + (uint32_t)stage * a_stage_bytes, &tmA, bar_full + 8u * stage,
+                    // one stage per (row, K block): the haloed box all kx taps share, or one box per kx tap side by side
+                    for (int kb = 0; kb < a.n_kb; ++kb) {
+                        if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                        if (!IDF_OK_AT(a.status, (sA - smem_u32(smem_raw)) + (uint32_t)stage * a_stage_bytes + (uint32_t)(n_box - 1) * a.a_box_pitch + a_box_bytes - 1,
+                                       bars - smem_u32(smem_raw))) { ok = false; break; }
+                        mbar_expect_tx(bar_full + 8u * stage, (uint32_t)n_box * a_box_bytes);
+                        for (int xl = 0; xl < n_box; ++xl)
+                            tma_load_4d(sA + (uint32_t)stage * a_stage_bytes + (uint32_t)xl * a.a_box_pitch, &tmA, bar_full + 8u * stage,
                                         kb * a.KB, x0 * a.sx - a.pad_x + xl, s0, c_ra + ri);
-                            ++t;
-                            if (++stage == a.nstage) { stage = 0; phase ^= 1u; }
-                        }
+                        ++t;
+                        if (++stage == a.nstage) { stage = 0; phase ^= 1u; }
+                    }
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -671,9 +675,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // row only arrives once its slot is free).
         {
             const uint64_t desc_hi = make_smem_desc(0, a.swb);
-            const int n_kx = a.shift_mode ? a.Kw : 1;
+            const int n_kx = a.shift_mode ? a.Kw : n_box;         // kx taps of a stage: row-shifted reads of one box, or one box each
             const int nslot = a.nslot;
-            const uint32_t kx_bytes = a.shift_mode ? (uint32_t)a.swb >> 4 : 0u;
+            const uint32_t kx_bytes = (KSTEPS == 4 || a.shift_mode) ? (uint32_t)a.swb >> 4 : (uint32_t)a.a_box_pitch >> 4;
             const uint32_t wtile_kx = ((uint32_t)(a.n_kb * a.Kh) * w_tile_bytes) >> 4;   // descriptor units per kx
             const uint32_t wtile_kb = ((uint32_t)a.Kh * w_tile_bytes) >> 4;
             const uint32_t a_stage_units = a_stage_bytes >> 4;
@@ -685,7 +689,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 ok = mbar_wait(bar_w + 8u * tap, 0, abort_flag);
             const uint64_t adesc_base = desc_hi | (uint64_t)((sA & 0x3FFFFu) >> 4);
             const uint64_t bdesc_base = desc_hi | (uint64_t)((sW & 0x3FFFFu) >> 4);
-            const int n_st = n_xload * n_kb;                     // tiles per input row
+            const int n_st = n_kb;                               // tiles (stages) per input row
             const bool issuer = elect_one();                     // the lane that issues (the warp stays converged)
             ok = ok && mbar_wait(bar_full, 0, abort_flag);       // first tile of the first row
             tc_fence_after();
@@ -701,7 +705,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // tap kx reads the same tile kxi rows further down: the swizzle is a function of the absolute
             // shared-memory address, so a start address moved by whole rows still meets the pattern the TMA
             // wrote (base-offset field stays 0).
-            const uint32_t b_xl_step = a.shift_mode ? 0u : wtile_kx;       // weight blocks of the next kx box (one box per kx)
             int ri = 0, st = 0, kb = 0, stage = 0;
             uint32_t phase = 0;
             uint64_t adesc_cur = adesc_base, bdesc_cur = bdesc_base;       // the tile at hand
@@ -725,8 +728,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (n_stage == nstage) { n_stage = 0; n_phase ^= 1u; adesc_nx = adesc_base; }
                 uint64_t bdesc_nx = bdesc_cur + wtile_kb;
                 int n_kbi = kb + 1;
-                if (n_kbi == n_kb) { n_kbi = 0; bdesc_nx += (uint64_t)b_xl_step - (uint64_t)((uint32_t)n_kb * wtile_kb); }
-                if (row_end) bdesc_nx = bdesc_base;
+                if (n_kbi == n_kb) { n_kbi = 0; bdesc_nx = bdesc_base; }
                 uint32_t next_ok = 1u;
                 if (!(last_row && row_end)) next_ok = mbar_test(bar_full + 8u * n_stage, n_phase);
                 uint4 nh = hdr, na = sa, nb = sb, nc = sc;
@@ -1354,8 +1356,14 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     // A stage holds exactly the TMA box (BS streams x BXP positions).  The MMAs read 128 rows from row kx on,
     // so for the last positions they run past the box into whatever follows in shared memory: those are
     // lanes outside the tile, whose accumulators nobody reads.
-    const size_t a_stage = ((size_t)p->BS * p->BXP * p->swb + 1023) / 1024 * 1024;
+    // kx taps that cannot share a haloed box (rows of 32 or 64 bytes, x-strided layers) get a box each, side by side in
+    // the stage, under one barrier
+    const int n_box = (!p->shift_mode && Kw > 1) ? Kw : 1;
+    const size_t box_pitch = ((size_t)p->BS * p->BXP * p->swb + 1023) / 1024 * 1024;
+    const size_t a_stage = (size_t)n_box * box_pitch;
     p->a_stage_bytes = (int)a_stage;
+    p->n_box = n_box;
+    p->a_box_pitch = (int)box_pitch;
     p->n_mt = p->n_xt * ((S + p->BS - 1) / p->BS);
     const int taps = Kh * Kw;
     // a launch that emits pooled rows stages half a tile of positions
@@ -1404,7 +1412,7 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     if (wb + (want_stages + 1) * a_stage + 2 * (size_t)p->out_groups * p->out_stage_bytes + 10240 <= SMEM_LIMIT) p->out_bufs = 2;
     // the MMAs' run past a small box (see a_stage) must end inside this CTA's shared memory: what follows the
     // last stage (the staging tiles) covers it, or padding is added behind them
-    const size_t overrun = (size_t)(128 + halo) * p->swb > a_stage ? (size_t)(128 + halo) * p->swb - a_stage : 0;
+    const size_t overrun = (size_t)(128 + halo) * p->swb > box_pitch ? (size_t)(128 + halo) * p->swb - box_pitch : 0;
     const size_t tail_have = (size_t)p->out_groups * p->out_bufs * p->out_stage_bytes;
     const size_t tail_pad = overrun > tail_have ? (overrun - tail_have + 1023) / 1024 * 1024 : 0;
     if (SMEM_LIMIT < 8192 + wb + 1024 + tail_have + tail_pad + 2 * a_stage) return false;
@@ -1500,7 +1508,7 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     t.pad_x = a.pad_x; t.relu = a.relu; t.shift = a.shift; t.ring_rows = a.ring_rows; t.out_elem = a.out_elem;
     t.BX = p.BX; t.BS = p.BS; t.n_xt = p.n_xt; t.Ntile = p.Ntile; t.n_nt = p.n_nt; t.KB = p.KB; t.n_kb = p.n_kb;
     t.swb = p.swb; t.nslot = p.nslot; t.nstage = p.nstage; t.tmem_cols = p.tmem_cols;
-    t.BXP = p.BXP; t.shift_mode = p.shift_mode; t.sx = p.sx; t.a_stage_bytes = p.a_stage_bytes;
+    t.BXP = p.BXP; t.shift_mode = p.shift_mode; t.sx = p.sx; t.a_stage_bytes = p.a_stage_bytes; t.n_box = p.n_box; t.a_box_pitch = p.a_box_pitch;
     t.out_esize = p.out_esize; t.out_pwb = p.out_pwb; t.out_panels = p.out_panels; t.out_stage_bytes = p.out_stage_bytes; t.out_stage_rows = p.out_stage_rows; t.out_groups = p.out_groups; t.out_bufs = p.out_bufs;
     t.out_row_dim = row_dim; t.out_row_first = (int)(a.o_begin - a.out_row_base);
     t.pool = a.pool_fused; t.pool_keep = a.pool_keep; t.pool_state = a.pool_state; t.pool_row_base = a.out_row_base;
