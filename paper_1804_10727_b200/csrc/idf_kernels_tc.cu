@@ -490,7 +490,9 @@ template <int DT> struct Acc;
 template <> struct Acc<1> { typedef float S; };
 template <> struct Acc<2> { typedef int S; };
 
-template <int DT, int KSTEPS>
+// KX3: the common case of 128-byte rows with three kx taps read row-shifted from one haloed box, known at compile time
+// (the MMA warp's loop is what the kernel's speed hangs on: every constant it sees helps)
+template <int DT, int KSTEPS, int KX3>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                const __grid_constant__ CUtensorMap tmO, const TcArgs a)
@@ -675,7 +677,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // row only arrives once its slot is free).
         {
             const uint64_t desc_hi = make_smem_desc(0, a.swb);
-            const int n_kx = a.shift_mode ? a.Kw : n_box;         // kx taps of a stage: row-shifted reads of one box, or one box each
+            const int n_kx = KX3 ? 3 : (a.shift_mode ? a.Kw : n_box);   // kx taps of a stage: row-shifted reads of one box, or one box each
             const int nslot = a.nslot;
             const uint32_t kx_bytes = (KSTEPS == 4 || a.shift_mode) ? (uint32_t)a.swb >> 4 : (uint32_t)a.a_box_pitch >> 4;
             const uint32_t wtile_kx = ((uint32_t)(a.n_kb * a.Kh) * w_tile_bytes) >> 4;   // descriptor units per kx
@@ -1549,12 +1551,12 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const 
     }
     const unsigned grid = (unsigned)(p.n_mt * p.n_nt * t.n_chunks);
     typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const TcArgs);
-    static const KernelFn kernels[2][3] = {
-        {conv_tc_kernel<1, 1>, conv_tc_kernel<1, 2>, conv_tc_kernel<1, 4>},
-        {conv_tc_kernel<2, 1>, conv_tc_kernel<2, 2>, conv_tc_kernel<2, 4>}};
-    const int kidx = p.swb == 32 ? 0 : (p.swb == 64 ? 1 : 2);
+    static const KernelFn kernels[2][4] = {
+        {conv_tc_kernel<1, 1, 0>, conv_tc_kernel<1, 2, 0>, conv_tc_kernel<1, 4, 0>, conv_tc_kernel<1, 4, 1>},
+        {conv_tc_kernel<2, 1, 0>, conv_tc_kernel<2, 2, 0>, conv_tc_kernel<2, 4, 0>, conv_tc_kernel<2, 4, 1>}};
+    const int kidx = p.swb == 32 ? 0 : (p.swb == 64 ? 1 : ((p.shift_mode && a.Kw == 3) ? 3 : 2));
     const KernelFn fn = kernels[dtype - 1][kidx];
-    static bool attr_set[2][3][64] = {};
+    static bool attr_set[2][4][64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!attr_set[dtype - 1][kidx][dev]) {
