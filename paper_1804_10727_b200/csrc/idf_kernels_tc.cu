@@ -685,7 +685,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t a_stage_units = a_stage_bytes >> 4;
             const int nstage = a.nstage, n_kb = a.n_kb;
             bool ok = true;
-            for (int slot = 0; slot < nslot && ok; ++slot)       // every slot has been cleared once
+            // every slot this launch uses has been cleared once (a short launch visits fewer rows than there are slots)
+            for (int slot = 0; slot < (c_n_orows < nslot ? c_n_orows : nslot) && ok; ++slot)
                 ok = mbar_wait(bar_free + 8u * slot, 0, abort_flag);
             for (int tap = 0; tap < taps && ok; ++tap)            // the CTA's weight slice has landed
                 ok = mbar_wait(bar_w + 8u * tap, 0, abort_flag);
@@ -821,7 +822,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         bool ok = true;
         // every ring slot in tensor memory starts at zero (all MMAs accumulate)
         if (grp == 0)
-            for (int slot = 0; slot < a.nslot; ++slot) {
+            for (int slot = 0; slot < (c_n_orows < a.nslot ? c_n_orows : a.nslot); ++slot) {
                 for (int c = 0; c < a.Ntile; c += 16) tmem_st16_zero(tlane + (uint32_t)(slot * a.Ntile + c));
                 tmem_st_wait();
                 tc_fence_before();
