@@ -85,3 +85,20 @@ SMALL_NETS = {
 
 def small_dims(name):
     return (61, 1) if name.startswith("oned") else (19, 14)
+
+
+# End-to-end criterion for the bf16 workloads (every hidden activation is a rounding decision on an fp32 sum in
+# tensor-core order; the strict tolerance holds layer by layer, see test_full_size_gpu.py): about twice what is measured
+# (vgg2d: relative rms 2^-9.3, largest error 2^-8.1 of max|o|, 66 % of the outputs inside 1e-4 + 1e-3|o|;
+#  audio1d: 2^-11.1 ... 2^-11.5, 2^-8.8, 96-98 %).
+BF16_E2E = {"vgg2d": (2.0 ** -8.3, 2.0 ** -7.1, 0.55), "audio1d": (2.0 ** -10.1, 2.0 ** -7.8, 0.93)}
+
+
+def assert_bf16_end_to_end(name, got, want, what=""):
+    rms_lim, max_lim, frac_lim = BF16_E2E[name]
+    err = np.asarray(got, dtype=np.float64) - np.asarray(want, dtype=np.float64)
+    rel_rms = np.sqrt((err ** 2).mean() / (want ** 2).mean())
+    rel_max = np.abs(err).max() / np.abs(want).max()
+    frac = (np.abs(err) <= ATOL + RTOL * np.abs(want)).mean()
+    print(f"{what}: relative rms 2^{np.log2(rel_rms):.2f}, largest error 2^{np.log2(rel_max):.2f} of max|o|, {100 * frac:.1f} % inside the strict tolerance")
+    assert rel_rms < rms_lim and rel_max < max_lim and frac > frac_lim, (what, rel_rms, rel_max, frac)

@@ -6,7 +6,7 @@ import torch
 
 from paper_1804_10727_b200 import idf, workloads
 from paper_1804_10727_b200.workloads import Layer, conv, POOL
-from helpers import (SMALL_NETS, assert_close, assert_equal, rand_net, small_dims, with_path, with_shifts)
+from helpers import (SMALL_NETS, assert_bf16_end_to_end, assert_close, assert_equal, rand_net, small_dims, with_path, with_shifts)
 
 pytestmark = pytest.mark.gpu
 
@@ -246,10 +246,7 @@ def test_workloads_match_oracle(orc, name, S, H):
         # order differs from the oracle's float64 sum; a decision that falls on the other side
         # moves that activation by one bf16 ulp (2^-8 relative).  The end-to-end comparison is
         # therefore statistical; the strict tolerance is checked layer by layer below.
-        err = got - want
-        rel_rms = np.sqrt((err ** 2).mean() / (want ** 2).mean())
-        assert rel_rms < 2.0 ** -7, rel_rms
-        assert np.abs(err).max() < 2.0 ** -4 * np.abs(want).max()
+        assert_bf16_end_to_end(name, got, want, name)
 
 
 @pytest.mark.parametrize("name,S,H", [("audio1d", 3, 3000), ("vgg2d", 2, None)])
