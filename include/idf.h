@@ -120,7 +120,12 @@ typedef struct {
     int in_w, in_c;            /* segment width (1 for 1D) and channels */
     int n_streams;             /* streams advanced together by every call */
     int row_block;             /* most segments pushed through all layers at once (bounds the   */
-                               /* transient workspace); 0 = library default                     */
+                               /* transient workspace); 0 = library default: about 25 000       */
+                               /* positions per stream (112 rows of a 224-wide image, at most   */
+                               /* 1024 rows), 4096 samples for 1D nets.  The buffers between    */
+                               /* layers hold 2 * row_block + 8 rows of every stream whatever   */
+                               /* the streams' real length: for short streams (a 28-row image)  */
+                               /* give the real row count and the workspace shrinks with it     */
     int emission;              /* idf_emission; 0 = IDF_EMIT_DEFERRED                           */
 } idf_spec;
 
