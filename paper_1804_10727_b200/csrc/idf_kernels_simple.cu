@@ -342,9 +342,13 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
                     for (int i = tid; i < (row_elems >> 2); i += SPARSE_THREADS) {
                         const int4 c = src[i];
                         ((int4*)src)[i] = make_int4(0, 0, 0, 0);
-                        const int v0 = min((max(c.x, 0) + rnd) >> a.shift, 127), v1 = min((max(c.y, 0) + rnd) >> a.shift, 127);
-                        const int v2 = min((max(c.z, 0) + rnd) >> a.shift, 127), v3 = min((max(c.w, 0) + rnd) >> a.shift, 127);
-                        dst[i] = __byte_perm(__byte_perm(v0, v1, 0x4040), __byte_perm(v2, v3, 0x4040), 0x5410);
+                        // (c + rnd) >> shift is negative exactly when max(c, 0) + rnd >> shift would be 0 (c < 0 means
+                        // c + rnd < 2^shift), so the ReLU is the saturating pack's lower bound; the upper bound is 127
+                        const int v0 = (c.x + rnd) >> a.shift, v1 = (c.y + rnd) >> a.shift, v2 = (c.z + rnd) >> a.shift, v3 = (c.w + rnd) >> a.shift;
+                        uint32_t hi2, all4;
+                        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(v3), "r"(v2));
+                        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(all4) : "r"(v1), "r"(v0), "r"(hi2));
+                        dst[i] = __vminu4(all4, 0x7f7f7f7fu);
                     }
                 } else
                 for (int i = tid * 4; i < row_elems; i += SPARSE_THREADS * 4) {
