@@ -39,7 +39,7 @@ struct LayerPlan {
     int in_elem, out_elem;   // Elem of the rows this layer receives / emits
     int use_sparse;
     TcPlan tc;                              // tensor-core path (tc.ok) for the dense update
-    std::vector<unsigned char> wtc_packed;  // [tap][Cout][Cin] in the activation type
+    std::vector<unsigned char> wtc_packed;  // [tap slot][Cout][Cin] in the activation type, tap slots in the order of tc_weight_slot
     size_t wtc_off = 0;
     alignas(64) unsigned char w_map[128];   // TMA descriptor of wtc in the workspace (made at open)
     TcPlan tc_pool;                         // plan of the launches that also emit the following max-pool's rows
@@ -825,7 +825,7 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
                             dst[((size_t)k * l.cin + ci) * l.cout + co] = v;
                         }
             }
-            // tensor-core layout [tap][Cout][Cin], activation type, when the layer qualifies
+            // tensor-core layout [tap slot][Cout][Cin], activation type, when the layer qualifies
             const int in_cap = i == 0 ? net->row_block : net->L[i - 1].out_cap_rows;
             const bool tc_allowed = !P.use_sparse && !(debug_flags() & IDF_DEBUG_NO_TENSOR_CORES) && spec->dtype != IDF_F32 && !net->eager;
             const size_t es = spec->dtype == IDF_I8_I32 ? 1 : 2;
@@ -839,7 +839,7 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
                 P.wtc_packed.resize(nw * es);
                 for (int co = 0; co < l.cout; ++co)
                     for (int k = 0; k < taps; ++k)
-                        memcpy(P.wtc_packed.data() + (((size_t)k * l.cout + co) * l.cin) * es,
+                        memcpy(P.wtc_packed.data() + (((size_t)tc_weight_slot(k / l.kw, k % l.kw, l.kh, l.stride) * l.cout + co) * l.cin) * es,
                                (const unsigned char*)weights[i] + (((size_t)co * taps + k) * l.cin) * es, (size_t)l.cin * es);
             } else if (tc_allowed) {
                 // thin (Cin*Kw below a tensor-core K step) or x-strided layer: unfold x first
@@ -858,7 +858,7 @@ int idf_net_create(const idf_spec* spec, const void* const* weights, const void*
                     P.wtc_packed.assign((size_t)l.kh * l.cout * kpad * es, 0);      // [ky][Cout][kx*Cin + ci], zero padded
                     for (int co = 0; co < l.cout; ++co)
                         for (int ky = 0; ky < l.kh; ++ky)
-                            memcpy(P.wtc_packed.data() + (((size_t)ky * l.cout + co) * kpad) * es,
+                            memcpy(P.wtc_packed.data() + (((size_t)tc_weight_slot(ky, 0, l.kh, l.stride) * l.cout + co) * kpad) * es,
                                    (const unsigned char*)weights[i] + (((size_t)co * l.kh + ky) * l.kw * l.cin) * es,
                                    (size_t)l.kw * l.cin * es);
                 }

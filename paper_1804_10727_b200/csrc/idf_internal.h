@@ -171,10 +171,11 @@ struct TcPlan {
     int out_esize = 0, out_pwb = 0, out_panels = 0, out_stage_bytes = 0;   // staging of emitted rows for the TMA store
     int out_stage_rows = 0;  // rows of one staging panel: 128, or 64 in a plan for launches that emit pooled rows
     size_t smem_bytes = 0;
-    size_t w_bytes = 0;      // device weights for this path: [tap][Cout][Cin] in the activation type
+    size_t w_bytes = 0;      // device weights for this path: [tap slot][Cout][Cin] in the activation type
 };
 bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh, int Kw, int stride_x, int ring_rows,
                   int out_esize, int pooled, TcPlan* p);
+int tc_weight_slot(int ky, int kx, int Kh, int stride);
 int tc_encode_weights(const TcPlan& p, int dtype, const void* d_w, int taps, int Cin, int Cout, void* map_out);
 cudaError_t launch_conv_tc(const ConvArgs& a, const TcPlan& p, int dtype, const void* w_map, int n_in_rows,
                            unsigned int* status, cudaStream_t st);

@@ -110,6 +110,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
 
 // true in exactly one lane of a converged warp
 __device__ __forceinline__ bool elect_one()
@@ -192,7 +198,7 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 // that the taps one input row uses (ky = ph, ph+stride, ...) sit next to each other with ky
 // descending: their output rows ascend, and so do the ring slots (TMEM columns) they accumulate
 // into, which lets one MMA of N = (taps)*Ntile serve several ring rows at once.
-__device__ __forceinline__ int weight_block(int ky, int Kh, int stride)
+__host__ __device__ __forceinline__ int weight_block(int ky, int Kh, int stride)
 {
     const int ph = ky % stride;
     int off = 0;
@@ -552,20 +558,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         s_abort = 0;
         s_issued = 0;
         if (!IDF_OK_AT(a.status, (bar_free - smem_u32(smem_raw)) + 8u * a.nslot - 1, a.smem_bytes)) s_abort = 1;
+        // The weights come first: they do not depend on earlier kernels of the stream (their fetch overlaps the
+        // previous kernel's tail under programmatic dependent launch), and a launch that brings a single row has
+        // little else to hide their latency behind.  One copy per K block carries all taps of the CTA's channel
+        // slice (the parameters are stored tap by tap in the order the stacked tiles want, see tc_pack_weights).
+        mbar_init(bar_w, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_expect_tx(bar_w, (uint32_t)(taps * a.n_kb) * w_tile_bytes);
+        for (int kb = 0; kb < a.n_kb; ++kb)
+            tma_load_3d(sW + (uint32_t)(kb * taps) * w_tile_bytes, &tmW, bar_w, kb * a.KB, n0, 0);
         for (int i = 0; i < a.nstage; ++i) { mbar_init(bar_full + 8u * i, 1); mbar_init(bar_empty + 8u * i, 1); }
-        for (int i = 0; i < taps; ++i) mbar_init(bar_w + 8u * i, 1);
         for (int i = 0; i < a.nslot; ++i) { mbar_init(bar_ready + 8u * i, 1); mbar_init(bar_free + 8u * i, 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        // The weights do not depend on earlier kernels of the stream: fetch them before waiting for
-        // the previous kernel (programmatic dependent launch), so the fetch overlaps its tail.
-        for (int kx = 0; kx < a.Kw; ++kx)
-            for (int ky = 0; ky < a.Kh; ++ky) {
-                const int tap = ky * a.Kw + kx;
-                mbar_expect_tx(bar_w + 8u * tap, (uint32_t)a.n_kb * w_tile_bytes);
-                for (int kb = 0; kb < a.n_kb; ++kb)
-                    tma_load_2d(sW + (uint32_t)((kx * a.n_kb + kb) * a.Kh + weight_block(ky, a.Kh, a.stride)) * w_tile_bytes,
-                                &tmW, bar_w + 8u * tap, kb * a.KB, tap * a.Cout + n0);
-            }
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)), "r"((uint32_t)a.tmem_cols) : "memory");
@@ -680,16 +684,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int n_kx = KX3 ? 3 : (a.shift_mode ? a.Kw : n_box);   // kx taps of a stage: row-shifted reads of one box, or one box each
             const int nslot = a.nslot;
             const uint32_t kx_bytes = (KSTEPS == 4 || a.shift_mode) ? (uint32_t)a.swb >> 4 : (uint32_t)a.a_box_pitch >> 4;
-            const uint32_t wtile_kx = ((uint32_t)(a.n_kb * a.Kh) * w_tile_bytes) >> 4;   // descriptor units per kx
-            const uint32_t wtile_kb = ((uint32_t)a.Kh * w_tile_bytes) >> 4;
+            // weight tiles in shared memory: [K block][kx][stacked ky block]
+            const uint32_t wtile_kx = ((uint32_t)a.Kh * w_tile_bytes) >> 4;              // descriptor units per kx
+            const uint32_t wtile_kb = ((uint32_t)taps * w_tile_bytes) >> 4;
             const uint32_t a_stage_units = a_stage_bytes >> 4;
             const int nstage = a.nstage, n_kb = a.n_kb;
             bool ok = true;
             // every slot this launch uses has been cleared once (a short launch visits fewer rows than there are slots)
             for (int slot = 0; slot < (c_n_orows < nslot ? c_n_orows : nslot) && ok; ++slot)
                 ok = mbar_wait(bar_free + 8u * slot, 0, abort_flag);
-            for (int tap = 0; tap < taps && ok; ++tap)            // the CTA's weight slice has landed
-                ok = mbar_wait(bar_w + 8u * tap, 0, abort_flag);
+            ok = ok && mbar_wait(bar_w, 0, abort_flag);          // the CTA's weight slice has landed
             const uint64_t adesc_base = desc_hi | (uint64_t)((sA & 0x3FFFFu) >> 4);
             const uint64_t bdesc_base = desc_hi | (uint64_t)((sW & 0x3FFFFu) >> 4);
             const int n_st = n_kb;                               // tiles (stages) per input row
@@ -843,10 +847,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int absp = (a.o_begin_par + c_oa) & 1;                // parity of the row's absolute index
         int pair_turn = (a.o_begin_half_mod + ((a.o_begin_par + c_oa) >> 1)) % G;   // (absolute index div 2) mod G
         int rslot_c = (a.ring_slot0 + c_oa) % a.ring_rows;    // absolute index mod ring_rows
+        int rslot_g = rslot_c % G;                            // ... mod G: the group that owns the ring slot
         for (int orel = 0; orel < c_n_orows && ok && grp < G; ++orel) {
             int owner;
             if (!a.pool) {
-                owner = (orel < n_cin || orel >= c_done_rel) ? 0 : turn;
+                // (rows that meet in one ring slot stay in one group, which takes them in order)
+                owner = (orel < n_cin || orel >= c_done_rel) ? rslot_g : turn;
             } else {
                 // both rows of a pooling pair go to one group; pairs touching the global ring or the pool layer's state
                 // (first < 0: the pair's first row came with an earlier launch) go to group 0
@@ -859,6 +865,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (++slot_c == a.nslot) { slot_c = 0; par_c ^= 1u; }
             if (++turn == G) turn = 0;
             if (++rslot_c == a.ring_rows) rslot_c = 0;
+            if (++rslot_g == G) rslot_g = 0;
+            if (rslot_c == 0) rslot_g = 0;
             if (absp && ++pair_turn == G) pair_turn = 0;
             absp ^= 1;
             if (owner != grp) continue;
@@ -960,8 +968,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (s_abort) {
         if (threadIdx.x == 0) {
             // let this CTA's own copies land before its shared memory is given back (bounded)
-            for (int tap = 0; tap < taps; ++tap)
-                for (uint32_t i = 0; i < 4096 && !mbar_try_wait(bar_w + 8u * tap, 0); ++i) __nanosleep(64);
+            for (uint32_t i = 0; i < 4096 && !mbar_try_wait(bar_w, 0); ++i) __nanosleep(64);
             const int issued = s_issued;
             for (int st = 0; st < a.nstage; ++st) {
                 int last = -1;
@@ -1430,16 +1437,22 @@ bool tc_make_plan(int dtype, int S, int Win, int Wout, int Cin, int Cout, int Kh
     return true;
 }
 
+// Where tap (ky, kx) of a layer goes in the tensor-core copy of its parameters, [tap'][Cout][Cin]: kx by kx, and
+// inside a kx the Kh tap rows in the order of the stacked weight tiles (weight_block), so that one copy delivers
+// a channel slice with all its taps in the shared-memory order the MMA schedule addresses.
+int tc_weight_slot(int ky, int kx, int Kh, int stride) { return kx * Kh + weight_block(ky, Kh, stride); }
+
 int tc_encode_weights(const TcPlan& p, int dtype, const void* d_w, int taps, int Cin, int Cout, void* map_out)
 {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return -1;
     const int esize = dtype == 1 ? 2 : 1;
-    cuuint64_t dims[2] = {(cuuint64_t)Cin, (cuuint64_t)taps * Cout};
-    cuuint64_t strides[1] = {(cuuint64_t)Cin * esize};
-    cuuint32_t box[2] = {(cuuint32_t)p.KB, (cuuint32_t)p.Ntile};
-    cuuint32_t es[2] = {1, 1};
-    CUresult r = enc((CUtensorMap*)map_out, dtype == 1 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
+    if (taps > 256) return -1;
+    cuuint64_t dims[3] = {(cuuint64_t)Cin, (cuuint64_t)Cout, (cuuint64_t)taps};
+    cuuint64_t strides[2] = {(cuuint64_t)Cin * esize, (cuuint64_t)Cout * Cin * esize};
+    cuuint32_t box[3] = {(cuuint32_t)p.KB, (cuuint32_t)p.Ntile, (cuuint32_t)taps};   // all taps of a channel slice and K block
+    cuuint32_t es[3] = {1, 1, 1};
+    CUresult r = enc((CUtensorMap*)map_out, dtype == 1 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 3,
                      const_cast<void*>(d_w), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(p.swb),
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? 0 : -1;
