@@ -357,6 +357,19 @@ __device__ __forceinline__ bool named_bar_and(int id, int count, bool pred)
 // Row finalisation of W accumulator columns of one (stream, x) position: add what earlier blocks
 // left in the ring, then either park the sum in the ring (row still open) or emit f(c + b) in the
 // layer's output type.
+// Ring rows in global memory are read and written 32 bytes per thread and instruction: a thread's run of channels
+// is its own, so narrower accesses would touch every 32-byte sector of the run twice.
+__device__ __forceinline__ void ld_global_v8(const void* p, uint32_t (&v)[8])
+{
+    asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]) : "l"(p));
+}
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&v)[8])
+{
+    asm volatile("st.global.v8.b32 [%8], {%0, %1, %2, %3, %4, %5, %6, %7};"
+                 :: "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "l"(p) : "memory");
+}
+
 template <int DT, int W, typename TS>
 __device__ __forceinline__ void finalise_chunk(const uint32_t (&v)[W], bool carried_in, bool emit, TS* rp,
                                                const TS* bias_c, const StageSink& sink, uint32_t col_byte, int out_elem,
@@ -366,32 +379,23 @@ __device__ __forceinline__ void finalise_chunk(const uint32_t (&v)[W], bool carr
 #pragma unroll
     for (int j = 0; j < W; ++j) acc[j] = DT == 1 ? (TS)__uint_as_float(v[j]) : (TS)(int)v[j];
     if (carried_in) {
-        const int4* p4 = (const int4*)(rp + carry_off);      // what earlier blocks left: the ring itself, or the launch's copy of it
+        const TS* p = rp + carry_off;                        // what earlier blocks left: the ring itself, or the launch's copy of it
+        uint32_t t[W / 8][8];
 #pragma unroll
-        for (int j4 = 0; j4 < W / 4; ++j4) {
-            const int4 t4 = p4[j4];
-            if (DT == 1) {
-                acc[4 * j4 + 0] += (TS)__int_as_float(t4.x); acc[4 * j4 + 1] += (TS)__int_as_float(t4.y);
-                acc[4 * j4 + 2] += (TS)__int_as_float(t4.z); acc[4 * j4 + 3] += (TS)__int_as_float(t4.w);
-            } else {
-                acc[4 * j4 + 0] += (TS)t4.x; acc[4 * j4 + 1] += (TS)t4.y;
-                acc[4 * j4 + 2] += (TS)t4.z; acc[4 * j4 + 3] += (TS)t4.w;
-            }
-        }
+        for (int j8 = 0; j8 < W / 8; ++j8) ld_global_v8(p + 8 * j8, t[j8]);
+#pragma unroll
+        for (int j8 = 0; j8 < W / 8; ++j8)
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                acc[8 * j8 + j] += DT == 1 ? (TS)__uint_as_float(t[j8][j]) : (TS)(int)t[j8][j];
     }
     if (!emit) {
-        int4* p4 = (int4*)rp;
 #pragma unroll
-        for (int j4 = 0; j4 < W / 4; ++j4) {
-            int4 t4;
-            if (DT == 1) {
-                t4.x = __float_as_int((float)acc[4 * j4 + 0]); t4.y = __float_as_int((float)acc[4 * j4 + 1]);
-                t4.z = __float_as_int((float)acc[4 * j4 + 2]); t4.w = __float_as_int((float)acc[4 * j4 + 3]);
-            } else {
-                t4.x = (int)acc[4 * j4 + 0]; t4.y = (int)acc[4 * j4 + 1];
-                t4.z = (int)acc[4 * j4 + 2]; t4.w = (int)acc[4 * j4 + 3];
-            }
-            p4[j4] = t4;
+        for (int j8 = 0; j8 < W / 8; ++j8) {
+            uint32_t t[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) t[j] = DT == 1 ? __float_as_uint((float)acc[8 * j8 + j]) : (uint32_t)(int)acc[8 * j8 + j];
+            st_global_v8(rp + 8 * j8, t);
         }
         return;
     }
