@@ -862,6 +862,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 // (first < 0: the pair's first row came with an earlier launch) go to group 0
                 const int first = orel - absp;
                 owner = (first < 0 || first < n_cin || first + 1 >= c_done_rel) ? 0 : pair_turn;
+                // a launch that emits at most one row has no pair to keep together and one row at most that touches the
+                // pool layer's state: its rows spread over the groups by ring slot as above
+                if (c_done_rel <= 1) owner = rslot_g;
             }
             const int slot = slot_c, rslot = rslot_c, row_odd = absp;
             const uint32_t par = par_c;
