@@ -277,7 +277,8 @@ def test_run_host_equals_device_path(orc, name, mode, rb):
     H, W = small_dims(name)
     C0 = next(l.cin for l in layers if l.kind == "conv")
     x, ws, bs = rand_net(mode, layers, H, W, C0, S=5, seed=21)
-    ref, _ = _run(mode, layers, x, ws, bs, row_block=rb, chunks=[rb] * H if rb else None, last=True)
+    # (run_host feeds the net half a row block at a time; fp32 sums depend on how the rows are grouped into pushes)
+    ref, _ = _run(mode, layers, x, ws, bs, row_block=rb, chunks=[max(rb // 2, 1)] * H if rb else None, last=True)
     net = idf.Net(mode, layers, W, C0, 5, ws, bs, row_block=rb)
     h_seg = idf.segments_from_maps(x, net.dtype).pin_memory()
     d_seg = torch.empty_like(h_seg, device="cuda")

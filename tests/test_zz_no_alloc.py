@@ -6,6 +6,8 @@ fixed memory pool, a real-time loop).  idf_conv_rows_noalloc serves them from a 
 inside the library.  Its results must equal those of the regular entry points, call after call,
 even though every call reuses the same scratch and finds the previous call's leftovers in it.
 """
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -30,6 +32,7 @@ def _noalloc(layer, x, w, b):
     rows = (H + 2 * layer.pad - layer.kh) // layer.stride + 1
     wo = 1 if x.shape[2] == 1 else (x.shape[2] + 2 * layer.pad - layer.kw) // layer.stride + 1
     out = torch.full((x.shape[0], rows, wo, layer.cout), float("nan"), device="cuda")
+    gc.collect()                                            # (tensors of earlier tests must not be freed in between)
     before = torch.cuda.memory_allocated()
     got_rows = idf.conv_rows_noalloc(seg, dw, db, layer.stride, layer.pad, bool(layer.relu), out)
     assert torch.cuda.memory_allocated() == before          # torch's allocator was not touched either
