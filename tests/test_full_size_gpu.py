@@ -48,6 +48,39 @@ def test_full_size_sampled_streams_match_oracle(orc, name, sample):
             assert_bf16_end_to_end(name, got, want, f"{name} stream {s}")
 
 
+@pytest.mark.parametrize("name,sample", [("vgg2d", [0, 63]), ("events2d", [5, 2047]), ("mnist2d", [0, 4095])])
+def test_full_size_one_segment_per_push_matches_oracle(orc, name, sample):
+    """The launch configuration of bench.py's `streaming` figure: all streams of the batch, one segment per push, the
+    last push carrying the end of input.  Every launch then brings one row: all rows exchange state with the ring
+    and spread over the epilogue groups by ring slot."""
+    w = workloads.get(name)
+    ws, bs = workloads.make_params(w)
+    net = idf.net_from_workload(w, ws, bs)
+    x = workloads.make_input(w)
+    seg = idf.segments_from_maps(x, w.dtype).cuda()
+    out = net.alloc_out(w.H)
+    net.open()
+    for r in range(w.H - 1):
+        net.push(seg[r:r + 1], out)
+    rows = net.push_last(seg[w.H - 1:], out)
+    net.status()
+    assert rows == net.out_shape(w.H)[0]
+    for s in sample:
+        want = orc.forward(w.dtype, w.layers, x[s:s + 1], ws, bs)[0]
+        got = out[s, :rows].cpu().numpy()
+        if w.dtype == "i8":
+            assert_equal(got, want, f"{name} stream {s}, one segment per push")
+        else:
+            assert_bf16_end_to_end(name, got, want, f"{name} stream {s}, one segment per push")
+    if w.dtype == "i8":
+        # integer nets: the grouping of segments into pushes changes nothing at all
+        whole = net.alloc_out(w.H)
+        net.reset()
+        assert net.push_last(seg, whole) == rows
+        assert torch.equal(whole[:, :rows], out[:, :rows])
+    net.close()
+
+
 def test_full_size_state_bytes_are_the_ring_formula():
     want = {"toy1d": 240, "mnist2d": 18432, "audio1d": 17024, "vgg2d": 1247232 + 14336, "events2d": 261248}
     for name, b in want.items():
