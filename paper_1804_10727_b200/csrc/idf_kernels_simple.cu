@@ -7,6 +7,8 @@
 //  pool_rows_kernel    2x2 max-pool fold with a one-row running maximum
 #include "idf_internal.h"
 
+#include <climits>
+
 namespace idf {
 
 __device__ __forceinline__ float to_acc(float v) { return v; }
@@ -382,6 +384,7 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
     // hide behind the arithmetic of the other); (B) the events are scattered into the ring.  The event
     // counter is double-buffered so that it can be cleared for the next pass while this one's is still read.
     int cb = 0;
+    int top_row = INT_MIN, top_slot = 0;             // 3x3 stride-1 scatter: the highest row the coming input row reaches, and its ring slot
     for (int rr = 0; rr <= n_in; ++rr) {
         // rr == n_in is the closing pass: no input, everything below done_end is finalised
         const bool have = rr < n_in;
@@ -390,7 +393,8 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
             // row o completes at input row o*stride - pad + Kh - 1, here: <= r - 1; relative to o_begin:
             // floor((r + pad - Kh) / stride) + 1 - o_begin, not below 0
             const int q = rr + c_q;
-            upto = q < 0 ? -((-q + a.stride - 1) / a.stride) + 1 : q / a.stride + 1;
+            if (a.stride == 1) upto = q + 1;           // (a division per row and thread costs as much as the scatter of an event)
+            else upto = q < 0 ? -((-q + a.stride - 1) / a.stride) + 1 : q / a.stride + 1;
             if (upto < 0) upto = 0;
             if (upto > done_end_rel) upto = done_end_rel;
         }
@@ -434,9 +438,24 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
             if (RING_IN_SMEM && w_in_smem && a.stride == 1 && a.stride_x == 1 && a.Kh == 3 && a.Kw == 3) {
                 // the common 3x3, stride-1 case with everything in shared memory, unrolled: the three target rows'
                 // slot offsets are worked out once per input row, a tap costs an address, a weight, a reduction
+                // (the slot of row ty0 steps with the input row: three runtime modulos per row and thread took longer than
+                // the events themselves)
                 int soff[3];
+                if (ty0 != top_row) { top_row = ty0; top_slot = ty0 >= 0 ? (slot0 + ty0) % a.ring_rows : 0; }
+                {
+                    int sl = top_slot;
 #pragma unroll
-                for (int ky = 0; ky < 3; ++ky) soff[ky] = ty0 - ky >= 0 ? ((slot0 + ty0 - ky) % a.ring_rows) * row_elems : -1;
+                    for (int ky = 0; ky < 3; ++ky) {
+                        soff[ky] = ty0 - ky >= 0 ? sl * row_elems : -1;
+                        if (--sl < 0) sl = a.ring_rows - 1;
+                    }
+                }
+                if (ty0 >= 0) {                                  // the next input row reaches one row further
+                    ++top_row;
+                    if (++top_slot == a.ring_rows) top_slot = 0;
+                } else {
+                    top_row = INT_MIN;
+                }
                 const int tap_w = a.Cin * a.Cout;
                 TS* ring_s = (TS*)smem_raw;
                 for (int e = tid >> 5; e < n_ev; e += SPARSE_THREADS / 32) {
