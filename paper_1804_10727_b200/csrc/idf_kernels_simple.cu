@@ -341,6 +341,17 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
                     const int rnd = a.shift > 0 ? 1 << (a.shift - 1) : 0;
                     const int4* src = (const int4*)(smem_raw) + (int)slot * (row_elems >> 2);
                     uint32_t* dst = (uint32_t*)orow;
+                    if (a.shift == 0) {
+                        // no requantisation shift (first layers fed with small integers): clamp and pack only
+                        for (int i = tid; i < (row_elems >> 2); i += SPARSE_THREADS) {
+                            const int4 c = src[i];
+                            ((int4*)src)[i] = make_int4(0, 0, 0, 0);
+                            uint32_t hi2, all4;
+                            asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(c.w), "r"(c.z));
+                            asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(all4) : "r"(c.y), "r"(c.x), "r"(hi2));
+                            dst[i] = __vminu4(all4, 0x7f7f7f7fu);
+                        }
+                    } else
                     for (int i = tid; i < (row_elems >> 2); i += SPARSE_THREADS) {
                         const int4 c = src[i];
                         ((int4*)src)[i] = make_int4(0, 0, 0, 0);
@@ -383,6 +394,7 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
     // while the rows that the PREVIOUS input row completed are finalised (independent work: the loads of one
     // hide behind the arithmetic of the other); (B) the events are scattered into the ring.  The event
     // counter is double-buffered so that it can be cleared for the next pass while this one's is still read.
+    const int cin_shift = (a.Cin & (a.Cin - 1)) == 0 ? 31 - __clz(a.Cin) : -1;     // (no division per event where Cin is a power of two)
     int cb = 0;
     int top_row = INT_MIN, top_slot = 0;             // 3x3 stride-1 scatter: the highest row the coming input row reaches, and its ring slot
     for (int rr = 0; rr <= n_in; ++rr) {
@@ -419,7 +431,7 @@ __global__ void __launch_bounds__(SPARSE_MAX_THREADS) conv_sparse_kernel(ConvArg
                         if (v != (TS)0) {
                             const int k = off + __popc(m & ((1u << lane) - 1u));
                             if (!IDF_OK_AT(a.status, k, SPARSE_MAX_EVENTS)) continue;
-                            const int x = i / a.Cin;
+                            const int x = cin_shift >= 0 ? i >> cin_shift : i / a.Cin;
                             ev_x[k] = (short)x;
                             ev_ci[k] = (short)(i - x * a.Cin);
                             ev_val[k] = v;
