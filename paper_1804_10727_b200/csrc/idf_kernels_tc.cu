@@ -262,6 +262,15 @@ __device__ __forceinline__ void tmem_st_zero(uint32_t taddr)
 }
 
 
+// 16 words of this thread's lane into 16 consecutive columns
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
+}
+
 // Where an emitted row goes first: a shared-memory tile [tile row][panel of pwb bytes], written in
 // the swizzle the output tensor map expects, from which one thread sends it out with a TMA store.
 struct StageSink {
@@ -371,24 +380,13 @@ __device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&v)[8])
 }
 
 template <int DT, int W, typename TS>
-__device__ __forceinline__ void finalise_chunk(const uint32_t (&v)[W], bool carried_in, bool emit, TS* rp,
+__device__ __forceinline__ void finalise_chunk(const uint32_t (&v)[W], bool emit, TS* rp,
                                                const TS* bias_c, const StageSink& sink, uint32_t col_byte, int out_elem,
-                                               int relu, int shift, const PoolCtx& pc, bool state_ok, long long carry_off)
+                                               int relu, int shift, const PoolCtx& pc, bool state_ok)
 {
     TS acc[W];
 #pragma unroll
     for (int j = 0; j < W; ++j) acc[j] = DT == 1 ? (TS)__uint_as_float(v[j]) : (TS)(int)v[j];
-    if (carried_in) {
-        const TS* p = rp + carry_off;                        // what earlier blocks left: the ring itself, or the launch's copy of it
-        uint32_t t[W / 8][8];
-#pragma unroll
-        for (int j8 = 0; j8 < W / 8; ++j8) ld_global_v8(p + 8 * j8, t[j8]);
-#pragma unroll
-        for (int j8 = 0; j8 < W / 8; ++j8)
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                acc[8 * j8 + j] += DT == 1 ? (TS)__uint_as_float(t[j8][j]) : (TS)(int)t[j8][j];
-    }
     if (!emit) {
 #pragma unroll
         for (int j8 = 0; j8 < W / 8; ++j8) {
@@ -804,7 +802,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const long long row_elems = (long long)a.Wout * a.Cout;
         TS* ring_pos = (TS*)a.ring + (long long)s * row_elems + (long long)x * a.Cout + n0;   // + ring slot * S * row_elems
         const long long ring_slot_stride = (long long)a.S * row_elems;
-        const long long carry_off = (const TS*)a.ring_in - (const TS*)a.ring;
         const uint32_t tlane = tmem_base + ((uint32_t)(q * 32) << 16);
         const int md = bs * a.BX + bx;                   // row of the dense output tile
         StageSink sink;
@@ -828,15 +825,42 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const bool state_ok = valid && (x >> 1) < wp;
         pc.state = (unsigned char*)a.pool_state + (((long long)s * wp + (x >> 1)) * a.Cout + n0) * a.out_esize;
         bool ok = true;
-        // every ring slot in tensor memory starts at zero (all MMAs accumulate)
-        if (grp == 0)
+        // Every ring slot in tensor memory starts from what its row has so far (all MMAs accumulate): zero, or, for a
+        // row begun by an earlier block, the partial sums that block left in the ring in global memory.  Taking those
+        // up here, while weights and the first rows are still on their way, keeps the ring's read latency out of the
+        // path between the last MMA and the emission; the three groups share the slots.
+        {
+            const long long carry_off0 = (const TS*)a.ring_in - (const TS*)a.ring;
+            int rs = (a.ring_slot0 + c_oa) % a.ring_rows;
             for (int slot = 0; slot < (c_n_orows < a.nslot ? c_n_orows : a.nslot); ++slot) {
-                for (int c = 0; c < a.Ntile; c += 16) tmem_st16_zero(tlane + (uint32_t)(slot * a.Ntile + c));
+                const int rslot = rs;
+                if (++rs == a.ring_rows) rs = 0;
+                if (slot % MAX_GROUPS != grp) continue;
+                bool carried = c_r0_positive && (slot * a.stride - c_base_ty < 0) && valid;
+                const TS* rp = ring_pos + (long long)rslot * ring_slot_stride + carry_off0;
+#ifdef IDF_BOUNDS
+                if (carried && !IDF_OK_AT(a.status, (rp - carry_off0 - (const TS*)a.ring) + a.Ntile - 1, a.ring_elems)) carried = false;
+#endif
+                for (int c = 0; c < a.Ntile; c += 16) {
+                    uint32_t v[16];
+                    if (carried) {
+                        uint32_t lo[8], hi[8];
+                        ld_global_v8(rp + c, lo);
+                        ld_global_v8(rp + c + 8, hi);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) { v[j] = lo[j]; v[8 + j] = hi[j]; }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) v[j] = 0u;
+                    }
+                    tmem_st16(tlane + (uint32_t)(slot * a.Ntile + c), v);
+                }
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_free + 8u * slot);   // one arrival per warp
             }
+        }
         // Rows that exchange state with the ring in global memory (those begun by an earlier block and
         // those left open by this one) may share a ring slot; group 0 takes them all, in order, so a
         // slot is read before it is rewritten.  The other rows go round the groups.
@@ -893,7 +917,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // (the barrier also makes the whole group leave together if any of its waits ran out)
             if (!named_bar_and(1 + grp, 128, got != 0)) { ok = false; break; }
             tc_fence_after();
-            const bool carried_in = c_r0_positive && (orel * a.stride - c_base_ty < 0);
             const bool pool_emit = a.pool && emit;
             if (pool_emit) {
                 pc.second = row_odd;
@@ -908,7 +931,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #ifdef IDF_BOUNDS
             {
                 fine = IDF_OK_AT(a.status, slot * a.Ntile + a.Ntile - 1, a.tmem_cols);
-                if (valid && (carried_in || !emit)) fine = fine && IDF_OK_AT(a.status, (rp - (TS*)a.ring) + a.Ntile - 1, a.ring_elems);
+                if (valid && !emit) fine = fine && IDF_OK_AT(a.status, (rp - (TS*)a.ring) + a.Ntile - 1, a.ring_elems);
                 if (pool_emit && state_ok && (pc.from_state || pc.to_state))
                     fine = fine && IDF_OK_AT(a.status, (pc.state - (unsigned char*)a.pool_state) + (long long)a.Ntile * a.out_esize - 1, a.pool_state_bytes);
                 // (a launch that emits pooled rows stages them in the half-size tile; the full-size addresses are not used then)
@@ -928,8 +951,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         tmem_ld_wait();
                         tmem_st_zero<32>(trow + c);           // the slot's next row starts from zero
                         if (pool_emit || (emit ? in_tile : valid))
-                            finalise_chunk<DT, 32, TS>(v, carried_in && valid, emit, rp + c, bias ? bias + c : nullptr, sink,
-                                                       (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift, pc, state_ok, carry_off);
+                            finalise_chunk<DT, 32, TS>(v, emit, rp + c, bias ? bias + c : nullptr, sink,
+                                                       (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift, pc, state_ok);
                     }
                 } else {
                     for (int c = 0; c < a.Ntile; c += 16) {
@@ -939,8 +962,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         tmem_ld_wait();
                         tmem_st_zero<16>(trow + c);
                         if (pool_emit || (emit ? in_tile : valid))
-                            finalise_chunk<DT, 16, TS>(v, carried_in && valid, emit, rp + c, bias ? bias + c : nullptr, sink,
-                                                       (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift, pc, state_ok, carry_off);
+                            finalise_chunk<DT, 16, TS>(v, emit, rp + c, bias ? bias + c : nullptr, sink,
+                                                       (uint32_t)(c * a.out_esize), a.out_elem, a.relu, a.shift, pc, state_ok);
                     }
                 }
                 tmem_st_wait();
@@ -1258,8 +1281,8 @@ conv_thin_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
                         tmem_ld<32>(trow + c, v);
                         tmem_ld_wait();
                         if (in_tile && fine)
-                            finalise_chunk<DT, 32, TS>(v, false, true, (TS*)nullptr, bias ? bias + c : nullptr, sink, (uint32_t)(c * a.out_esize),
-                                                       a.out_elem, a.relu, a.shift, pc, false, 0);
+                            finalise_chunk<DT, 32, TS>(v, true, (TS*)nullptr, bias ? bias + c : nullptr, sink, (uint32_t)(c * a.out_esize),
+                                                       a.out_elem, a.relu, a.shift, pc, false);
                     }
                 } else {
                     for (int c = 0; c < a.Cout; c += 16) {
@@ -1267,8 +1290,8 @@ conv_thin_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
                         tmem_ld<16>(trow + c, v);
                         tmem_ld_wait();
                         if (in_tile && fine)
-                            finalise_chunk<DT, 16, TS>(v, false, true, (TS*)nullptr, bias ? bias + c : nullptr, sink, (uint32_t)(c * a.out_esize),
-                                                       a.out_elem, a.relu, a.shift, pc, false, 0);
+                            finalise_chunk<DT, 16, TS>(v, true, (TS*)nullptr, bias ? bias + c : nullptr, sink, (uint32_t)(c * a.out_esize),
+                                                       a.out_elem, a.relu, a.shift, pc, false);
                     }
                 }
             }
