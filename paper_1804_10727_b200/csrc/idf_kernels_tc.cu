@@ -836,7 +836,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int rslot = rs;
                 if (++rs == a.ring_rows) rs = 0;
                 if (slot % MAX_GROUPS != grp) continue;
-                bool carried = c_r0_positive && (slot * a.stride - c_base_ty < 0) && valid;
+                // (carried_row is the same in all threads: the tensor-memory stores below are warp-wide instructions and
+                // every branch around them must be uniform; what differs per thread is only whether it has values to load)
+                const bool carried_row = c_r0_positive && (slot * a.stride - c_base_ty < 0);
+                bool carried = carried_row && valid;
                 const TS* rp = ring_pos + (long long)rslot * ring_slot_stride + carry_off0;
 #ifdef IDF_BOUNDS
                 if (carried && !IDF_OK_AT(a.status, (rp - carry_off0 - (const TS*)a.ring) + a.Ntile - 1, a.ring_elems)) carried = false;
@@ -853,6 +856,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                         for (int j = 0; j < 16; ++j) v[j] = 0u;
                     }
+                    __syncwarp();
                     tmem_st16(tlane + (uint32_t)(slot * a.Ntile + c), v);
                 }
                 tmem_st_wait();
@@ -861,9 +865,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (lane == 0) mbar_arrive(bar_free + 8u * slot);   // one arrival per warp
             }
         }
-        // Rows that exchange state with the ring in global memory (those begun by an earlier block and
-        // those left open by this one) may share a ring slot; group 0 takes them all, in order, so a
-        // slot is read before it is rewritten.  The other rows go round the groups.
+        // Rows left open by this block go back to the ring in global memory; those that meet in one ring slot stay in
+        // one group, in order.  (Rows begun by an earlier block were read above, before the first MMA, so nothing
+        // reads a ring slot any more once rows are written.)  The other rows go round the groups.
         const int n_cin = c_r0_positive ? (c_base_ty + a.stride - 1) / a.stride : 0;
         // Per-row bookkeeping is kept with small counters that step from row to row (a division or a 64-bit
         // operation per row and thread costs more than the row's arithmetic): TMEM slot and barrier parity of the row,
