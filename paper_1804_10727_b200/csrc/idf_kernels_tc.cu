@@ -951,6 +951,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int c = 0; c < a.Ntile; c += 32) {
                         uint32_t v[32];
                         if (!fine) continue;
+                        __syncwarp();                         // (the finalisation of the previous chunk is per thread)
                         tmem_ld<32>(trow + c, v);
                         tmem_ld_wait();
                         tmem_st_zero<32>(trow + c);           // the slot's next row starts from zero
@@ -962,6 +963,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int c = 0; c < a.Ntile; c += 16) {
                         uint32_t v[16];
                         if (!fine) continue;
+                        __syncwarp();
                         tmem_ld<16>(trow + c, v);
                         tmem_ld_wait();
                         tmem_st_zero<16>(trow + c);
