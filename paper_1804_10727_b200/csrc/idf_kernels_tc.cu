@@ -1284,6 +1284,7 @@ conv_thin_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
                 if ((a.Cout & 31) == 0) {
                     for (int c = 0; c < a.Cout; c += 32) {
                         uint32_t v[32];
+                        __syncwarp();
                         tmem_ld<32>(trow + c, v);
                         tmem_ld_wait();
                         if (in_tile && fine)
@@ -1293,6 +1294,7 @@ conv_thin_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
                 } else {
                     for (int c = 0; c < a.Cout; c += 16) {
                         uint32_t v[16];
+                        __syncwarp();
                         tmem_ld<16>(trow + c, v);
                         tmem_ld_wait();
                         if (in_tile && fine)
