@@ -581,12 +581,24 @@ __global__ void __launch_bounds__(256) unfold_rows_kernel(const T* __restrict__ 
     const int vecs = kpad / V;
     const long long total = n_pos * vecs;
     const bool vec_ok = (Cin % V) == 0 && (((uintptr_t)in) & 15) == 0;     // channels of a position in whole 16-byte groups
+    const bool small = total <= 0x7fffffffLL;
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (long long)gridDim.x * blockDim.x) {
-        const int v = (int)(idx % vecs);
-        const long long p = idx / vecs;              // (row, stream, x') flattened
-        const int xo = (int)(p % Wout);
-        const long long rs = p / Wout;               // (row, stream)
+        // (v, x', (row, stream)) of this 16-byte piece; in 32 bits where the launch allows: the four 64-bit divisions
+        // cost more than the copy
+        int v, xo;
+        long long p, rs;
+        if (small) {
+            const unsigned int i = (unsigned int)idx, pp = i / (unsigned int)vecs, r = pp / (unsigned int)Wout;
+            v = (int)(i - pp * (unsigned int)vecs);
+            xo = (int)(pp - r * (unsigned int)Wout);
+            p = pp; rs = r;
+        } else {
+            v = (int)(idx % vecs);
+            p = idx / vecs;                          // (row, stream, x') flattened
+            xo = (int)(p % Wout);
+            rs = p / Wout;                           // (row, stream)
+        }
         const T* row = in + rs * (long long)Win * Cin;
         __align__(16) T vals[V];
         if (vec_ok) {
