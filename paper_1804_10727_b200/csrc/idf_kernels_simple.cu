@@ -625,6 +625,43 @@ __global__ void __launch_bounds__(256) unfold_rows_kernel(const T* __restrict__ 
     }
 }
 
+// The same for layers whose positions are not whole 16-byte groups (three channels, say), where the kernel above would
+// fetch every value with a load of its own: a block takes one input row of one stream at a time, brings it into shared
+// memory with 16-byte loads, and every thread puts its 16-byte pieces together from there.
+constexpr int UNFOLD_ROW_BYTES = 16384;      // longest input row this form takes
+template <typename T>
+__global__ void __launch_bounds__(256) unfold_rows_staged_kernel(const T* __restrict__ in, T* __restrict__ out, int n_rs,
+                                                                 int Win, int Wout, int Cin, int Kw, int stride_x, int pad_x, int kpad,
+                                                                 long long in_elems, unsigned int* status)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    __shared__ __align__(16) unsigned char raw[UNFOLD_ROW_BYTES];
+    constexpr int V = 16 / (int)sizeof(T);
+    const int vecs = kpad / V;
+    const int row_elems = Win * Cin, n16 = row_elems * (int)sizeof(T) / 16, pieces = Wout * vecs;
+    const int k_all = Kw * Cin;
+    const T* rawT = (const T*)raw;
+    for (int rs = blockIdx.x; rs < n_rs; rs += gridDim.x) {
+        const T* row = in + (long long)rs * row_elems;
+        if (IDF_OK_AT(status, (long long)rs * row_elems + row_elems - 1, in_elems))
+            for (int i = threadIdx.x; i < n16; i += 256) ((int4*)raw)[i] = ((const int4*)row)[i];
+        __syncthreads();
+        T* orow = out + (long long)rs * Wout * kpad;
+        for (int pc = threadIdx.x; pc < pieces; pc += 256) {
+            const int xo = pc / vecs, v = pc - xo * vecs;
+            const int e0 = (xo * stride_x - pad_x) * Cin + v * V, k_end = k_all - v * V;
+            __align__(16) T vals[V];
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+                const int e = e0 + j;
+                vals[j] = (j < k_end && e >= 0 && e < row_elems) ? rawT[e] : (T)0;
+            }
+            ((int4*)orow)[pc] = *(const int4*)vals;
+        }
+        __syncthreads();
+    }
+}
+
 cudaError_t launch_unfold(const ConvArgs& a, int n_rows, int kpad, void* out, cudaStream_t st)
 {
     const long long n_pos = (long long)n_rows * a.S * a.Wout;
@@ -633,6 +670,22 @@ cudaError_t launch_unfold(const ConvArgs& a, int n_rows, int kpad, void* out, cu
     const long long total = n_pos * (kpad * esize / 16);
     long long blocks = (total + 255) / 256;
     if (blocks > 148LL * 32) blocks = 148LL * 32;
+    // rows whose positions are not whole 16-byte groups: staged through shared memory, a block per (row, stream)
+    const long long n_rs = (long long)n_rows * a.S;
+    const long long row_bytes = (long long)a.Win * a.Cin * esize;
+    if ((a.Cin * esize) % 16 != 0 && row_bytes % 16 == 0 && row_bytes <= UNFOLD_ROW_BYTES && (((uintptr_t)a.in) & 15) == 0 &&
+        n_rs <= 0x7fffffffLL && (long long)a.Wout * (kpad * esize / 16) <= 0x7fffffffLL) {
+        const unsigned grid = (unsigned)(n_rs < 148LL * 8 ? n_rs : 148LL * 8);
+        if (a.in_elem == E_BF16)
+            unfold_rows_staged_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)a.in, (__nv_bfloat16*)out, (int)n_rs, a.Win, a.Wout,
+                                                                         a.Cin, a.Kw, a.stride_x, a.pad_x, kpad, a.in_elems, a.status);
+        else if (a.in_elem == E_I8)
+            unfold_rows_staged_kernel<int8_t><<<grid, 256, 0, st>>>((const int8_t*)a.in, (int8_t*)out, (int)n_rs, a.Win, a.Wout, a.Cin, a.Kw,
+                                                                  a.stride_x, a.pad_x, kpad, a.in_elems, a.status);
+        else
+            return cudaErrorInvalidValue;
+        return cudaGetLastError();
+    }
     if (a.in_elem == E_BF16)
         unfold_rows_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)a.in, (__nv_bfloat16*)out, n_pos,
                                                                           a.Win, a.Wout, a.Cin, a.Kw, a.stride_x, a.pad_x, kpad, a.in_elems, a.status);
