@@ -230,9 +230,9 @@ int idf_stream_push_last(idf_net* net, const void* d_segments, int n_seg,
  * pinned) to d_segments, push every segment and the end of input (as idf_stream_push_last), copy the
  * completed output rows back to h_out ([n_streams][out_capacity_rows][out_w][out_c], host, ideally
  * pinned; rows beyond the last completed one are left as they are) and wait until all of it is done.
- * The work is pipelined over blocks of row_block segments: while one block is computed on the
- * handle's stream, the next one travels to the device and the output rows of the one before travel
- * back, on two copy streams the handle creates at its first idf_run_host (streams and events only,
+ * The work is pipelined over steps of row_block / 2 segments (the first and the last step half of
+ * that, so that the copies nothing overlaps are short): while one step is computed on the handle's
+ * stream, the next one travels to the device and the output rows of the one before travel back, on two copy streams the handle creates at its first idf_run_host (streams and events only,
  * no device memory) and orders after whatever was enqueued on the handle's stream before the call.
  * d_segments and d_out are device staging buffers of the same sizes, owned by the caller.  The handle
  * must be freshly opened or reset. */

@@ -1199,7 +1199,18 @@ int idf_run_host(idf_net* net, const void* h_segments, int n_seg, void* d_segmen
     // that nothing overlaps, and they shrink with the block, while the launches grow only a little more numerous
     // (vgg2d: 2.20 -> 1.98 ms per batch; a quarter block is slower again).
     const long long pipe = net->row_block >= 2 ? net->row_block / 2 : 1;
-    const long long nb = n_seg > 0 ? (n_seg + pipe - 1) / pipe : 1;
+    // ... and the first and the last step take half of that again when there are steps enough
+    std::vector<long long> cut;                      // segment index where step b starts; cut.back() = n_seg
+    {
+        const long long edge = (n_seg >= 3 * pipe && pipe >= 2) ? pipe / 2 : 0;
+        long long pos = 0;
+        cut.push_back(0);
+        if (edge) { pos = edge; cut.push_back(pos); }
+        while (pos < n_seg - edge) { pos = std::min<long long>(pos + pipe, n_seg - edge); cut.push_back(pos); }
+        if (edge) cut.push_back(n_seg);
+        if (cut.size() < 2) cut.push_back(n_seg);
+    }
+    const long long nb = (long long)cut.size() - 1;
     if (!net->copy_in) {
         if (cudaStreamCreateWithFlags(&net->copy_in, cudaStreamNonBlocking) != cudaSuccess ||
             cudaStreamCreateWithFlags(&net->copy_out, cudaStreamNonBlocking) != cudaSuccess)
@@ -1220,7 +1231,7 @@ int idf_run_host(idf_net* net, const void* h_segments, int n_seg, void* d_segmen
     if (e != cudaSuccess) return fail(IDF_ERR_CUDA, "run_host: %s", cudaGetErrorString(e));
     long long tot = 0, copied = 0;
     for (long long b = 0; b < nb; ++b) {
-        const long long s0 = b * pipe, n = std::min<long long>(pipe, n_seg - s0);
+        const long long s0 = cut[b], n = cut[b + 1] - cut[b];
         const bool last_block = b + 1 == nb;
         cudaEvent_t ev_in = net->order_events[1 + 2 * b], ev_done = net->order_events[2 + 2 * b];
         if (n > 0) {
