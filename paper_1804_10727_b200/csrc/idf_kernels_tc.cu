@@ -11,10 +11,12 @@
 //   - Δ-rows stream through a ring of shared-memory stages, one TMA box per (input row, kx, K block);
 //     the kx shift and the zero padding in x come from the box's start coordinate (out-of-range
 //     coordinates read zeros);
+//   - an accumulator starts from what its row has so far: zero, or, for a row begun by an earlier
+//     block, the partial sums that block left in the ring in global memory (copied in at the start
+//     of the launch);
 //   - when an input row was the last one an output row was waiting for, the epilogue warps read that
-//     accumulator, add what the ring held from earlier blocks and the bias, apply f, round or
-//     requantise, and write the row for the next layer; rows still open at the end of the block go
-//     back to the ring in global memory.
+//     accumulator, add the bias, apply f, round or requantise, and write the row for the next layer;
+//     rows still open at the end of the block go back to the ring in global memory.
 // Warp roles: warp 0 = TMA producer and row scheduler, warp 1 = TMEM owner and MMA issuer,
 // warps 2.. = epilogue groups of four warps (one warp per TMEM lane quarter) that take output rows in turn.
 // Every wait is bounded; on expiry the kernel records IDF_ERR_TIMEOUT in the status word and leaves.
